@@ -1,0 +1,304 @@
+"""Float64 CPU checker for the subsampled Gauss-Newton product path.
+
+TEST INFRASTRUCTURE ONLY.  This file is the plain, slow statement of what the
+CUDA library must compute, written from the paper ("Distributed Newton Methods
+for Deep Neural Networks", arXiv 1802.00130).  It shares no code with the CUDA
+path and must never be imported by it; only tests, the smoke check and the
+benchmark's CPU-baseline leg call it.
+
+Two tiers:
+
+* tier D ("definition"): explicit per-sample Jacobians J^i built with the
+  paper's backward recurrence (Section 3.3), the dense Gauss-Newton matrix
+  (Eq. def-gauss-newton / sampled-Gauss), its block-diagonal version
+  (Eq. gausshat) - tiny inputs only.
+* tier M ("matrix form"): the same quantities for all rows at once in float64
+  matrix form (forward directional derivative for J v, the back-propagation
+  equations of Section 2.2 for J^T u).  Usable at the paper's network sizes.
+
+Pins (see tests/test_oracle_pins.py): f(0) closed form, a hand-computed 2-1-1
+network, finite differences of f and of the network output, symmetry and
+positive-definiteness of G, the closed form of G for a network with no hidden
+layer, the exact-Hessian property in that case, tier M against tier D, dense
+solves for CG.  The paper prints no numeric worked example of f, grad f, J or
+G v, so beyond those pins the values are unpinned by the paper itself.
+
+Readings of the paper taken here (each is also listed in the design notes):
+biases are part of theta and are regularised (Section 3.2.1 sums (b_j)^2 into
+the regulariser); the loss has no 1/2 so B^i = 2I (Section 3.1); f and grad f
+average over all l rows, G^S over |S|; the Jacobian's backward pass starts from
+the identity (Eq. zLindependent) while the gradient's starts from 2(z^L - y)
+(Section 3.4); the block-diagonal blocks are the layers (split 1-1-...-1).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------- layout
+def num_params(widths):
+    """n = sum_m (n_{m-1} n_m + n_m)  (Section 2.1)."""
+    return sum(widths[m - 1] * widths[m] + widths[m] for m in range(1, len(widths)))
+
+
+def block_slices(widths):
+    """Coordinates of layer block m = (w^m, b^m) inside theta, m = 1..L."""
+    out, off = [], 0
+    for m in range(1, len(widths)):
+        size = widths[m - 1] * widths[m] + widths[m]
+        out.append(slice(off, off + size))
+        off += size
+    return out
+
+
+def unpack(theta, widths):
+    """theta -> [(W^m, b^m)], W^m of shape n_{m-1} x n_m.
+
+    w^m lists the columns of W^m one after another (Section 2.1): entry
+    w^m_{tj} sits at position j*n_{m-1} + t of the layer's weight run.
+    """
+    theta = np.asarray(theta, dtype=np.float64)
+    layers, off = [], 0
+    for m in range(1, len(widths)):
+        a, b = widths[m - 1], widths[m]
+        W = theta[off:off + a * b].reshape(b, a).T
+        off += a * b
+        bias = theta[off:off + b]
+        off += b
+        layers.append((W, bias))
+    assert off == theta.size
+    return layers
+
+
+def pack(layers):
+    """Inverse of `unpack`."""
+    parts = []
+    for W, b in layers:
+        parts.append(np.asarray(W, dtype=np.float64).T.reshape(-1))
+        parts.append(np.asarray(b, dtype=np.float64).reshape(-1))
+    return np.concatenate(parts)
+
+
+# --------------------------------------------------------------------------- forward, f, grad
+def sigmoid(s):
+    return 1.0 / (1.0 + np.exp(-s))
+
+
+def forward(theta, widths, X):
+    """Eq. (xtoz) with the activation of Section 3.3.2: returns [Z_0, ..., Z_L], rows = instances."""
+    layers = unpack(theta, widths)
+    L = len(layers)
+    Z = [np.asarray(X, dtype=np.float64)]
+    for m, (W, b) in enumerate(layers, start=1):
+        S = Z[-1] @ W + b
+        Z.append(sigmoid(S) if m < L else S)
+    return Z
+
+
+def fun(theta, widths, C, X, Y):
+    """Eq. (obj-function) with the squared loss of Eq. (thiswork-loss)."""
+    theta = np.asarray(theta, dtype=np.float64)
+    ZL = forward(theta, widths, X)[-1]
+    l = ZL.shape[0]
+    loss = np.sum((ZL - np.asarray(Y, dtype=np.float64)) ** 2)
+    return float(theta @ theta / (2.0 * C) + loss / l)
+
+
+def act_derivative(Z, m, L):
+    """sigma'(s^m) = z^m (1 - z^m) below the output layer, 1 at it (Section 3.3.2)."""
+    return Z[m] * (1.0 - Z[m]) if m < L else np.ones_like(Z[m])
+
+
+def backprop(theta, widths, Z, dZL):
+    """Eqs. (ztox-g)-(xtow-g-bias) without the 1/C and 1/l factors.
+
+    Given d xi / d z^L for every row, returns sum_i (J^i)^T (dZL row i) in theta layout.
+    """
+    layers = unpack(theta, widths)
+    L = len(layers)
+    out = [None] * L
+    dZ = dZL
+    for m in range(L, 0, -1):
+        W, _ = layers[m - 1]
+        dS = dZ * act_derivative(Z, m, L)              # (ztox-g)
+        gW = Z[m - 1].T @ dS                           # (xtow-g): sum_i z^{m-1}_t dS_j
+        gb = dS.sum(axis=0)                            # (xtow-g-bias)
+        out[m - 1] = (gW, gb)
+        if m > 1:
+            dZ = dS @ W.T                              # (communi-g)
+    return pack(out)
+
+
+def grad(theta, widths, C, X, Y):
+    """Eq. (whole-gradient); the backward pass starts from 2 (z^L - y) (Section 3.4)."""
+    theta = np.asarray(theta, dtype=np.float64)
+    Z = forward(theta, widths, X)
+    l = Z[0].shape[0]
+    dZL = 2.0 * (Z[-1] - np.asarray(Y, dtype=np.float64))
+    return theta / C + backprop(theta, widths, Z, dZL) / l
+
+
+# --------------------------------------------------------------------------- tier D
+def jacobian(theta, widths, x):
+    """Explicit J^i (n_L x n) for one instance by the backward recurrence of Section 3.3.
+
+    A^m[u, j] = d z^L_u / d z^m_j starts as the identity at m = L (Eq. zLindependent);
+    E^m = A^m diag(sigma'(s^m)) is d z^L_u / d s^m_j (Eq. ztox-jaco); the columns of J^i
+    for w^m_{tj} are E^m[:, j] z^{m-1}_t and for b^m_j are E^m[:, j] (Eqs. xtow-jaco,
+    xtow-jaco-bias); A^{m-1} = E^m (W^m)^T (Eq. communi-jaco).
+    """
+    layers = unpack(theta, widths)
+    L = len(layers)
+    Z = forward(theta, widths, np.asarray(x, dtype=np.float64).reshape(1, -1))
+    z = [a[0] for a in Z]
+    nL = widths[-1]
+    J = np.zeros((nL, num_params(widths)))
+    blocks = block_slices(widths)
+    A = np.eye(nL)
+    for m in range(L, 0, -1):
+        W, _ = layers[m - 1]
+        dsig = z[m] * (1.0 - z[m]) if m < L else np.ones(nL)
+        E = A * dsig[None, :]
+        a, b = widths[m - 1], widths[m]
+        off = blocks[m - 1].start
+        for u in range(nL):
+            for j in range(b):
+                for t in range(a):
+                    J[u, off + j * a + t] = E[u, j] * z[m - 1][t]
+                J[u, off + a * b + j] = E[u, j]
+        A = E @ W.T
+    return J
+
+
+def gauss_newton_dense(theta, widths, C, XS):
+    """G^S = I/C + (1/|S|) sum_{i in S} (J^i)^T B^i J^i with B^i = 2I (Eq. sampled-Gauss)."""
+    n = num_params(widths)
+    G = np.zeros((n, n))
+    for x in np.asarray(XS, dtype=np.float64):
+        J = jacobian(theta, widths, x)
+        G += J.T @ (2.0 * J)
+    return np.eye(n) / C + G / len(XS)
+
+
+def block_diagonal_of(G, widths):
+    """Eq. (gausshat): keep the diagonal layer blocks of a dense matrix, zero the rest."""
+    H = np.zeros_like(G)
+    for sl in block_slices(widths):
+        H[sl, sl] = G[sl, sl]
+    return H
+
+
+def Gv_definition(theta, widths, C, XS, v):
+    """G^S v accumulated sample by sample from explicit J^i (Eq. real-jaco with one partition)."""
+    v = np.asarray(v, dtype=np.float64)
+    acc = np.zeros_like(v)
+    for x in np.asarray(XS, dtype=np.float64):
+        J = jacobian(theta, widths, x)
+        acc += J.T @ (2.0 * (J @ v))
+    return v / C + acc / len(XS)
+
+
+def Gv_blockdiag_definition(theta, widths, C, XS, v):
+    """Eq. (approx-jaco): each layer block uses only its own columns J^i_p of J^i."""
+    v = np.asarray(v, dtype=np.float64)
+    acc = np.zeros_like(v)
+    blocks = block_slices(widths)
+    for x in np.asarray(XS, dtype=np.float64):
+        J = jacobian(theta, widths, x)
+        for sl in blocks:
+            Jp = J[:, sl]
+            acc[sl] += Jp.T @ (2.0 * (Jp @ v[sl]))
+    return v / C + acc / len(XS)
+
+
+# --------------------------------------------------------------------------- tier M
+def Jv(theta, widths, Z, v):
+    """J^i v for every row at once: the directional derivative of Eq. (xtoz) along v.
+
+    With v = (V^1, c^1, ..., V^L, c^L) in theta layout,
+    R s^m = R z^{m-1} W^m + z^{m-1} V^m + c^m and R z^m = sigma'(s^m) * R s^m, R z^0 = 0.
+    Summing the per-layer terms is the sum over partitions of Eq. (real-jaco).
+    """
+    layers = unpack(theta, widths)
+    dirs = unpack(v, widths)
+    L = len(layers)
+    RZ = np.zeros_like(Z[0])
+    for m in range(1, L + 1):
+        W, _ = layers[m - 1]
+        V, c = dirs[m - 1]
+        RS = RZ @ W + Z[m - 1] @ V + c
+        RZ = RS * act_derivative(Z, m, L)
+    return RZ
+
+
+def Gv(theta, widths, C, XS, v):
+    """Eq. (sampled-Gauss) applied to v: v/C + (1/|S|) J^T (2 J v)."""
+    v = np.asarray(v, dtype=np.float64)
+    Z = forward(theta, widths, XS)
+    U = 2.0 * Jv(theta, widths, Z, v)                       # B^i = 2I
+    return v / C + backprop(theta, widths, Z, U) / Z[0].shape[0]
+
+
+def Gv_blockdiag(theta, widths, C, XS, v):
+    """Eq. (approx-jaco) with one block per layer: block m sees only its own part of v and
+    keeps only its own part of J^T (2 J_m v_m)."""
+    v = np.asarray(v, dtype=np.float64)
+    Z = forward(theta, widths, XS)
+    rows = Z[0].shape[0]
+    out = v / C
+    for sl in block_slices(widths):
+        vm = np.zeros_like(v)
+        vm[sl] = v[sl]
+        U = 2.0 * Jv(theta, widths, Z, vm)
+        out[sl] += backprop(theta, widths, Z, U)[sl] / rows
+    return out
+
+
+# --------------------------------------------------------------------------- CG
+def cg(matvec, g, lam, max_iter, tol, segments=None):
+    """Conjugate gradient on (A + lam I) d = -g, d_0 = 0, no preconditioner.
+
+    Stop rule of Eq. (CG-stopping-cond): ||(A + lam I) d + g|| <= tol ||g|| (the left side
+    is the CG residual norm) or `max_iter` steps.  `segments` (list of slices) runs the
+    independent systems of Eq. (p-linear) side by side: every scalar is per segment and a
+    segment that met its stop rule is frozen.  Returns (d, iterates, resnorms) where
+    resnorms[k][s] is segment s's residual norm after k steps.
+    """
+    g = np.asarray(g, dtype=np.float64)
+    if segments is None:
+        segments = [slice(0, g.size)]
+    d = np.zeros_like(g)
+    r = -g.copy()
+    p = r.copy()
+    rho = np.array([r[s] @ r[s] for s in segments])
+    gnorm = np.sqrt(rho.copy())
+    active = np.array([tol <= 0 or np.sqrt(rho[k]) > tol * gnorm[k] for k in range(len(segments))])
+    active &= rho > 0
+    iterates, resnorms = [], [np.sqrt(rho.copy())]
+    it = 0
+    while it < max_iter and active.any():
+        q = matvec(p) + lam * p
+        for k, s in enumerate(segments):
+            if not active[k]:
+                continue
+            alpha = rho[k] / (p[s] @ q[s])
+            d[s] += alpha * p[s]
+            r[s] -= alpha * q[s]
+            rho_new = r[s] @ r[s]
+            beta = rho_new / rho[k]
+            p[s] = r[s] + beta * p[s]
+            rho[k] = rho_new
+            if tol > 0 and np.sqrt(rho_new) <= tol * gnorm[k]:
+                active[k] = False
+        it += 1
+        iterates.append(d.copy())
+        resnorms.append(np.sqrt(rho.copy()))
+    return d, iterates, resnorms
+
+
+def cg_solve(theta, widths, C, XS, g, lam, blockdiag, max_iter, tol):
+    """CG on the full system (Eq. sample-gaussnewton) or the per-layer systems (Eq. block-gaussnewton)."""
+    if blockdiag:
+        return cg(lambda p: Gv_blockdiag(theta, widths, C, XS, p), g, lam, max_iter, tol,
+                  segments=block_slices(widths))
+    return cg(lambda p: Gv(theta, widths, C, XS, p), g, lam, max_iter, tol)
