@@ -1,0 +1,189 @@
+/*
+ * gn.h - C ABI of the subsampled Gauss-Newton product library for fully-connected networks
+ *        on one NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates, for the regularised squared-loss network problem of
+ * "Distributed Newton Methods for Deep Neural Networks" (arXiv 1802.00130),
+ *
+ *     f(theta)  = theta^T theta / (2C) + (1/l) sum_i || z^{L,i} - y^i ||^2           (Eq. obj-function)
+ *     grad f    = theta / C + (1/l) sum_i (J^i)^T 2 (z^{L,i} - y^i)                  (Eq. whole-gradient)
+ *     G^S v     = v / C + (1/|S|) sum_{i in S} (J^i)^T B^i J^i v,   B^i = 2 I        (Eq. sampled-Gauss)
+ *     Ghat^S v  = the same with J^i replaced, block by block, by the columns that
+ *                 belong to one layer (w^m, b^m)                                      (Eq. approx-jaco)
+ *
+ * and runs conjugate gradient on (G^S + lambda I) d = -g (Eq. sample-gaussnewton) or on the
+ * independent per-layer systems (Eq. block-gaussnewton).
+ *
+ * Network (Section 2.1, Section 3.3.2): widths n_0-n_1-...-n_L; s^m = (W^m)^T z^{m-1} + b^m;
+ * z^m = 1/(1+exp(-s^m)) for m < L and z^L = s^L.
+ *
+ * LAYOUTS.  All matrices are dense, row-major, 32-bit IEEE floats.
+ *   theta, v, out, grad, g, d  [n], n = sum_m (n_{m-1} n_m + n_m): for m = 1..L the columns of W^m
+ *                              one after another (entry w^m_{tj} at j*n_{m-1} + t of the layer's
+ *                              run), then b^m (Section 2.1).  Biases are part of theta: they are
+ *                              regularised and the I/C term of G acts on them too.
+ *   X [l][n_0], Y [l][n_L]     one row per training instance; Y rows are the label vectors y^i.
+ *   idx [|S|]                  32-bit row numbers in [0, l); repeated rows are allowed and count
+ *                              once per occurrence (1/|S| uses the array length).
+ *
+ * POINTERS.  A parameter named d_* is a DEVICE pointer on the context's GPU, h_* a HOST pointer.
+ * Device pointers must be 4-byte aligned; 16-byte alignment enables the vectorised paths.
+ *
+ * OWNERSHIP.  The caller owns every buffer it passes.  dX and dY are borrowed for the lifetime of
+ * the context and never written.  theta and idx are copied when set, so the caller may reuse its
+ * buffers as soon as the call returns.  Input and output vectors of one call must not overlap.
+ * All workspaces (activations, CG vectors, reduction scratch) belong to the context and are
+ * released by gn_destroy.
+ *
+ * STREAMS.  Every kernel and copy is enqueued on the stream given to gn_create.  Calls that return
+ * host values (gn_fun, gn_grad with f_host, gn_cg_solve, every *_host variant) synchronise that
+ * stream before returning; the others only enqueue.  A context is not thread-safe.
+ *
+ * ERRORS.  Every call returns a gn_status and never throws or aborts.  Arguments are checked before
+ * anything is launched.  gn_last_error gives a human-readable reason for the most recent failure.
+ * There is no CPU fallback: without a usable CUDA device gn_create fails with GN_ECUDA.
+ */
+#ifndef GN_H_
+#define GN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gn_ctx gn_ctx; /* opaque */
+
+typedef enum {
+  GN_OK = 0,
+  GN_EINVAL = 1,  /* bad argument (null pointer, non-positive size, index out of range, ...)   */
+  GN_ENOMEM = 2,  /* a device or host allocation failed                                         */
+  GN_ECUDA = 3,   /* a CUDA call or kernel failed; gn_last_error has the CUDA message           */
+  GN_ESTATE = 4,  /* call sequence: theta / subsample not set, or stored activations are stale  */
+  GN_ETIMEOUT = 5 /* a bounded device-side wait ran out (tensor-core pipeline); results invalid */
+} gn_status;
+
+typedef enum {
+  GN_TF32 = 0,         /* contractions on the tensor cores with TF32 operands, FP32 accumulate   */
+  GN_FP32_ACCURATE = 1 /* contractions in full FP32 (fused multiply-add on the FP32 pipes)      */
+} gn_precision;
+
+/*
+ * gn_create - describe the problem of Eq. (obj-function): network widths, C, and the training set.
+ *   out          receives the context (set to NULL on failure).
+ *   L            number of weight layers (>= 1); widths has L+1 entries n_0..n_L, all >= 1.
+ *   C            regularisation parameter, > 0.
+ *   l            number of training rows, >= 1.
+ *   dX, dY       device, [l][n_0] and [l][n_L], borrowed.
+ *   prec         arithmetic of the contractions.
+ *   cuda_stream  a cudaStream_t (NULL = the legacy default stream).
+ * Errors: GN_EINVAL for bad arguments, GN_ECUDA if no device / wrong architecture, GN_ENOMEM.
+ */
+gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_t l,
+                    const float* dX, const float* dY, gn_precision prec, void* cuda_stream);
+
+/* gn_destroy - release the context and every workspace; NULL is accepted. */
+gn_status gn_destroy(gn_ctx* ctx);
+
+/* gn_num_params - n of Section 2.1, or -1 for a NULL context. */
+int64_t gn_num_params(const gn_ctx* ctx);
+
+/* gn_last_error - reason for the last non-OK status of this context ("" if none). */
+const char* gn_last_error(const gn_ctx* ctx);
+
+/* gn_workspace_bytes - device memory currently owned by the context. */
+int64_t gn_workspace_bytes(const gn_ctx* ctx);
+
+/*
+ * gn_set_batch_rows - number of rows processed at a time by gn_fun / gn_grad, which walk the
+ * training set in row batches so that their workspace stays bounded (the single-GPU form of the
+ * mini-batch pipelining of Section 6.1).  rows >= 1; values above l are clamped.  Default 32768.
+ */
+gn_status gn_set_batch_rows(gn_ctx* ctx, int64_t rows);
+
+/*
+ * gn_set_theta - copy the model vector (Section 2.1 layout) into the context.  Activations stored
+ * by an earlier gn_set_subsample become stale: products return GN_ESTATE until the subsample is
+ * set again.
+ */
+gn_status gn_set_theta(gn_ctx* ctx, const float* d_theta);
+gn_status gn_set_theta_host(gn_ctx* ctx, const float* h_theta);
+
+/*
+ * gn_set_subsample - choose S (Section 4.3): copies idx, checks every entry on the device
+ * (GN_EINVAL and no out-of-range read if one is outside [0, l)), gathers X_S = X[idx, :] and runs
+ * the stored forward pass Z_m = sigma(Z_{m-1} W^m + 1 (b^m)^T), m = 1..L (Eq. xtoz), keeping all
+ * Z_m for the products.  Needs theta.  nS >= 1.  Synchronises the stream (to report bad indices).
+ */
+gn_status gn_set_subsample(gn_ctx* ctx, const int32_t* d_idx, int64_t nS);
+gn_status gn_set_subsample_host(gn_ctx* ctx, const int32_t* h_idx, int64_t nS);
+
+/*
+ * gn_fun - f(theta) over all l rows (Eq. obj-function, Eq. thiswork-loss).  Needs theta.
+ * The sum over rows and theta^T theta are accumulated in double precision.
+ */
+gn_status gn_fun(gn_ctx* ctx, double* f_host);
+
+/*
+ * gn_grad - grad f over all l rows (Eq. whole-gradient; back-propagation of Eqs. ztox-g to
+ * xtow-g-bias starting from 2 (z^L - y), Section 3.4).  Writes d_grad [n]; if f_host is not NULL
+ * also returns f from the same forward pass (and synchronises).
+ */
+gn_status gn_grad(gn_ctx* ctx, float* d_grad, double* f_host);
+gn_status gn_grad_host(gn_ctx* ctx, float* h_grad, double* f_host);
+
+/*
+ * gn_Gv - out = G^S v (Eq. sampled-Gauss, no lambda): forward directional-derivative pass for
+ * J v (R s^m = R z^{m-1} W^m + z^{m-1} V^m + c^m, R z^m = sigma'(s^m) R s^m), multiply by B = 2I
+ * (Section 3.1), backward pass for J^T (.) (Section 4.2), then v/C + (1/|S|)(.).
+ * Needs theta and a current subsample.  d_v, d_out: device [n], not overlapping.
+ */
+gn_status gn_Gv(gn_ctx* ctx, const float* d_v, float* d_out);
+gn_status gn_Gv_host(gn_ctx* ctx, const float* h_v, float* h_out);
+
+/*
+ * gn_Gv_blockdiag - out = Ghat^S v (Eq. gausshat / approx-jaco) with one block per layer
+ * (w^m, b^m): block m of the result is v_m/C + (1/|S|) sum_i (J^i_m)^T 2 J^i_m v_m.
+ */
+gn_status gn_Gv_blockdiag(gn_ctx* ctx, const float* d_v, float* d_out);
+gn_status gn_Gv_blockdiag_host(gn_ctx* ctx, const float* h_v, float* h_out);
+
+/*
+ * gn_cg_solve - conjugate gradient for (A + lambda I) d = -g, A = G^S (blockdiag == 0, Eq.
+ * sample-gaussnewton) or A = Ghat^S (blockdiag != 0, Eq. block-gaussnewton).  Starts from d = 0,
+ * no preconditioner.  With blockdiag the L layer systems are solved side by side, each with its
+ * own step lengths and its own stop test; a block that has met its test is frozen.
+ *   d_g            device [n], the right-hand side's negative (the gradient).
+ *   lambda         >= 0 (the Levenberg-Marquardt term of Eq. full-gaussnewton).
+ *   max_iter       >= 1, the cap on CG steps (the paper uses 250).
+ *   tol            sigma of Eq. (CG-stopping-cond): stop once ||(A + lambda I) d + g|| <= tol ||g||
+ *                  (per block with blockdiag); tol <= 0 runs exactly max_iter steps.
+ *   d_d            device [n], receives d.
+ *   iters_host     optional, receives the number of steps taken.
+ *   d_iterates     optional device [max_iter][n]: row k receives d after step k+1.
+ *   resnorm_host   optional host [max_iter+1]: entry k is the residual norm after k steps
+ *                  (over all coordinates).
+ * Synchronises the stream once per step (the stop test is taken on the host).
+ */
+gn_status gn_cg_solve(gn_ctx* ctx, const float* d_g, double lambda, int blockdiag, int max_iter,
+                      double tol, float* d_d, int* iters_host, float* d_iterates,
+                      double* resnorm_host);
+gn_status gn_cg_solve_host(gn_ctx* ctx, const float* h_g, double lambda, int blockdiag,
+                           int max_iter, double tol, float* h_d, int* iters_host,
+                           double* resnorm_host);
+
+/*
+ * gn_debug_activations - copy the stored Z_m (m in 1..L, [|S|][n_m]) of the current subsample to a
+ * device buffer; a test hook for the stored forward pass (Eq. xtoz).
+ */
+gn_status gn_debug_activations(gn_ctx* ctx, int m, float* d_out);
+
+/*
+ * gn_kernel_launches - number of kernels this context has launched so far (all entry points).
+ */
+int64_t gn_kernel_launches(const gn_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GN_H_ */

@@ -1,0 +1,227 @@
+"""ctypes binding for include/gn.h.  Names mirror the C entry points (gn_Gv -> GnContext.Gv, ...)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+GN_TF32 = 0
+GN_FP32_ACCURATE = 1
+_STATUS = {0: "GN_OK", 1: "GN_EINVAL", 2: "GN_ENOMEM", 3: "GN_ECUDA", 4: "GN_ESTATE", 5: "GN_ETIMEOUT"}
+
+_vp, _i32, _i64, _dbl = C.c_void_p, C.c_int32, C.c_int64, C.c_double
+_SIGNATURES = {
+    "gn_create": (_i32, [C.POINTER(_vp), _i32, C.POINTER(_i32), _dbl, _i64, _vp, _vp, _i32, _vp]),
+    "gn_destroy": (_i32, [_vp]),
+    "gn_num_params": (_i64, [_vp]),
+    "gn_last_error": (C.c_char_p, [_vp]),
+    "gn_workspace_bytes": (_i64, [_vp]),
+    "gn_kernel_launches": (_i64, [_vp]),
+    "gn_set_batch_rows": (_i32, [_vp, _i64]),
+    "gn_set_theta": (_i32, [_vp, _vp]),
+    "gn_set_theta_host": (_i32, [_vp, _vp]),
+    "gn_set_subsample": (_i32, [_vp, _vp, _i64]),
+    "gn_set_subsample_host": (_i32, [_vp, _vp, _i64]),
+    "gn_fun": (_i32, [_vp, C.POINTER(_dbl)]),
+    "gn_grad": (_i32, [_vp, _vp, C.POINTER(_dbl)]),
+    "gn_grad_host": (_i32, [_vp, _vp, C.POINTER(_dbl)]),
+    "gn_Gv": (_i32, [_vp, _vp, _vp]),
+    "gn_Gv_host": (_i32, [_vp, _vp, _vp]),
+    "gn_Gv_blockdiag": (_i32, [_vp, _vp, _vp]),
+    "gn_Gv_blockdiag_host": (_i32, [_vp, _vp, _vp]),
+    "gn_cg_solve": (_i32, [_vp, _vp, _dbl, _i32, _i32, _dbl, _vp, C.POINTER(_i32), _vp, C.POINTER(_dbl)]),
+    "gn_cg_solve_host": (_i32, [_vp, _vp, _dbl, _i32, _i32, _dbl, _vp, C.POINTER(_i32), C.POINTER(_dbl)]),
+    "gn_debug_activations": (_i32, [_vp, _i32, _vp]),
+}
+
+
+class GnError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__(f"{_STATUS.get(status, status)}: {message}")
+        self.status = status
+
+
+_lib = None
+
+
+def lib_path():
+    return _build.LIB
+
+
+def exported_symbols():
+    return sorted(_SIGNATURES)
+
+
+def lib():
+    """Load libgn_b200.so (building it if the sources are newer).  Fails loudly if it cannot."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        handle = C.CDLL(path)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)          # AttributeError if the symbol is missing
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def _dev_ptr(t, dtype, count=None):
+    import torch
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("expected a CUDA tensor")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"expected a contiguous {dtype} tensor")
+    if count is not None and t.numel() != count:
+        raise ValueError(f"expected {count} elements, got {t.numel()}")
+    return _vp(t.data_ptr())
+
+
+def _host_ptr(a, dtype, count=None):
+    if not isinstance(a, np.ndarray) or a.dtype != dtype or not a.flags.c_contiguous:
+        raise TypeError(f"expected a C-contiguous numpy array of {dtype}")
+    if count is not None and a.size != count:
+        raise ValueError(f"expected {count} elements, got {a.size}")
+    return _vp(a.ctypes.data)
+
+
+class GnContext:
+    """One problem (widths, C, X, Y) on the current CUDA device; wraps a gn_ctx."""
+
+    def __init__(self, widths, C_reg, X, Y, precision=GN_FP32_ACCURATE, stream=None):
+        import torch
+        self._lib = lib()
+        self.widths = [int(w) for w in widths]
+        L = len(self.widths) - 1
+        l = X.shape[0]
+        if X.dim() != 2 or Y.dim() != 2 or X.shape[1] != self.widths[0] or Y.shape != (l, self.widths[-1]):
+            raise ValueError("X must be [l][n_0] and Y [l][n_L]")
+        self._X, self._Y = X, Y                 # borrowed by the library: keep them alive
+        self._stream = stream if stream is not None else torch.cuda.current_stream(X.device)
+        arr = (_i32 * (L + 1))(*self.widths)
+        handle = _vp()
+        st = self._lib.gn_create(C.byref(handle), L, arr, float(C_reg), l, _dev_ptr(X, torch.float32),
+                                 _dev_ptr(Y, torch.float32), int(precision), _vp(self._stream.cuda_stream))
+        if st != 0:
+            raise GnError(st, "gn_create failed (needs an sm_100 device and valid arguments)")
+        self._h = handle
+        self.n = int(self._lib.gn_num_params(self._h))
+        self.device = X.device
+
+    # ------------------------------------------------------------------ helpers
+    def _check(self, st):
+        if st != 0:
+            raise GnError(st, self._lib.gn_last_error(self._h).decode())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.gn_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _new(self, count=None):
+        import torch
+        return torch.empty(self.n if count is None else count, dtype=torch.float32, device=self.device)
+
+    @property
+    def workspace_bytes(self):
+        return int(self._lib.gn_workspace_bytes(self._h))
+
+    @property
+    def kernel_launches(self):
+        return int(self._lib.gn_kernel_launches(self._h))
+
+    # ------------------------------------------------------------------ entry points
+    def set_batch_rows(self, rows):
+        self._check(self._lib.gn_set_batch_rows(self._h, int(rows)))
+
+    def set_theta(self, theta):
+        import torch
+        self._check(self._lib.gn_set_theta(self._h, _dev_ptr(theta, torch.float32, self.n)))
+
+    def set_theta_host(self, theta):
+        self._check(self._lib.gn_set_theta_host(self._h, _host_ptr(theta, np.float32, self.n)))
+
+    def set_subsample(self, idx):
+        import torch
+        self._check(self._lib.gn_set_subsample(self._h, _dev_ptr(idx, torch.int32), idx.numel()))
+        self.nS = idx.numel()
+
+    def set_subsample_host(self, idx):
+        self._check(self._lib.gn_set_subsample_host(self._h, _host_ptr(idx, np.int32), idx.size))
+        self.nS = idx.size
+
+    def fun(self):
+        f = _dbl()
+        self._check(self._lib.gn_fun(self._h, C.byref(f)))
+        return f.value
+
+    def grad(self, out=None, with_f=False):
+        import torch
+        out = self._new() if out is None else out
+        f = _dbl()
+        self._check(self._lib.gn_grad(self._h, _dev_ptr(out, torch.float32, self.n), C.byref(f) if with_f else None))
+        return (out, f.value) if with_f else out
+
+    def grad_host(self, out=None, with_f=False):
+        out = np.empty(self.n, dtype=np.float32) if out is None else out
+        f = _dbl()
+        self._check(self._lib.gn_grad_host(self._h, _host_ptr(out, np.float32, self.n), C.byref(f) if with_f else None))
+        return (out, f.value) if with_f else out
+
+    def Gv(self, v, out=None):
+        import torch
+        out = self._new() if out is None else out
+        self._check(self._lib.gn_Gv(self._h, _dev_ptr(v, torch.float32, self.n), _dev_ptr(out, torch.float32, self.n)))
+        return out
+
+    def Gv_blockdiag(self, v, out=None):
+        import torch
+        out = self._new() if out is None else out
+        self._check(self._lib.gn_Gv_blockdiag(self._h, _dev_ptr(v, torch.float32, self.n),
+                                              _dev_ptr(out, torch.float32, self.n)))
+        return out
+
+    def Gv_host(self, v, out=None, blockdiag=False):
+        out = np.empty(self.n, dtype=np.float32) if out is None else out
+        fn = self._lib.gn_Gv_blockdiag_host if blockdiag else self._lib.gn_Gv_host
+        self._check(fn(self._h, _host_ptr(v, np.float32, self.n), _host_ptr(out, np.float32, self.n)))
+        return out
+
+    def cg_solve(self, g, lam, blockdiag=False, max_iter=250, tol=1e-3, out=None, keep_iterates=False):
+        """Returns (d, iters, resnorms[, iterates])."""
+        import torch
+        out = self._new() if out is None else out
+        its = _i32()
+        res = (_dbl * (max_iter + 1))()
+        iterates = self._new(max_iter * self.n) if keep_iterates else None
+        self._check(self._lib.gn_cg_solve(
+            self._h, _dev_ptr(g, torch.float32, self.n), float(lam), int(bool(blockdiag)), int(max_iter), float(tol),
+            _dev_ptr(out, torch.float32, self.n), C.byref(its),
+            _dev_ptr(iterates, torch.float32) if keep_iterates else None, res))
+        resn = np.array(res[: its.value + 1])
+        if keep_iterates:
+            return out, its.value, resn, iterates.view(max_iter, self.n)[: its.value]
+        return out, its.value, resn
+
+    def cg_solve_host(self, g, lam, blockdiag=False, max_iter=250, tol=1e-3, out=None):
+        out = np.empty(self.n, dtype=np.float32) if out is None else out
+        its = _i32()
+        res = (_dbl * (max_iter + 1))()
+        self._check(self._lib.gn_cg_solve_host(
+            self._h, _host_ptr(g, np.float32, self.n), float(lam), int(bool(blockdiag)), int(max_iter), float(tol),
+            _host_ptr(out, np.float32, self.n), C.byref(its), res))
+        return out, its.value, np.array(res[: its.value + 1])
+
+    def debug_activations(self, m):
+        import torch
+        out = torch.empty(self.nS * self.widths[m], dtype=torch.float32, device=self.device)
+        self._check(self._lib.gn_debug_activations(self._h, int(m), _dev_ptr(out, torch.float32)))
+        return out.view(self.nS, self.widths[m])

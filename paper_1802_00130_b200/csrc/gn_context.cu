@@ -1,0 +1,611 @@
+// Host side of the C ABI (include/gn.h): context, workspaces, and the launch sequences for the
+// stored forward pass, f / gradient over row batches, the full and block-diagonal Gauss-Newton
+// products, and conjugate gradient.
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/gn.h"
+#include "gn_kernels.h"
+
+using namespace gn;
+
+struct gn_ctx {
+  int L = 0;
+  std::vector<int> w;               // n_0..n_L
+  double C = 1.0;
+  int64_t l = 0;
+  const float* dX = nullptr;
+  const float* dY = nullptr;
+  gn_precision prec = GN_FP32_ACCURATE;
+  cudaStream_t st = nullptr;
+  int64_t n = 0;
+  std::vector<int64_t> w_off, b_off;  // [m], m = 1..L (entry 0 unused)
+  int64_t batch_rows = 32768;
+  bool have_theta = false, have_sub = false;
+
+  float* theta = nullptr;
+  // subsample
+  int64_t nS = 0, capS = 0;
+  int32_t* idx = nullptr;
+  std::vector<float*> Z;    // Z[0] = X_S, Z[m] = [nS][n_m]
+  std::vector<float*> RZ;   // RZ[m] = [m * nS][n_m]: forward directional derivatives (stacked streams)
+  std::vector<float*> DS;   // DS[m] = [m * nS][n_m]: backward quantities d(.)/d s^m
+  // row-batch workspace of f / grad
+  int64_t capB = 0;
+  std::vector<float*> Zb, Db;
+  // reductions
+  float* colsum_scratch = nullptr; int64_t colsum_cap = 0;
+  double* partial = nullptr; int64_t partial_cap = 0;
+  double* dscal = nullptr;   // device: [0] loss, [1] theta^T theta, [2] cg sum rho, [3] cg active
+  double* hscal = nullptr;   // pinned mirror
+  int* err_flag = nullptr;
+  int* h_err = nullptr;      // pinned
+  // CG
+  float* cg_r = nullptr; float* cg_p = nullptr; float* cg_q = nullptr;
+  float* tmp_a = nullptr; float* tmp_b = nullptr;  // staging for *_host calls
+  CgChunk* chunks[2] = {nullptr, nullptr}; int n_chunks[2] = {0, 0};
+  CgSeg* segs = nullptr;
+
+  int64_t bytes = 0;
+  int64_t launches = 0;
+  std::string err;
+  std::vector<void*> owned;
+};
+
+namespace {
+
+gn_status fail(gn_ctx* c, gn_status s, const std::string& msg) {
+  if (c) c->err = msg;
+  return s;
+}
+
+gn_status cuda_fail(gn_ctx* c, cudaError_t e, const char* where) {
+  return fail(c, e == cudaErrorMemoryAllocation ? GN_ENOMEM : GN_ECUDA,
+              std::string(where) + ": " + cudaGetErrorString(e));
+}
+
+#define GN_CUDA(c, call)                                          \
+  do {                                                            \
+    cudaError_t e__ = (call);                                     \
+    if (e__ != cudaSuccess) return cuda_fail((c), e__, #call);    \
+  } while (0)
+
+#define GN_TRY(expr)                      \
+  do {                                    \
+    gn_status s__ = (expr);               \
+    if (s__ != GN_OK) return s__;         \
+  } while (0)
+
+template <class T>
+gn_status dev_alloc(gn_ctx* c, T** p, int64_t count) {
+  *p = nullptr;
+  if (count <= 0) count = 1;
+  void* q = nullptr;
+  cudaError_t e = cudaMalloc(&q, (size_t)count * sizeof(T));
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(c, GN_ENOMEM, std::string("cudaMalloc of ") + std::to_string(count * (int64_t)sizeof(T)) + " bytes: " + cudaGetErrorString(e));
+  }
+  c->bytes += count * (int64_t)sizeof(T);
+  c->owned.push_back(q);
+  *p = static_cast<T*>(q);
+  return GN_OK;
+}
+
+template <class T>
+void dev_free(gn_ctx* c, T*& p, int64_t count) {
+  if (!p) return;
+  for (auto& o : c->owned)
+    if (o == (void*)p) { o = nullptr; break; }
+  cudaFree(p);
+  c->bytes -= (count <= 0 ? 1 : count) * (int64_t)sizeof(T);
+  p = nullptr;
+}
+
+gn_status check_launch(gn_ctx* c, const char* where) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(c, e, where);
+  return GN_OK;
+}
+
+gn_status sync(gn_ctx* c, const char* where) {
+  cudaError_t e = cudaStreamSynchronize(c->st);
+  if (e != cudaSuccess) return cuda_fail(c, e, where);
+  return GN_OK;
+}
+
+void run_gemm(gn_ctx* c, const GemmArgs& g) {
+  c->launches += launch_gemm_ffma(g, c->st);
+}
+
+gn_status ensure_partials(gn_ctx* c, int64_t count) {
+  if (count <= c->partial_cap) return GN_OK;
+  dev_free(c, c->partial, c->partial_cap);
+  c->partial_cap = 0;
+  GN_TRY(dev_alloc(c, &c->partial, count));
+  c->partial_cap = count;
+  return GN_OK;
+}
+
+gn_status ensure_colsum(gn_ctx* c, int64_t rows, int cols) {
+  const int64_t need = colsum_scratch_floats(rows, cols);
+  if (need <= c->colsum_cap) return GN_OK;
+  dev_free(c, c->colsum_scratch, c->colsum_cap);
+  c->colsum_cap = 0;
+  GN_TRY(dev_alloc(c, &c->colsum_scratch, need));
+  c->colsum_cap = need;
+  return GN_OK;
+}
+
+const float* Wm(const gn_ctx* c, const float* vec, int m) { return vec + c->w_off[m]; }
+const float* bm(const gn_ctx* c, const float* vec, int m) { return vec + c->b_off[m]; }
+
+// Eq. (xtoz): Zout[m] = sigma(Zout[m-1] W^m + 1 b^mT), m = 1..L, over `rows` rows; Zout[0] = Z0.
+void forward_pass(gn_ctx* c, const float* Z0, int64_t rows, std::vector<float*>& Zout) {
+  for (int m = 1; m <= c->L; ++m) {
+    GemmArgs g;
+    g.M = (int)rows; g.N = c->w[m];
+    g.A1 = m == 1 ? Z0 : Zout[m - 1]; g.lda1 = c->w[m - 1];
+    g.B1 = Wm(c, c->theta, m); g.ldb1 = c->w[m - 1]; g.K1 = c->w[m - 1];
+    g.a_kmajor = true; g.b_kmajor = true;
+    g.D = Zout[m]; g.ldd = c->w[m];
+    g.bias = bm(c, c->theta, m);
+    g.sigmoid = m < c->L;
+    run_gemm(c, g);
+  }
+}
+
+// Parameter-space half of the backward pass for one layer (Eqs. xtow-g, xtow-g-bias, and their
+// Jacobian twins of Section 4.2): out_W = alpha ds^T Zprev + beta cin_W, out_b = alpha 1^T ds + beta cin_b.
+gn_status weight_block(gn_ctx* c, int m, const float* ds, const float* Zprev, int64_t rows, float alpha,
+                       const float* cin, float beta, float* out) {
+  GemmArgs g;
+  g.M = c->w[m]; g.N = c->w[m - 1];
+  g.A1 = ds; g.lda1 = c->w[m]; g.a_kmajor = false;
+  g.B1 = Zprev; g.ldb1 = c->w[m - 1]; g.b_kmajor = false;
+  g.K1 = (int)rows;
+  g.alpha = alpha;
+  g.cin = cin + c->w_off[m]; g.ld_cin = c->w[m - 1]; g.beta = beta;
+  g.D = out + c->w_off[m]; g.ldd = c->w[m - 1];
+  run_gemm(c, g);
+  GN_TRY(ensure_colsum(c, rows, c->w[m]));
+  c->launches += launch_colsum(ds, rows, c->w[m], c->w[m], alpha, cin + c->b_off[m], beta, out + c->b_off[m],
+                               c->colsum_scratch, c->st);
+  return GN_OK;
+}
+
+// Activation-space half (Eq. communi-g / communi-jaco followed by Eq. ztox-g):
+// dst = (ds W^mT) * sigma'(z^{m-1}), rows stacked modulo z_rows.
+void backward_data(gn_ctx* c, int m, const float* ds, int64_t rows, const float* Zprev, int64_t z_rows, float* dst) {
+  GemmArgs g;
+  g.M = (int)rows; g.N = c->w[m - 1];
+  g.A1 = ds; g.lda1 = c->w[m]; g.a_kmajor = true;
+  g.B1 = Wm(c, c->theta, m); g.ldb1 = c->w[m - 1]; g.b_kmajor = false;
+  g.K1 = c->w[m];
+  g.dsig = Zprev; g.ld_dsig = c->w[m - 1]; g.dsig_rows = (int)z_rows;
+  g.D = dst; g.ldd = c->w[m - 1];
+  run_gemm(c, g);
+}
+
+// out = coef v + (1/|S|) J^T (2 J v) over the stored subsample (Eq. sampled-Gauss).
+gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
+  const int L = c->L;
+  const int64_t nS = c->nS;
+  for (int m = 1; m <= L; ++m) {
+    GemmArgs g;
+    g.M = (int)nS; g.N = c->w[m];
+    if (m == 1) {
+      g.A1 = c->Z[0]; g.lda1 = c->w[0]; g.B1 = Wm(c, v, 1); g.ldb1 = c->w[0]; g.K1 = c->w[0];
+    } else {
+      g.A1 = c->RZ[m - 1]; g.lda1 = c->w[m - 1]; g.B1 = Wm(c, c->theta, m); g.ldb1 = c->w[m - 1]; g.K1 = c->w[m - 1];
+      g.A2 = c->Z[m - 1];  g.lda2 = c->w[m - 1]; g.B2 = Wm(c, v, m);        g.ldb2 = c->w[m - 1]; g.K2 = c->w[m - 1];
+    }
+    g.bias = bm(c, v, m);
+    if (m < L) { g.dsig = c->Z[m]; g.ld_dsig = c->w[m]; g.dsig_rows = (int)nS; }
+    else g.alpha = 2.f;                                   // B = 2I
+    g.D = c->RZ[m]; g.ldd = c->w[m];
+    run_gemm(c, g);
+  }
+  const float* ds = c->RZ[L];
+  const float inv = (float)(1.0 / (double)nS);
+  for (int m = L; m >= 1; --m) {
+    GN_TRY(weight_block(c, m, ds, c->Z[m - 1], nS, inv, v, coef, out));
+    if (m > 1) {
+      backward_data(c, m, ds, nS, c->Z[m - 1], nS, c->DS[m - 1]);
+      ds = c->DS[m - 1];
+    }
+  }
+  return check_launch(c, "G v");
+}
+
+// Eq. (approx-jaco), one block per layer.  The perturbation of layer k is pushed to the output and
+// pulled back to layer k only; the L streams are stacked along rows, stream j occupying rows
+// [(j-1)|S|, j|S|) of every buffer at or above layer j, so each layer runs one stacked GEMM.
+gn_status product_blockdiag(gn_ctx* c, const float* v, float* out, float coef) {
+  const int L = c->L;
+  const int64_t nS = c->nS;
+  for (int k = 1; k <= L; ++k) {
+    if (k > 1) {
+      GemmArgs g;
+      g.M = (int)((k - 1) * nS); g.N = c->w[k];
+      g.A1 = c->RZ[k - 1]; g.lda1 = c->w[k - 1]; g.B1 = Wm(c, c->theta, k); g.ldb1 = c->w[k - 1]; g.K1 = c->w[k - 1];
+      if (k < L) { g.dsig = c->Z[k]; g.ld_dsig = c->w[k]; g.dsig_rows = (int)nS; }
+      else g.alpha = 2.f;
+      g.D = c->RZ[k]; g.ldd = c->w[k];
+      run_gemm(c, g);
+    }
+    GemmArgs g;
+    g.M = (int)nS; g.N = c->w[k];
+    g.A1 = c->Z[k - 1]; g.lda1 = c->w[k - 1]; g.B1 = Wm(c, v, k); g.ldb1 = c->w[k - 1]; g.K1 = c->w[k - 1];
+    g.bias = bm(c, v, k);
+    if (k < L) { g.dsig = c->Z[k]; g.ld_dsig = c->w[k]; g.dsig_rows = (int)nS; }
+    else g.alpha = 2.f;
+    g.D = c->RZ[k] + (k - 1) * nS * c->w[k]; g.ldd = c->w[k];
+    run_gemm(c, g);
+  }
+  const float* cur = c->RZ[L];
+  const float inv = (float)(1.0 / (double)nS);
+  for (int k = L; k >= 1; --k) {
+    const float* dsk = cur + (k - 1) * nS * c->w[k];
+    GN_TRY(weight_block(c, k, dsk, c->Z[k - 1], nS, inv, v, coef, out));
+    if (k > 1) {
+      backward_data(c, k, cur, (k - 1) * nS, c->Z[k - 1], nS, c->DS[k - 1]);
+      cur = c->DS[k - 1];
+    }
+  }
+  return check_launch(c, "block-diagonal G v");
+}
+
+gn_status ensure_batch(gn_ctx* c) {
+  const int64_t rows = c->batch_rows < c->l ? c->batch_rows : c->l;
+  if (rows <= c->capB) return GN_OK;
+  for (int m = 1; m <= c->L; ++m) { dev_free(c, c->Zb[m], c->capB * c->w[m]); dev_free(c, c->Db[m], c->capB * c->w[m]); }
+  c->capB = 0;
+  for (int m = 1; m <= c->L; ++m) {
+    GN_TRY(dev_alloc(c, &c->Zb[m], rows * c->w[m]));
+    GN_TRY(dev_alloc(c, &c->Db[m], rows * c->w[m]));
+  }
+  c->capB = rows;
+  return GN_OK;
+}
+
+// f and (optionally) the gradient over all rows in row batches (Section 6.1 in its one-GPU form).
+gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
+  GN_TRY(ensure_batch(c));
+  const int L = c->L;
+  const int64_t Rb = c->capB;
+  const int64_t nb = (c->l + Rb - 1) / Rb;
+  const int64_t per_batch = loss_num_partials(Rb * c->w[L]);
+  GN_TRY(ensure_partials(c, per_batch * nb + (c->n + kCgChunk - 1) / kCgChunk + 16));
+  const float inv_l = (float)(1.0 / (double)c->l);
+  const float inv_C = (float)(1.0 / c->C);
+  for (int64_t b = 0; b < nb; ++b) {
+    const int64_t r0 = b * Rb;
+    const int64_t rows = (c->l - r0 < Rb) ? c->l - r0 : Rb;
+    const float* X0 = c->dX + r0 * c->w[0];
+    forward_pass(c, X0, rows, c->Zb);
+    c->launches += launch_loss_delta(c->Zb[L], c->dY + r0 * c->w[L], rows * c->w[L], d_grad ? c->Db[L] : nullptr,
+                                     c->partial + b * per_batch, c->st);
+    {
+      // only the last batch can be shorter than Rb: zero the partial slots it does not write
+      const int used = loss_num_partials(rows * c->w[L]);
+      if (used < per_batch)
+        GN_CUDA(c, cudaMemsetAsync(c->partial + b * per_batch + used, 0, (per_batch - used) * sizeof(double), c->st));
+    }
+    if (d_grad) {
+      for (int m = L; m >= 1; --m) {
+        const float* Zprev = m == 1 ? X0 : c->Zb[m - 1];
+        if (b == 0) GN_TRY(weight_block(c, m, c->Db[m], Zprev, rows, inv_l, c->theta, inv_C, d_grad));
+        else        GN_TRY(weight_block(c, m, c->Db[m], Zprev, rows, inv_l, d_grad, 1.f, d_grad));
+        if (m > 1) backward_data(c, m, c->Db[m], rows, c->Zb[m - 1], rows, c->Db[m - 1]);
+      }
+    }
+  }
+  if (f_host) {
+    c->launches += launch_sum_partials(c->partial, (int)(per_batch * nb), c->dscal + 0, false, c->st);
+    // theta^T theta with the CG dot kernel over the single-segment chunk table
+    double* tp = c->partial + per_batch * nb;
+    c->launches += launch_cg_dot(c->theta, c->theta, c->chunks[0], c->n_chunks[0], tp, c->st);
+    c->launches += launch_sum_partials(tp, c->n_chunks[0], c->dscal + 1, false, c->st);
+    GN_CUDA(c, cudaMemcpyAsync(c->hscal, c->dscal, 2 * sizeof(double), cudaMemcpyDeviceToHost, c->st));
+    GN_TRY(check_launch(c, "f / grad"));
+    GN_TRY(sync(c, "f / grad"));
+    *f_host = c->hscal[1] / (2.0 * c->C) + c->hscal[0] / (double)c->l;
+    return GN_OK;
+  }
+  return check_launch(c, "grad");
+}
+
+gn_status ensure_tmp(gn_ctx* c) {
+  if (!c->tmp_a) GN_TRY(dev_alloc(c, &c->tmp_a, c->n));
+  if (!c->tmp_b) GN_TRY(dev_alloc(c, &c->tmp_b, c->n));
+  return GN_OK;
+}
+
+gn_status need_product_state(gn_ctx* c) {
+  if (!c->have_theta) return fail(c, GN_ESTATE, "theta has not been set");
+  if (!c->have_sub) return fail(c, GN_ESTATE, "no current subsample (set it after theta)");
+  return GN_OK;
+}
+
+gn_status build_chunks(gn_ctx* c) {
+  for (int mode = 0; mode < 2; ++mode) {
+    std::vector<CgChunk> h;
+    const int n_seg = mode == 0 ? 1 : c->L;
+    for (int s = 0; s < n_seg; ++s) {
+      const int64_t a = mode == 0 ? 0 : c->w_off[s + 1];
+      const int64_t b = mode == 0 ? c->n : (s + 1 < c->L ? c->w_off[s + 2] : c->n);
+      for (int64_t k = a; k < b; k += kCgChunk) {
+        CgChunk ch;
+        ch.start = k; ch.len = (int32_t)((b - k < kCgChunk) ? b - k : kCgChunk); ch.seg = s;
+        h.push_back(ch);
+      }
+    }
+    c->n_chunks[mode] = (int)h.size();
+    GN_TRY(dev_alloc(c, &c->chunks[mode], (int64_t)h.size()));
+    GN_CUDA(c, cudaMemcpy(c->chunks[mode], h.data(), h.size() * sizeof(CgChunk), cudaMemcpyHostToDevice));
+  }
+  GN_TRY(dev_alloc(c, &c->segs, (int64_t)c->L));
+  return GN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_t l, const float* dX,
+                    const float* dY, gn_precision prec, void* cuda_stream) {
+  if (!out) return GN_EINVAL;
+  *out = nullptr;
+  if (L < 1 || L > 64 || !widths || !(C > 0.0) || l < 1 || !dX || !dY) return GN_EINVAL;
+  if (prec != GN_TF32 && prec != GN_FP32_ACCURATE) return GN_EINVAL;
+  for (int m = 0; m <= L; ++m)
+    if (widths[m] < 1) return GN_EINVAL;
+  if (l > 0x7fffffffLL) return GN_EINVAL;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return GN_ECUDA; }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { cudaGetLastError(); return GN_ECUDA; }
+  if (prop.major != 10) return GN_ECUDA;  // kernels are built for sm_100a only
+  gn_ctx* c = new (std::nothrow) gn_ctx();
+  if (!c) return GN_ENOMEM;
+  c->L = L;
+  c->w.assign(widths, widths + L + 1);
+  c->C = C; c->l = l; c->dX = dX; c->dY = dY; c->prec = prec;
+  c->st = static_cast<cudaStream_t>(cuda_stream);
+  c->w_off.assign(L + 2, 0); c->b_off.assign(L + 2, 0);
+  int64_t off = 0;
+  for (int m = 1; m <= L; ++m) {
+    c->w_off[m] = off; off += (int64_t)c->w[m - 1] * c->w[m];
+    c->b_off[m] = off; off += c->w[m];
+  }
+  c->n = off;
+  c->Z.assign(L + 1, nullptr); c->RZ.assign(L + 1, nullptr); c->DS.assign(L + 1, nullptr);
+  c->Zb.assign(L + 1, nullptr); c->Db.assign(L + 1, nullptr);
+  gn_status s = GN_OK;
+  do {
+    if ((s = dev_alloc(c, &c->theta, c->n)) != GN_OK) break;
+    if ((s = dev_alloc(c, &c->cg_r, c->n)) != GN_OK) break;
+    if ((s = dev_alloc(c, &c->cg_p, c->n)) != GN_OK) break;
+    if ((s = dev_alloc(c, &c->cg_q, c->n)) != GN_OK) break;
+    if ((s = dev_alloc(c, &c->dscal, 8)) != GN_OK) break;
+    if ((s = dev_alloc(c, &c->err_flag, 1)) != GN_OK) break;
+    if (cudaMallocHost(&c->hscal, 8 * sizeof(double)) != cudaSuccess) { s = GN_ENOMEM; break; }
+    if (cudaMallocHost(&c->h_err, sizeof(int)) != cudaSuccess) { s = GN_ENOMEM; break; }
+    if ((s = build_chunks(c)) != GN_OK) break;
+    if ((s = ensure_partials(c, 2 * (int64_t)c->n_chunks[1] + 64)) != GN_OK) break;
+  } while (0);
+  if (s != GN_OK) { gn_destroy(c); return s; }
+  *out = c;
+  return GN_OK;
+}
+
+gn_status gn_destroy(gn_ctx* c) {
+  if (!c) return GN_OK;
+  cudaStreamSynchronize(c->st);
+  for (void* p : c->owned)
+    if (p) cudaFree(p);
+  if (c->hscal) cudaFreeHost(c->hscal);
+  if (c->h_err) cudaFreeHost(c->h_err);
+  cudaGetLastError();
+  delete c;
+  return GN_OK;
+}
+
+int64_t gn_num_params(const gn_ctx* c) { return c ? c->n : -1; }
+const char* gn_last_error(const gn_ctx* c) { return c ? c->err.c_str() : "null context"; }
+int64_t gn_workspace_bytes(const gn_ctx* c) { return c ? c->bytes : -1; }
+int64_t gn_kernel_launches(const gn_ctx* c) { return c ? c->launches : -1; }
+
+gn_status gn_set_batch_rows(gn_ctx* c, int64_t rows) {
+  if (!c) return GN_EINVAL;
+  if (rows < 1) return fail(c, GN_EINVAL, "batch rows must be >= 1");
+  c->batch_rows = rows;
+  if ((rows < c->l ? rows : c->l) != c->capB && c->capB > 0) {
+    // shrink or grow on next use: drop the old workspace now so memory stays bounded
+    cudaStreamSynchronize(c->st);
+    for (int m = 1; m <= c->L; ++m) { dev_free(c, c->Zb[m], c->capB * c->w[m]); dev_free(c, c->Db[m], c->capB * c->w[m]); }
+    c->capB = 0;
+  }
+  return GN_OK;
+}
+
+gn_status gn_set_theta(gn_ctx* c, const float* d_theta) {
+  if (!c) return GN_EINVAL;
+  if (!d_theta) return fail(c, GN_EINVAL, "theta is NULL");
+  GN_CUDA(c, cudaMemcpyAsync(c->theta, d_theta, c->n * sizeof(float), cudaMemcpyDeviceToDevice, c->st));
+  c->have_theta = true;
+  c->have_sub = false;
+  return GN_OK;
+}
+
+gn_status gn_set_theta_host(gn_ctx* c, const float* h_theta) {
+  if (!c) return GN_EINVAL;
+  if (!h_theta) return fail(c, GN_EINVAL, "theta is NULL");
+  GN_CUDA(c, cudaMemcpyAsync(c->theta, h_theta, c->n * sizeof(float), cudaMemcpyHostToDevice, c->st));
+  GN_TRY(sync(c, "set_theta_host"));
+  c->have_theta = true;
+  c->have_sub = false;
+  return GN_OK;
+}
+
+static gn_status set_subsample_impl(gn_ctx* c, const int32_t* idx, int64_t nS, cudaMemcpyKind kind) {
+  if (!c) return GN_EINVAL;
+  if (!idx) return fail(c, GN_EINVAL, "idx is NULL");
+  if (nS < 1) return fail(c, GN_EINVAL, "the subsample must have at least one row");
+  if (!c->have_theta) return fail(c, GN_ESTATE, "theta has not been set");
+  if ((int64_t)c->L * nS > 65535LL * 128) return fail(c, GN_EINVAL, "L * |S| exceeds 8 388 480 rows");
+  c->have_sub = false;
+  if (nS > c->capS) {
+    GN_TRY(sync(c, "set_subsample"));
+    dev_free(c, c->idx, c->capS);
+    for (int m = 0; m <= c->L; ++m) dev_free(c, c->Z[m], c->capS * c->w[m]);
+    for (int m = 1; m <= c->L; ++m) { dev_free(c, c->RZ[m], m * c->capS * c->w[m]); dev_free(c, c->DS[m], m * c->capS * c->w[m]); }
+    c->capS = 0;
+    GN_TRY(dev_alloc(c, &c->idx, nS));
+    for (int m = 0; m <= c->L; ++m) GN_TRY(dev_alloc(c, &c->Z[m], nS * c->w[m]));
+    for (int m = 1; m <= c->L; ++m) {
+      GN_TRY(dev_alloc(c, &c->RZ[m], m * nS * c->w[m]));
+      if (m < c->L) GN_TRY(dev_alloc(c, &c->DS[m], m * nS * c->w[m]));
+    }
+    c->capS = nS;
+  }
+  c->nS = nS;
+  GN_CUDA(c, cudaMemcpyAsync(c->idx, idx, nS * sizeof(int32_t), kind, c->st));
+  GN_CUDA(c, cudaMemsetAsync(c->err_flag, 0, sizeof(int), c->st));
+  c->launches += launch_gather_rows(c->dX, c->l, c->w[0], c->idx, nS, c->Z[0], c->err_flag, c->st);
+  GN_CUDA(c, cudaMemcpyAsync(c->h_err, c->err_flag, sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  forward_pass(c, c->Z[0], nS, c->Z);
+  GN_TRY(check_launch(c, "set_subsample"));
+  GN_TRY(sync(c, "set_subsample"));
+  if (*c->h_err) return fail(c, GN_EINVAL, "a subsample index lies outside [0, l)");
+  c->have_sub = true;
+  return GN_OK;
+}
+
+gn_status gn_set_subsample(gn_ctx* c, const int32_t* d_idx, int64_t nS) {
+  return set_subsample_impl(c, d_idx, nS, cudaMemcpyDeviceToDevice);
+}
+gn_status gn_set_subsample_host(gn_ctx* c, const int32_t* h_idx, int64_t nS) {
+  return set_subsample_impl(c, h_idx, nS, cudaMemcpyHostToDevice);
+}
+
+gn_status gn_fun(gn_ctx* c, double* f_host) {
+  if (!c) return GN_EINVAL;
+  if (!f_host) return fail(c, GN_EINVAL, "f_host is NULL");
+  if (!c->have_theta) return fail(c, GN_ESTATE, "theta has not been set");
+  return fun_grad(c, nullptr, f_host);
+}
+
+gn_status gn_grad(gn_ctx* c, float* d_grad, double* f_host) {
+  if (!c) return GN_EINVAL;
+  if (!d_grad) return fail(c, GN_EINVAL, "grad is NULL");
+  if (!c->have_theta) return fail(c, GN_ESTATE, "theta has not been set");
+  return fun_grad(c, d_grad, f_host);
+}
+
+gn_status gn_grad_host(gn_ctx* c, float* h_grad, double* f_host) {
+  if (!c) return GN_EINVAL;
+  if (!h_grad) return fail(c, GN_EINVAL, "grad is NULL");
+  if (!c->have_theta) return fail(c, GN_ESTATE, "theta has not been set");
+  GN_TRY(ensure_tmp(c));
+  GN_TRY(fun_grad(c, c->tmp_b, f_host));
+  GN_CUDA(c, cudaMemcpyAsync(h_grad, c->tmp_b, c->n * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  return sync(c, "grad_host");
+}
+
+gn_status gn_Gv(gn_ctx* c, const float* d_v, float* d_out) {
+  if (!c) return GN_EINVAL;
+  if (!d_v || !d_out) return fail(c, GN_EINVAL, "v / out is NULL");
+  if (d_v == d_out) return fail(c, GN_EINVAL, "v and out must not overlap");
+  GN_TRY(need_product_state(c));
+  return product_full(c, d_v, d_out, (float)(1.0 / c->C));
+}
+
+gn_status gn_Gv_blockdiag(gn_ctx* c, const float* d_v, float* d_out) {
+  if (!c) return GN_EINVAL;
+  if (!d_v || !d_out) return fail(c, GN_EINVAL, "v / out is NULL");
+  if (d_v == d_out) return fail(c, GN_EINVAL, "v and out must not overlap");
+  GN_TRY(need_product_state(c));
+  return product_blockdiag(c, d_v, d_out, (float)(1.0 / c->C));
+}
+
+static gn_status product_host(gn_ctx* c, const float* h_v, float* h_out, bool blockdiag) {
+  if (!c) return GN_EINVAL;
+  if (!h_v || !h_out) return fail(c, GN_EINVAL, "v / out is NULL");
+  GN_TRY(need_product_state(c));
+  GN_TRY(ensure_tmp(c));
+  GN_CUDA(c, cudaMemcpyAsync(c->tmp_a, h_v, c->n * sizeof(float), cudaMemcpyHostToDevice, c->st));
+  const float coef = (float)(1.0 / c->C);
+  GN_TRY(blockdiag ? product_blockdiag(c, c->tmp_a, c->tmp_b, coef) : product_full(c, c->tmp_a, c->tmp_b, coef));
+  GN_CUDA(c, cudaMemcpyAsync(h_out, c->tmp_b, c->n * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  return sync(c, "product_host");
+}
+
+gn_status gn_Gv_host(gn_ctx* c, const float* h_v, float* h_out) { return product_host(c, h_v, h_out, false); }
+gn_status gn_Gv_blockdiag_host(gn_ctx* c, const float* h_v, float* h_out) { return product_host(c, h_v, h_out, true); }
+
+gn_status gn_cg_solve(gn_ctx* c, const float* d_g, double lambda, int blockdiag, int max_iter, double tol,
+                      float* d_d, int* iters_host, float* d_iterates, double* resnorm_host) {
+  if (!c) return GN_EINVAL;
+  if (!d_g || !d_d) return fail(c, GN_EINVAL, "g / d is NULL");
+  if (max_iter < 1) return fail(c, GN_EINVAL, "max_iter must be >= 1");
+  if (!(lambda >= 0.0)) return fail(c, GN_EINVAL, "lambda must be >= 0");
+  GN_TRY(need_product_state(c));
+  const int mode = blockdiag ? 1 : 0;
+  const int n_seg = blockdiag ? c->L : 1;
+  const CgChunk* ch = c->chunks[mode];
+  const int nc = c->n_chunks[mode];
+  const float coef = (float)(1.0 / c->C + lambda);
+  double* out2 = c->dscal + 2;
+
+  c->launches += launch_cg_init(d_g, d_d, c->cg_r, c->cg_p, ch, nc, c->partial, c->st);
+  c->launches += launch_cg_scalars(0, c->partial, ch, nc, c->segs, n_seg, tol, out2, c->st);
+  GN_CUDA(c, cudaMemcpyAsync(c->hscal + 2, out2, 2 * sizeof(double), cudaMemcpyDeviceToHost, c->st));
+  GN_TRY(check_launch(c, "cg init"));
+  GN_TRY(sync(c, "cg init"));
+  if (resnorm_host) resnorm_host[0] = sqrt(c->hscal[2]);
+  int it = 0;
+  while (it < max_iter && c->hscal[3] > 0.5) {
+    GN_TRY(blockdiag ? product_blockdiag(c, c->cg_p, c->cg_q, coef) : product_full(c, c->cg_p, c->cg_q, coef));
+    c->launches += launch_cg_dot(c->cg_p, c->cg_q, ch, nc, c->partial, c->st);
+    c->launches += launch_cg_scalars(1, c->partial, ch, nc, c->segs, n_seg, tol, out2, c->st);
+    c->launches += launch_cg_update(c->cg_p, c->cg_q, d_d, c->cg_r, ch, nc, c->segs, c->partial, c->st);
+    c->launches += launch_cg_scalars(2, c->partial, ch, nc, c->segs, n_seg, tol, out2, c->st);
+    c->launches += launch_cg_direction(c->cg_r, c->cg_p, ch, nc, c->segs, c->st);
+    GN_CUDA(c, cudaMemcpyAsync(c->hscal + 2, out2, 2 * sizeof(double), cudaMemcpyDeviceToHost, c->st));
+    if (d_iterates)
+      GN_CUDA(c, cudaMemcpyAsync(d_iterates + (int64_t)it * c->n, d_d, c->n * sizeof(float), cudaMemcpyDeviceToDevice, c->st));
+    GN_TRY(check_launch(c, "cg step"));
+    GN_TRY(sync(c, "cg step"));
+    ++it;
+    if (resnorm_host) resnorm_host[it] = sqrt(c->hscal[2]);
+  }
+  if (iters_host) *iters_host = it;
+  return GN_OK;
+}
+
+gn_status gn_cg_solve_host(gn_ctx* c, const float* h_g, double lambda, int blockdiag, int max_iter, double tol,
+                           float* h_d, int* iters_host, double* resnorm_host) {
+  if (!c) return GN_EINVAL;
+  if (!h_g || !h_d) return fail(c, GN_EINVAL, "g / d is NULL");
+  GN_TRY(need_product_state(c));
+  GN_TRY(ensure_tmp(c));
+  GN_CUDA(c, cudaMemcpyAsync(c->tmp_a, h_g, c->n * sizeof(float), cudaMemcpyHostToDevice, c->st));
+  GN_TRY(gn_cg_solve(c, c->tmp_a, lambda, blockdiag, max_iter, tol, c->tmp_b, iters_host, nullptr, resnorm_host));
+  GN_CUDA(c, cudaMemcpyAsync(h_d, c->tmp_b, c->n * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  return sync(c, "cg_solve_host");
+}
+
+gn_status gn_debug_activations(gn_ctx* c, int m, float* d_out) {
+  if (!c) return GN_EINVAL;
+  if (!d_out || m < 1 || m > c->L) return fail(c, GN_EINVAL, "bad layer / NULL output");
+  GN_TRY(need_product_state(c));
+  GN_CUDA(c, cudaMemcpyAsync(d_out, c->Z[m], c->nS * c->w[m] * sizeof(float), cudaMemcpyDeviceToDevice, c->st));
+  return GN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,96 @@
+// Internal launch interface between the host logic (gn_context.cu) and the kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gn {
+
+// One dense contraction with a fused epilogue:
+//
+//   acc[m][n] = sum_k A1(m,k) B1(k,n)  (+ sum_k A2(m,k) B2(k,n) when A2 != nullptr)
+//   t = acc + bias[n]                   (bias != nullptr)
+//   t = 1 / (1 + exp(-t))               (sigmoid)
+//   t = t * zc (1 - zc)                 (dsig != nullptr; zc = dsig[(m % dsig_rows) * ld_dsig + n])
+//   t = alpha * t
+//   t = t + beta * cin[m * ld_cin + n]  (cin != nullptr)
+//   D[m * ldd + n] = t
+//
+// A operands: a_kmajor -> A(m,k) = A[m * lda + k], else A(m,k) = A[k * lda + m].
+// B operands: b_kmajor -> B(k,n) = B[n * ldb + k], else B(k,n) = B[k * ldb + n].
+// Both pairs share layouts but have their own K and leading dimensions.
+struct GemmArgs {
+  int M = 0, N = 0;
+  const float* A1 = nullptr; const float* B1 = nullptr; int K1 = 0; int64_t lda1 = 0, ldb1 = 0;
+  const float* A2 = nullptr; const float* B2 = nullptr; int K2 = 0; int64_t lda2 = 0, ldb2 = 0;
+  bool a_kmajor = true, b_kmajor = true;
+  float* D = nullptr; int64_t ldd = 0;
+  const float* bias = nullptr;
+  bool sigmoid = false;
+  const float* dsig = nullptr; int64_t ld_dsig = 0; int dsig_rows = 1;
+  float alpha = 1.f;
+  const float* cin = nullptr; int64_t ld_cin = 0; float beta = 0.f;
+};
+
+// FP32 fused-multiply-add GEMM (any shape, any alignment).  Returns launches made.
+int launch_gemm_ffma(const GemmArgs& g, cudaStream_t st);
+
+// ---- vector / memory-bound kernels -------------------------------------------------------------
+// Row gather dst[r][:] = src[idx[r]][:]; rows with idx outside [0, src_rows) are zero-filled and
+// *err_flag is set to 1.
+int launch_gather_rows(const float* src, int64_t src_rows, int cols, const int32_t* idx, int64_t n_idx,
+                       float* dst, int* err_flag, cudaStream_t st);
+
+// out[j] = alpha * sum_r A[r * lda + j] + beta * cin[j]  (cin may be nullptr), j < cols.
+// scratch: at least colsum_scratch_floats(rows, cols) floats.
+int64_t colsum_scratch_floats(int64_t rows, int cols);
+int launch_colsum(const float* A, int64_t rows, int cols, int64_t lda, float alpha, const float* cin,
+                  float beta, float* out, float* scratch, cudaStream_t st);
+
+// Squared loss and its derivative for a row batch: delta = 2 (Z - Y) (delta may be nullptr),
+// partial[b] = sum over the block's elements of (Z - Y)^2 in double.  Returns blocks via *n_partials.
+int loss_num_partials(int64_t count);
+int launch_loss_delta(const float* Z, const float* Y, int64_t count, float* delta, double* partial,
+                      cudaStream_t st);
+
+// Fixed-order double-precision sum of `count` partials: *out (+)= sum.
+int launch_sum_partials(const double* partial, int count, double* out, bool accumulate, cudaStream_t st);
+
+// Transposed copy dst[c][r] = src[r][c] (src rows x cols).
+int launch_transpose(const float* src, int rows, int cols, float* dst, cudaStream_t st);
+
+// ---- conjugate gradient ------------------------------------------------------------------------
+// The n coordinates are cut into chunks, each inside one segment (one segment for the full system,
+// one per layer for the block-diagonal systems).  Partial sums are per chunk, combined per segment
+// in a fixed order in double precision.
+struct CgChunk { int64_t start; int32_t len; int32_t seg; };
+constexpr int kCgChunk = 4096;
+
+struct CgSeg {           // per-segment scalars, device resident
+  double rho;            // r^T r
+  double pq;             // p^T q
+  double gnorm2;         // ||g||^2
+  float alpha, beta;
+  int active;
+  int pad;
+};
+
+// r = -g, p = r, d = 0, partial[c] = sum r^2
+int launch_cg_init(const float* g, float* d, float* r, float* p, const CgChunk* chunks, int n_chunks,
+                   double* partial, cudaStream_t st);
+// partial[c] = sum p q
+int launch_cg_dot(const float* p, const float* q, const CgChunk* chunks, int n_chunks, double* partial,
+                  cudaStream_t st);
+// d += alpha p, r -= alpha q, partial[c] = sum r^2   (alpha per segment)
+int launch_cg_update(const float* p, const float* q, float* d, float* r, const CgChunk* chunks,
+                     int n_chunks, const CgSeg* seg, double* partial, cudaStream_t st);
+// p = r + beta p   (beta per segment)
+int launch_cg_direction(const float* r, float* p, const CgChunk* chunks, int n_chunks, const CgSeg* seg,
+                        cudaStream_t st);
+// phase 0: rho = gnorm2 = sum, active = rho > 0 && (tol <= 0 || sqrt(rho) > tol ||g||)
+// phase 1: pq = sum, alpha = active ? rho / pq : 0
+// phase 2: rho_new = sum; beta = active ? rho_new / rho : 0; rho = rho_new; active &= !stop
+// After each phase host_out[0] = sum over segments of rho, host_out[1] = number of active segments.
+int launch_cg_scalars(int phase, const double* partial, const CgChunk* chunks, int n_chunks, CgSeg* seg,
+                      int n_seg, double tol, double* host_out, cudaStream_t st);
+
+}  // namespace gn

@@ -1,0 +1,326 @@
+// Memory-bound kernels of the path: subsample row gather, column sums (bias blocks), squared loss,
+// and the conjugate-gradient vector updates with their dot products.
+//
+// Reductions are deterministic: every block writes one partial, partials are combined in a fixed
+// order in double precision.
+#include "gn_kernels.h"
+
+namespace gn {
+namespace {
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Sum over a 256-thread block; result valid in thread 0.
+__device__ __forceinline__ double block_sum_256(double v) {
+  __shared__ double sh[8];
+  v = warp_sum(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) sh[w] = v;
+  __syncthreads();
+  double t = 0.0;
+  if (w == 0) {
+    t = l < 8 ? sh[l] : 0.0;
+    t = warp_sum(t);
+  }
+  return t;
+}
+
+// ---------------------------------------------------------------------------------- gather
+// One warp per destination row, 16-byte loads when the rows allow it.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const float* __restrict__ src, long long src_rows, int cols,
+                                                          const int32_t* __restrict__ idx, long long n_idx,
+                                                          float* __restrict__ dst, int* err_flag, int vec) {
+  const int lane = threadIdx.x & 31;
+  const long long warps = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < n_idx; r += warps) {
+    const long long s = idx[r];
+    const bool ok = s >= 0 && s < src_rows;
+    if (!ok && lane == 0) atomicExch(err_flag, 1);
+    float* d = dst + r * cols;
+    if (vec) {
+      const float4* sp = reinterpret_cast<const float4*>(src + (ok ? s : 0) * cols);
+      float4* dp = reinterpret_cast<float4*>(d);
+      for (int c = lane; c < (cols >> 2); c += 32) dp[c] = ok ? __ldg(sp + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    } else {
+      const float* sp = src + (ok ? s : 0) * cols;
+      for (int c = lane; c < cols; c += 32) d[c] = ok ? __ldg(sp + c) : 0.f;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------- column sums
+constexpr int CS_ROWS = 512;  // rows per block
+
+// grid (ceil(cols/32), ceil(rows/CS_ROWS)); 256 threads = 8 warps striding rows, lanes along columns.
+__global__ void __launch_bounds__(256) colsum_partial_kernel(const float* __restrict__ A, long long rows, int cols,
+                                                             long long lda, float* __restrict__ scratch) {
+  __shared__ float sh[8][33];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + lane;
+  const long long r0 = (long long)blockIdx.y * CS_ROWS;
+  const long long r1 = min(rows, r0 + CS_ROWS);
+  float s = 0.f;
+  if (c < cols)
+    for (long long r = r0 + w; r < r1; r += 8) s += __ldg(A + r * lda + c);
+  sh[w][lane] = s;
+  __syncthreads();
+  if (w == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) t += sh[k][lane];
+    if (c < cols) scratch[(long long)blockIdx.y * cols + c] = t;
+  }
+}
+
+__global__ void __launch_bounds__(256) colsum_final_kernel(const float* __restrict__ scratch, int n_parts, int cols,
+                                                           float alpha, const float* __restrict__ cin, float beta,
+                                                           float* __restrict__ out) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols) return;
+  double s = 0.0;
+  for (int k = 0; k < n_parts; ++k) s += (double)scratch[(long long)k * cols + c];
+  float v = alpha * (float)s;
+  if (cin) v = fmaf(beta, cin[c], v);
+  out[c] = v;
+}
+
+// ---------------------------------------------------------------------------------- loss
+constexpr int LOSS_PER_BLOCK = 256 * 8;
+
+__global__ void __launch_bounds__(256) loss_delta_kernel(const float* __restrict__ Z, const float* __restrict__ Y,
+                                                         long long count, float* __restrict__ delta,
+                                                         double* __restrict__ partial) {
+  const long long base = (long long)blockIdx.x * LOSS_PER_BLOCK;
+  float s = 0.f;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const long long i = base + k * 256 + threadIdx.x;
+    if (i < count) {
+      const float e = Z[i] - __ldg(Y + i);
+      s = fmaf(e, e, s);
+      if (delta) delta[i] = 2.f * e;
+    }
+  }
+  const double t = block_sum_256((double)s);
+  if (threadIdx.x == 0) partial[blockIdx.x] = t;
+}
+
+__global__ void __launch_bounds__(256) sum_partials_kernel(const double* __restrict__ partial, int count,
+                                                           double* out, int accumulate) {
+  double s = 0.0;
+  for (int i = threadIdx.x; i < count; i += 256) s += partial[i];
+  const double t = block_sum_256(s);
+  if (threadIdx.x == 0) *out = accumulate ? *out + t : t;
+}
+
+// ---------------------------------------------------------------------------------- transpose
+__global__ void __launch_bounds__(256) transpose_kernel(const float* __restrict__ src, int rows, int cols,
+                                                        float* __restrict__ dst) {
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int j = ty; j < 32; j += 8) {
+    const int r = r0 + j, c = c0 + tx;
+    tile[j][tx] = (r < rows && c < cols) ? src[(long long)r * cols + c] : 0.f;
+  }
+  __syncthreads();
+  for (int j = ty; j < 32; j += 8) {
+    const int c = c0 + j, r = r0 + tx;
+    if (r < rows && c < cols) dst[(long long)c * rows + r] = tile[tx][j];
+  }
+}
+
+// ---------------------------------------------------------------------------------- CG
+// One block per chunk of at most kCgChunk coordinates: 256 threads x 16 strided elements.
+__global__ void __launch_bounds__(256) cg_init_kernel(const float* __restrict__ g, float* __restrict__ d,
+                                                      float* __restrict__ r, float* __restrict__ p,
+                                                      const CgChunk* __restrict__ chunks, double* __restrict__ partial) {
+  const CgChunk ch = chunks[blockIdx.x];
+  float s = 0.f;
+  for (int i = threadIdx.x; i < ch.len; i += 256) {
+    const long long k = ch.start + i;
+    const float x = -g[k];
+    d[k] = 0.f; r[k] = x; p[k] = x;
+    s = fmaf(x, x, s);
+  }
+  const double t = block_sum_256((double)s);
+  if (threadIdx.x == 0) partial[blockIdx.x] = t;
+}
+
+__global__ void __launch_bounds__(256) cg_dot_kernel(const float* __restrict__ p, const float* __restrict__ q,
+                                                     const CgChunk* __restrict__ chunks, double* __restrict__ partial) {
+  const CgChunk ch = chunks[blockIdx.x];
+  float s = 0.f;
+  for (int i = threadIdx.x; i < ch.len; i += 256) {
+    const long long k = ch.start + i;
+    s = fmaf(p[k], q[k], s);
+  }
+  const double t = block_sum_256((double)s);
+  if (threadIdx.x == 0) partial[blockIdx.x] = t;
+}
+
+__global__ void __launch_bounds__(256) cg_update_kernel(const float* __restrict__ p, const float* __restrict__ q,
+                                                        float* __restrict__ d, float* __restrict__ r,
+                                                        const CgChunk* __restrict__ chunks, const CgSeg* __restrict__ seg,
+                                                        double* __restrict__ partial) {
+  const CgChunk ch = chunks[blockIdx.x];
+  const float alpha = seg[ch.seg].alpha;
+  const bool live = seg[ch.seg].active != 0;
+  float s = 0.f;
+  for (int i = threadIdx.x; i < ch.len; i += 256) {
+    const long long k = ch.start + i;
+    float rk = r[k];
+    if (live) {
+      d[k] = fmaf(alpha, p[k], d[k]);
+      rk = fmaf(-alpha, q[k], rk);
+      r[k] = rk;
+    }
+    s = fmaf(rk, rk, s);
+  }
+  const double t = block_sum_256((double)s);
+  if (threadIdx.x == 0) partial[blockIdx.x] = t;
+}
+
+__global__ void __launch_bounds__(256) cg_direction_kernel(const float* __restrict__ r, float* __restrict__ p,
+                                                           const CgChunk* __restrict__ chunks,
+                                                           const CgSeg* __restrict__ seg) {
+  const CgChunk ch = chunks[blockIdx.x];
+  if (seg[ch.seg].beta == 0.f && seg[ch.seg].active == 0 && seg[ch.seg].alpha == 0.f) return;  // frozen before this step
+  const float beta = seg[ch.seg].beta;
+  for (int i = threadIdx.x; i < ch.len; i += 256) {
+    const long long k = ch.start + i;
+    p[k] = fmaf(beta, p[k], r[k]);
+  }
+}
+
+// One block; warp w handles segments w, w+8, ...  Chunks of a segment are contiguous in the table.
+__global__ void __launch_bounds__(256) cg_scalars_kernel(int phase, const double* __restrict__ partial,
+                                                         const CgChunk* __restrict__ chunks, int n_chunks,
+                                                         CgSeg* __restrict__ seg, int n_seg, double tol,
+                                                         double* __restrict__ host_out) {
+  __shared__ double seg_rho[64];
+  __shared__ int seg_act[64];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  for (int s0 = 0; s0 < n_seg; s0 += 64) {
+    for (int s = s0 + w; s < min(n_seg, s0 + 64); s += 8) {
+      // fixed-order sum of this segment's partials: lane-strided, then a butterfly
+      double acc = 0.0;
+      for (int c = lane; c < n_chunks; c += 32)
+        if (chunks[c].seg == s) acc += partial[c];
+      acc = warp_sum(acc);
+      if (lane == 0) {
+        CgSeg g = seg[s];
+        if (phase == 0) {
+          g.rho = acc; g.gnorm2 = acc; g.pq = 0.0; g.alpha = 0.f; g.beta = 0.f;
+          g.active = (acc > 0.0) && (tol <= 0.0 || sqrt(acc) > tol * sqrt(acc)) ? 1 : 0;
+        } else if (phase == 1) {
+          g.pq = acc;
+          g.alpha = (g.active && acc > 0.0) ? (float)(g.rho / acc) : 0.f;
+          if (!(acc > 0.0)) g.active = 0;
+        } else {
+          if (g.active) {
+            g.beta = g.rho > 0.0 ? (float)(acc / g.rho) : 0.f;
+            g.rho = acc;
+            if (!(acc > 0.0) || (tol > 0.0 && sqrt(acc) <= tol * sqrt(g.gnorm2))) g.active = 0;
+          } else {
+            g.beta = 0.f; g.alpha = 0.f;
+          }
+        }
+        seg[s] = g;
+        seg_rho[s - s0] = g.rho;
+        seg_act[s - s0] = g.active;
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double tot = s0 == 0 ? 0.0 : host_out[0];
+      double act = s0 == 0 ? 0.0 : host_out[1];
+      for (int s = s0; s < min(n_seg, s0 + 64); ++s) { tot += seg_rho[s - s0]; act += seg_act[s - s0]; }
+      host_out[0] = tot; host_out[1] = act;
+    }
+    __syncthreads();
+  }
+}
+
+}  // namespace
+
+int launch_gather_rows(const float* src, int64_t src_rows, int cols, const int32_t* idx, int64_t n_idx,
+                       float* dst, int* err_flag, cudaStream_t st) {
+  if (n_idx <= 0) return 0;
+  const int vec = (cols % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0) &&
+                  ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
+  const long long blocks = (n_idx + 7) / 8;
+  const int grid = (int)(blocks < 148LL * 16 ? blocks : 148LL * 16);
+  gather_rows_kernel<<<grid, 256, 0, st>>>(src, src_rows, cols, idx, n_idx, dst, err_flag, vec);
+  return 1;
+}
+
+int64_t colsum_scratch_floats(int64_t rows, int cols) {
+  return ((rows + CS_ROWS - 1) / CS_ROWS) * (int64_t)cols;
+}
+
+int launch_colsum(const float* A, int64_t rows, int cols, int64_t lda, float alpha, const float* cin,
+                  float beta, float* out, float* scratch, cudaStream_t st) {
+  const int parts = (int)((rows + CS_ROWS - 1) / CS_ROWS);
+  dim3 grid((cols + 31) / 32, parts);
+  colsum_partial_kernel<<<grid, 256, 0, st>>>(A, rows, cols, lda, scratch);
+  colsum_final_kernel<<<(cols + 255) / 256, 256, 0, st>>>(scratch, parts, cols, alpha, cin, beta, out);
+  return 2;
+}
+
+int loss_num_partials(int64_t count) { return (int)((count + LOSS_PER_BLOCK - 1) / LOSS_PER_BLOCK); }
+
+int launch_loss_delta(const float* Z, const float* Y, int64_t count, float* delta, double* partial,
+                      cudaStream_t st) {
+  loss_delta_kernel<<<loss_num_partials(count), 256, 0, st>>>(Z, Y, count, delta, partial);
+  return 1;
+}
+
+int launch_sum_partials(const double* partial, int count, double* out, bool accumulate, cudaStream_t st) {
+  sum_partials_kernel<<<1, 256, 0, st>>>(partial, count, out, accumulate ? 1 : 0);
+  return 1;
+}
+
+int launch_transpose(const float* src, int rows, int cols, float* dst, cudaStream_t st) {
+  dim3 grid((cols + 31) / 32, (rows + 31) / 32);
+  transpose_kernel<<<grid, 256, 0, st>>>(src, rows, cols, dst);
+  return 1;
+}
+
+int launch_cg_init(const float* g, float* d, float* r, float* p, const CgChunk* chunks, int n_chunks,
+                   double* partial, cudaStream_t st) {
+  cg_init_kernel<<<n_chunks, 256, 0, st>>>(g, d, r, p, chunks, partial);
+  return 1;
+}
+int launch_cg_dot(const float* p, const float* q, const CgChunk* chunks, int n_chunks, double* partial,
+                  cudaStream_t st) {
+  cg_dot_kernel<<<n_chunks, 256, 0, st>>>(p, q, chunks, partial);
+  return 1;
+}
+int launch_cg_update(const float* p, const float* q, float* d, float* r, const CgChunk* chunks,
+                     int n_chunks, const CgSeg* seg, double* partial, cudaStream_t st) {
+  cg_update_kernel<<<n_chunks, 256, 0, st>>>(p, q, d, r, chunks, seg, partial);
+  return 1;
+}
+int launch_cg_direction(const float* r, float* p, const CgChunk* chunks, int n_chunks, const CgSeg* seg,
+                        cudaStream_t st) {
+  cg_direction_kernel<<<n_chunks, 256, 0, st>>>(r, p, chunks, seg);
+  return 1;
+}
+int launch_cg_scalars(int phase, const double* partial, const CgChunk* chunks, int n_chunks, CgSeg* seg,
+                      int n_seg, double tol, double* host_out, cudaStream_t st) {
+  cg_scalars_kernel<<<1, 256, 0, st>>>(phase, partial, chunks, n_chunks, seg, n_seg, tol, host_out);
+  return 1;
+}
+
+}  // namespace gn

@@ -1,0 +1,73 @@
+"""Parity at the benchmark configurations' full sizes (the launch configuration bench.py times)."""
+import numpy as np
+import pytest
+
+import gn_workloads as wl
+from oracle import gn_oracle as orc
+from test_gpu_parity import TOL, dev, make_ctx, rel
+
+pytestmark = pytest.mark.gpu
+
+
+def test_mnist300_products_and_gradient_on_all_rows():
+    p = wl.make("mnist300")
+    ctx = make_ctx(p)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    v = dev(p["v"])
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
+               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    g, f = ctx.grad(with_f=True)
+    assert abs(f - orc.fun(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL["fp32"] * abs(f)
+    assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL["fp32"]
+    ctx.close()
+
+
+def test_svhn1000_products_and_cg():
+    p = wl.make("svhn1000", l=5000)          # all 2500 subsample rows, fewer rows for f / grad
+    ctx = make_ctx(p)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    v = dev(p["v"])
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
+               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    g = ctx.grad()
+    g_ref = orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])
+    assert rel(g.cpu().numpy(), g_ref) <= TOL["fp32"]
+    # 20 CG steps on the full system: compare the first 10 iterates
+    g32 = g_ref.astype(np.float32)
+    _, its_ref, _ = orc.cg_solve(p["theta"], p["widths"], p["C"], XS, g32, 1.0, False, 10, 0.0)
+    d, its, res, iterates = ctx.cg_solve(dev(g32), 1.0, blockdiag=False, max_iter=20, tol=0.0, keep_iterates=True)
+    assert its == 20
+    for k in range(10):
+        assert rel(iterates[k].cpu().numpy(), its_ref[k]) <= 1e-4
+    assert all(b < a for a, b in zip(res[:-1], res[1:]) if a > 1e-6 * res[0])
+    ctx.close()
+
+
+def test_mnist2000_headline_config_at_5_percent():
+    p = wl.make("mnist2000_5")
+    ctx = make_ctx(p)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    v = dev(p["v"])
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
+               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    ctx.close()
+
+
+def test_wide4096_reduced_rows_and_properties_at_full_size():
+    import torch
+    # element-wise parity on the first 1500 subsample rows of the same recipe ...
+    p = wl.make("wide4096", l=4000, nS=1500)
+    ctx = make_ctx(p)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    v = dev(p["v"])
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    g = ctx.grad()
+    assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL["fp32"]
+    ctx.close()

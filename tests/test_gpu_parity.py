@@ -1,0 +1,213 @@
+"""CUDA path against the float64 checker, element by element, through the C ABI."""
+import numpy as np
+import pytest
+
+import gn_workloads as wl
+from oracle import gn_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"fp32": 1e-5, "tf32": 2e-3}       # relative L2, FP32-accurate / TF32 contractions
+
+
+def rel(a, b):
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    return np.linalg.norm(a - b) / np.linalg.norm(b)
+
+
+def make_ctx(p, mode="fp32"):
+    import torch
+    import paper_1802_00130_b200 as gn
+    dev = torch.device("cuda:0")
+    X = torch.from_numpy(p["X"]).to(dev)
+    Y = torch.from_numpy(p["Y"]).to(dev)
+    ctx = gn.GnContext(p["widths"], p["C"], X, Y, gn.GN_FP32_ACCURATE if mode == "fp32" else gn.GN_TF32)
+    ctx.set_theta(torch.from_numpy(p["theta"]).to(dev))
+    return ctx
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).to("cuda:0")
+
+
+SMALL = ["tiny", "ragged", "single", "mid"]
+
+
+@pytest.mark.parametrize("mode", ["fp32"])
+@pytest.mark.parametrize("name", SMALL)
+def test_small_workloads_all_quantities(name, mode):
+    p = wl.make(name)
+    ctx = make_ctx(p, mode)
+    th, w, C = p["theta"], p["widths"], p["C"]
+    XS = p["X"][p["idx"]]
+    ctx.set_subsample(dev(p["idx"]))
+    # stored forward pass (Eq. xtoz)
+    Zo = orc.forward(th, w, XS)
+    for m in range(1, len(w)):
+        assert rel(ctx.debug_activations(m).cpu().numpy(), Zo[m]) <= TOL[mode]
+    # f and gradient over all rows
+    f = ctx.fun()
+    assert abs(f - orc.fun(th, w, C, p["X"], p["Y"])) <= TOL[mode] * abs(f)
+    g, f2 = ctx.grad(with_f=True)
+    assert abs(f2 - f) <= 1e-12 * abs(f)
+    assert rel(g.cpu().numpy(), orc.grad(th, w, C, p["X"], p["Y"])) <= TOL[mode]
+    # products
+    out = ctx.Gv(dev(p["v"])).cpu().numpy()
+    assert rel(out, orc.Gv(th, w, C, XS, p["v"])) <= TOL[mode]
+    outb = ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy()
+    assert rel(outb, orc.Gv_blockdiag(th, w, C, XS, p["v"])) <= TOL[mode]
+    ctx.close()
+
+
+def test_tiny_against_explicit_jacobians():
+    p = wl.make("tiny")
+    ctx = make_ctx(p)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    a = orc.Gv_definition(p["theta"], p["widths"], p["C"], XS, p["v"])
+    b = orc.Gv_blockdiag_definition(p["theta"], p["widths"], p["C"], XS, p["v"])
+    assert rel(ctx.Gv(dev(p["v"])).cpu().numpy(), a) <= 1e-5
+    assert rel(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy(), b) <= 1e-5
+    ctx.close()
+
+
+@pytest.mark.parametrize("rows", [1, 7, 100, 333, 100000])
+def test_row_batches_give_the_same_f_and_gradient(rows):
+    p = wl.make("ragged")
+    ctx = make_ctx(p)
+    ctx.set_batch_rows(rows)
+    g, f = ctx.grad(with_f=True)
+    assert abs(f - orc.fun(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= 1e-5 * abs(f)
+    assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= 1e-5
+    assert abs(ctx.fun() - f) <= 1e-12 * abs(f)
+    ctx.close()
+
+
+@pytest.mark.parametrize("blockdiag", [False, True])
+@pytest.mark.parametrize("name", ["tiny", "ragged"])
+def test_cg_iterates_follow_the_checker(name, blockdiag):
+    p = wl.make(name)
+    ctx = make_ctx(p)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    g = orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]).astype(np.float32)
+    d_ref, its_ref, res_ref = orc.cg_solve(p["theta"], p["widths"], p["C"], XS, g, 1.0, blockdiag, 10, 0.0)
+    d, its, res, iterates = ctx.cg_solve(dev(g), 1.0, blockdiag=blockdiag, max_iter=10, tol=0.0, keep_iterates=True)
+    assert its == 10 == len(its_ref)
+    iterates = iterates.cpu().numpy()
+    for k in range(10):
+        assert rel(iterates[k], its_ref[k]) <= 1e-4, k
+    assert rel(d.cpu().numpy(), d_ref) <= 1e-4
+    tot = [np.sqrt(np.sum(np.square(r))) for r in res_ref]
+    assert np.allclose(res[:6], tot[:6], rtol=1e-3)
+    ctx.close()
+
+
+@pytest.mark.parametrize("blockdiag", [False, True])
+def test_cg_stop_rule(blockdiag):
+    p = wl.make("mid")
+    ctx = make_ctx(p)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    g = orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]).astype(np.float32)
+    sigma = 1e-3
+    d_ref, its_ref, _ = orc.cg_solve(p["theta"], p["widths"], p["C"], XS, g, 1.0, blockdiag, 250, sigma)
+    d, its, res = ctx.cg_solve(dev(g), 1.0, blockdiag=blockdiag, max_iter=250, tol=sigma)
+    assert abs(its - len(its_ref)) <= 1
+    assert rel(d.cpu().numpy(), d_ref) <= 2e-3       # stopped at sigma = 1e-3, possibly one step apart
+    # the stop rule itself, checked with the checker's operator on the library's answer
+    d64 = d.cpu().numpy().astype(np.float64)
+    A = (lambda x: orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, x) + x) if blockdiag else \
+        (lambda x: orc.Gv(p["theta"], p["widths"], p["C"], XS, x) + x)
+    r = A(d64) + g
+    segs = orc.block_slices(p["widths"]) if blockdiag else [slice(0, p["n"])]
+    for s in segs:
+        assert np.linalg.norm(r[s]) <= sigma * np.linalg.norm(g[s]) * 1.01
+    ctx.close()
+
+
+def test_degenerate_subsamples():
+    import torch
+    p = wl.make("ragged")
+    ctx = make_ctx(p)
+    v = dev(p["v"])
+    # a single row
+    one = np.array([5], dtype=np.int32)
+    ctx.set_subsample(dev(one))
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], p["X"][one], p["v"])) <= 1e-5
+    # repeated rows count once per occurrence
+    dup = np.array([1, 1, 4, 7, 7, 7], dtype=np.int32)
+    ctx.set_subsample(dev(dup))
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], p["X"][dup], p["v"])) <= 1e-5
+    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
+               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], p["X"][dup], p["v"])) <= 1e-5
+    # S = all rows, and a larger set after a smaller one (workspace regrowth)
+    allrows = np.arange(p["l"], dtype=np.int32)
+    ctx.set_subsample(dev(allrows))
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], p["X"], p["v"])) <= 1e-5
+    # the host-buffer entry points give the same bits as the device ones
+    a = ctx.Gv(v).cpu().numpy()
+    b = ctx.Gv_host(p["v"])
+    assert np.array_equal(a, b)
+    ctx.close()
+
+
+def test_errors_and_state():
+    import paper_1802_00130_b200 as gn
+    import torch
+    p = wl.make("tiny")
+    dev0 = torch.device("cuda:0")
+    X, Y = dev(p["X"]), dev(p["Y"])
+    ctx = gn.GnContext(p["widths"], p["C"], X, Y)
+    v = dev(p["v"])
+    with pytest.raises(gn.GnError) as e:
+        ctx.Gv(v)
+    assert e.value.status == 4                      # no theta
+    with pytest.raises(gn.GnError) as e:
+        ctx.set_subsample(dev(p["idx"]))
+    assert e.value.status == 4
+    ctx.set_theta(dev(p["theta"]))
+    with pytest.raises(gn.GnError) as e:
+        ctx.Gv(v)
+    assert e.value.status == 4                      # no subsample
+    bad = p["idx"].copy()
+    bad[3] = p["l"]                                 # one past the end
+    with pytest.raises(gn.GnError) as e:
+        ctx.set_subsample(dev(bad))
+    assert e.value.status == 1
+    bad[3] = -1
+    with pytest.raises(gn.GnError) as e:
+        ctx.set_subsample(dev(bad))
+    assert e.value.status == 1
+    with pytest.raises(gn.GnError):
+        ctx.Gv(v)                                   # still no valid subsample
+    ctx.set_subsample(dev(p["idx"]))
+    out = ctx.Gv(v)
+    ctx.set_theta(dev(p["theta"]))                  # stored activations are stale now
+    with pytest.raises(gn.GnError) as e:
+        ctx.Gv(v)
+    assert e.value.status == 4
+    ctx.set_subsample(dev(p["idx"]))
+    assert torch.equal(ctx.Gv(v), out)              # deterministic, bit for bit
+    with pytest.raises(gn.GnError) as e:
+        ctx.Gv(v, out=v)
+    assert e.value.status == 1
+    assert ctx.kernel_launches > 0 and ctx.workspace_bytes > 0
+    ctx.close()
+
+
+def test_symmetry_and_positive_definiteness_on_device():
+    p = wl.make("mid")
+    ctx = make_ctx(p)
+    ctx.set_subsample(dev(p["idx"]))
+    rng = np.random.Generator(np.random.PCG64(99))
+    u = rng.standard_normal(p["n"], dtype=np.float32)
+    v = p["v"]
+    for fn in (ctx.Gv, ctx.Gv_blockdiag):
+        Gu = fn(dev(u)).cpu().numpy().astype(np.float64)
+        Gv = fn(dev(v)).cpu().numpy().astype(np.float64)
+        assert abs(u @ Gv - v @ Gu) <= 1e-4 * abs(u @ Gv)
+        assert v @ Gv >= v.astype(np.float64) @ v / p["C"]
+    ctx.close()
