@@ -1,0 +1,335 @@
+"""Benchmark of the subsampled Gauss-Newton product path on synthetic data.
+
+One step = one pass of the whole path at the 784-2000-2000-2000-10 network:
+    set_subsample (row gather + stored forward pass on S)
+    grad          (f and gradient over all l rows, in row batches)
+    cg_solve      (n_cg CG steps on the full system: one G^S v each + vector updates)
+    cg_solve      (n_cg CG steps on the per-layer systems: one block-diagonal product each)
+The metric is Gauss-Newton matrix-vector products per second over whole steps (2 n_cg products per
+step); the breakdown gives the product-only rates and FLOP/s.
+
+    python bench.py --gpus N --steps K --warmup W            (N > 1: launched with torch.distributed.run)
+    python bench.py --impl reference ...                      (the float64 CPU checker on a bounded sample)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import gn_workloads as wl  # noqa: E402
+
+METRIC = "gauss_newton_matvecs_per_s"
+UNIT = "matvec/s"
+FP32_LANES_PER_SM, SMS = 128, 148
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    sm_max_mhz=d.get("sm_max_mhz", 1965.0), src="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, sm_max_mhz=1965.0, src="fallback")
+
+
+def mac_counts(widths):
+    g = [widths[m - 1] * widths[m] for m in range(1, len(widths))]
+    L = len(g)
+    fwd = sum(g)
+    grad = 2 * sum(g) + sum(g[1:])
+    full = 2 * g[0] + 4 * sum(g[1:])
+    b1 = sum(2 * g[m] + 2 * sum(g[m + 1:]) for m in range(L))
+    paper_block = sum(2 * g[m] + 2 * widths[-1] * widths[m + 1] for m in range(L))
+    return dict(fwd=fwd, grad=grad, full=full, block_executed=b1, block_paper=paper_block)
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons for one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 and len(r) >= 8] or [r for _, r in self.rows if len(r) >= 8]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = sorted(float(r[0]) for r in rows)
+        reasons = set()
+        for r in rows:
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][1]), "samples": len(rows),
+                "power_w_max": max(float(r[2]) for r in rows), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle arm
+def oracle_sample_rates(p, sample_rows, n_cg, threads_note=True):
+    """Times the float64 checker on `sample_rows` rows and scales to the step's row counts."""
+    from oracle import gn_oracle as orc
+    rows = min(sample_rows, p["nS"])
+    XS = p["X"][p["idx"][:rows]]
+    th, w, C = p["theta"], p["widths"], p["C"]
+    t0 = time.perf_counter(); orc.Gv(th, w, C, XS, p["v"]); t_full = time.perf_counter() - t0
+    t0 = time.perf_counter(); orc.Gv_blockdiag(th, w, C, XS, p["v"]); t_blk = time.perf_counter() - t0
+    t0 = time.perf_counter(); orc.grad(th, w, C, p["X"][:rows], p["Y"][:rows]); t_grad = time.perf_counter() - t0
+    t0 = time.perf_counter(); orc.forward(th, w, XS); t_fwd = time.perf_counter() - t0
+    step = (t_fwd * p["nS"] / rows + t_grad * p["l"] / rows + n_cg * (t_full + t_blk) * p["nS"] / rows)
+    return dict(value=2 * n_cg / step, step_s=step, rows=rows, t_full=t_full, t_blk=t_blk, t_grad=t_grad,
+                Gv_per_s=rows / (t_full * p["nS"]), cpu_s=t_full + t_blk + t_grad + t_fwd)
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 1) for d in threadpool_info() if d.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    p = wl.make(args.workload)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_rates(p, max(64, args.ref_rows // 8), args.n_cg)
+    vals = []
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        vals.append(oracle_sample_rates(p, args.ref_rows, args.n_cg))
+    dt = time.perf_counter() - t0
+    v = float(np.median([x["value"] for x in vals]))
+    cores = blas_threads()
+    sample = (f"{vals[0]['rows']} rows per product and per gradient pass, scaled by row count to "
+              f"|S|={p['nS']}, l={p['l']}; numpy float64")
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * float(np.median([x["step_s"] for x in vals])),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "widths": p["widths"], "l": p["l"], "S": p["nS"], "n_cg": args.n_cg},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "wall_s": dt}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def run_ours(args):
+    import torch
+    import paper_1802_00130_b200 as gn
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    p = wl.make(args.workload)
+    mode = gn.GN_TF32 if args.mode == "tf32" else gn.GN_FP32_ACCURATE
+    X, Y = torch.from_numpy(p["X"]).to(dev), torch.from_numpy(p["Y"]).to(dev)
+    ctx = gn.GnContext(p["widths"], p["C"], X, Y, mode)
+    theta = torch.from_numpy(p["theta"]).to(dev)
+    # a fresh subsample per step, as in the Newton iteration: rotations of one permutation
+    rng = np.random.Generator(np.random.PCG64(4242 + rank))
+    perm = rng.permutation(p["l"]).astype(np.int32)
+    n_sets = args.steps + args.warmup + 2
+    idx_host = [np.ascontiguousarray(np.roll(perm, 977 * k)[: p["nS"]]) for k in range(n_sets)]
+    idx_dev = [torch.from_numpy(a).to(dev) for a in idx_host]
+    g = torch.empty(ctx.n, dtype=torch.float32, device=dev)
+    d = torch.empty(ctx.n, dtype=torch.float32, device=dev)
+    n_cg = args.n_cg
+
+    def step(k):
+        ctx.set_theta(theta)
+        ctx.set_subsample(idx_dev[k % n_sets])
+        ctx.grad(out=g)
+        ctx.cg_solve(g, 1.0, blockdiag=False, max_iter=n_cg, tol=0.0, out=d)
+        ctx.cg_solve(g, 1.0, blockdiag=True, max_iter=n_cg, tol=0.0, out=d)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for k in range(args.warmup):
+        step(k)
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = ctx.kernel_launches
+    ctx.profile(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    e0.record()
+    for k in range(args.steps):
+        step(args.warmup + k)
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    ms = e0.elapsed_time(e1)
+    prof = ctx.profile_read()
+    ctx.profile(False)
+    launches = ctx.kernel_launches - launches0
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    if dist:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    matvecs = 2 * n_cg * args.steps * world
+    value = matvecs / (ms * 1e-3)
+
+    # ---- product-only rates (device-resident, outside the step timing)
+    v = torch.from_numpy(p["v"]).to(dev)
+    out = torch.empty_like(v)
+    breakdown = {}
+    macs = mac_counts(p["widths"])
+    for name, fn, mac_exec, mac_alg in (("Gv", ctx.Gv, macs["full"], macs["full"]),
+                                        ("Gv_blockdiag", ctx.Gv_blockdiag, macs["block_executed"], macs["block_paper"])):
+        for _ in range(3):
+            fn(v, out=out)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = args.product_reps
+        a.record()
+        for _ in range(reps):
+            fn(v, out=out)
+        b.record()
+        torch.cuda.synchronize()
+        t = a.elapsed_time(b) * 1e-3 / reps
+        breakdown[name] = {"per_s": 1.0 / t, "ms": 1e3 * t,
+                           "executed_tflops": 2.0 * mac_exec * p["nS"] / t / 1e12,
+                           "algorithmic_tflops": 2.0 * mac_alg * p["nS"] / t / 1e12}
+
+    # ---- end to end through the host-buffer entry points (pinned host memory)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory().numpy()
+    h_theta, h_g, h_d = pin(p["theta"]), pin(np.zeros(ctx.n, np.float32)), pin(np.zeros(ctx.n, np.float32))
+    h_idx = [pin(a) for a in idx_host]
+
+    def step_host(k):
+        ctx.set_theta_host(h_theta)
+        ctx.set_subsample_host(h_idx[k % n_sets])
+        ctx.grad_host(out=h_g)
+        ctx.cg_solve_host(h_g, 1.0, blockdiag=False, max_iter=n_cg, tol=0.0, out=h_d)
+        ctx.cg_solve_host(h_g, 1.0, blockdiag=True, max_iter=n_cg, tol=0.0, out=h_d)
+
+    step_host(0)
+    barrier()
+    e0.record()
+    for k in range(args.steps):
+        step_host(args.warmup + k)
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if dist:
+        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    n4 = 4 * ctx.n
+    e2e = {"value": matvecs / (ms_e2e * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": n4 + 4 * p["nS"] + 2 * n4, "d2h_bytes_per_step": n4 + 2 * n4}
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    if args.mode == "tf32":
+        peak = pk["bf16_sustained"] / 2.0
+        roof = {"bound": "tensor", "unit": "TFLOP/s", "peak": peak,
+                "peak_note": f"TF32 = 1/2 of the {pk['src']} sustained bf16 cuBLAS rate ({pk['bf16_sustained']} TFLOP/s)"}
+    else:
+        peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
+        roof = {"bound": "alu", "unit": "TFLOP/s", "peak": peak,
+                "peak_note": "148 SMs x 128 FP32 lanes x 2 FLOP x max SM clock"}
+    achieved = prof["gemm_flop"] / (prof["gemm_ms"] * 1e-3) / 1e12 if prof["gemm_ms"] > 0 else None
+    roof.update({"kernel": prof["kernel"], "achieved": achieved, "frac": achieved / peak if achieved else None,
+                 "traffic": None, "launches": prof["gemm_launches"], "avg_launch_us": 1e3 * prof["gemm_ms"] / max(1, prof["gemm_launches"]),
+                 "share_of_step": prof["gemm_ms"] / (ms / 1.0) if ms > 0 else None})
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        r = oracle_sample_rates(p, args.ref_rows, n_cg)
+        cpu = {"value": r["value"], "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"{r['rows']} rows per product and per gradient pass ({r['cpu_s']:.1f} s of CPU work), "
+                         f"scaled by row count to |S|={p['nS']}, l={p['l']}",
+               "Gv_per_s": r["Gv_per_s"]}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "tf32" if args.mode == "tf32" else "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "widths": p["widths"], "l": p["l"], "S": p["nS"], "C": p["C"],
+                       "n_cg": n_cg, "step": "set_subsample + grad(all rows) + n_cg CG steps full + n_cg CG steps block-diagonal",
+                       "l2": "per-step working set (activations of S and of the row batches) exceeds the 126 MB L2",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof, "cpu_baseline": cpu,
+            "breakdown": breakdown}
+    print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mnist2000_20", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--mode", default="fp32", choices=["fp32", "tf32"])
+    ap.add_argument("--n-cg", dest="n_cg", type=int, default=10)
+    ap.add_argument("--product-reps", type=int, default=10)
+    ap.add_argument("--ref-rows", type=int, default=1024)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -179,6 +179,16 @@ gn_status gn_cg_solve_host(gn_ctx* ctx, const float* h_g, double lambda, int blo
 gn_status gn_debug_activations(gn_ctx* ctx, int m, float* d_out);
 
 /*
+ * gn_profile - switch per-launch timing of the contraction kernels on (enable != 0) or off.  While on,
+ * every GEMM launch is bracketed by a pair of CUDA events on the context's stream.
+ * gn_profile_read - synchronise the stream, return the summed GEMM device time in milliseconds, the
+ * floating-point operations those launches executed (2 M N K each) and their number, and reset the
+ * counters.  Any of the three outputs may be NULL.
+ */
+gn_status gn_profile(gn_ctx* ctx, int enable);
+gn_status gn_profile_read(gn_ctx* ctx, double* gemm_ms, double* gemm_flop, int64_t* gemm_launches);
+
+/*
  * gn_kernel_launches - number of kernels this context has launched so far (all entry points).
  */
 int64_t gn_kernel_launches(const gn_ctx* ctx);

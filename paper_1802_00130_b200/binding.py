@@ -35,6 +35,8 @@ _SIGNATURES = {
     "gn_cg_solve": (_i32, [_vp, _vp, _dbl, _i32, _i32, _dbl, _vp, C.POINTER(_i32), _vp, C.POINTER(_dbl)]),
     "gn_cg_solve_host": (_i32, [_vp, _vp, _dbl, _i32, _i32, _dbl, _vp, C.POINTER(_i32), C.POINTER(_dbl)]),
     "gn_debug_activations": (_i32, [_vp, _i32, _vp]),
+    "gn_profile": (_i32, [_vp, _i32]),
+    "gn_profile_read": (_i32, [_vp, C.POINTER(_dbl), C.POINTER(_dbl), C.POINTER(_i64)]),
 }
 
 
@@ -107,6 +109,7 @@ class GnContext:
         if st != 0:
             raise GnError(st, "gn_create failed (needs an sm_100 device and valid arguments)")
         self._h = handle
+        self.precision = int(precision)
         self.n = int(self._lib.gn_num_params(self._h))
         self.device = X.device
 
@@ -219,6 +222,15 @@ class GnContext:
             self._h, _host_ptr(g, np.float32, self.n), float(lam), int(bool(blockdiag)), int(max_iter), float(tol),
             _host_ptr(out, np.float32, self.n), C.byref(its), res))
         return out, its.value, np.array(res[: its.value + 1])
+
+    def profile(self, enable):
+        self._check(self._lib.gn_profile(self._h, int(bool(enable))))
+
+    def profile_read(self):
+        ms, flop, cnt = _dbl(), _dbl(), _i64()
+        self._check(self._lib.gn_profile_read(self._h, C.byref(ms), C.byref(flop), C.byref(cnt)))
+        return {"gemm_ms": ms.value, "gemm_flop": flop.value, "gemm_launches": cnt.value,
+                "kernel": "gemm_ffma_kernel" if self.precision == GN_FP32_ACCURATE else "gemm_tf32_kernel"}
 
     def debug_activations(self, m):
         import torch

@@ -49,6 +49,12 @@ struct gn_ctx {
   CgChunk* chunks[2] = {nullptr, nullptr}; int n_chunks[2] = {0, 0};
   CgSeg* segs = nullptr;
 
+  // optional per-GEMM timing
+  struct EvPair { cudaEvent_t a, b; double flop; };
+  std::vector<EvPair> ev;
+  size_t ev_used = 0;
+  bool profiling = false;
+
   int64_t bytes = 0;
   int64_t launches = 0;
   std::string err;
@@ -118,7 +124,20 @@ gn_status sync(gn_ctx* c, const char* where) {
 }
 
 void run_gemm(gn_ctx* c, const GemmArgs& g) {
+  gn_ctx::EvPair* e = nullptr;
+  if (c->profiling) {
+    if (c->ev_used == c->ev.size()) {
+      gn_ctx::EvPair p{};
+      if (cudaEventCreate(&p.a) == cudaSuccess && cudaEventCreate(&p.b) == cudaSuccess) c->ev.push_back(p);
+    }
+    if (c->ev_used < c->ev.size()) {
+      e = &c->ev[c->ev_used++];
+      e->flop = 2.0 * g.M * (double)g.N * ((double)g.K1 + (g.A2 ? (double)g.K2 : 0.0));
+      cudaEventRecord(e->a, c->st);
+    }
+  }
   c->launches += launch_gemm_ffma(g, c->st);
+  if (e) cudaEventRecord(e->b, c->st);
 }
 
 gn_status ensure_partials(gn_ctx* c, int64_t count) {
@@ -408,6 +427,7 @@ gn_status gn_destroy(gn_ctx* c) {
   cudaStreamSynchronize(c->st);
   for (void* p : c->owned)
     if (p) cudaFree(p);
+  for (auto& p : c->ev) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   if (c->hscal) cudaFreeHost(c->hscal);
   if (c->h_err) cudaFreeHost(c->h_err);
   cudaGetLastError();
@@ -598,6 +618,29 @@ gn_status gn_cg_solve_host(gn_ctx* c, const float* h_g, double lambda, int block
   GN_TRY(gn_cg_solve(c, c->tmp_a, lambda, blockdiag, max_iter, tol, c->tmp_b, iters_host, nullptr, resnorm_host));
   GN_CUDA(c, cudaMemcpyAsync(h_d, c->tmp_b, c->n * sizeof(float), cudaMemcpyDeviceToHost, c->st));
   return sync(c, "cg_solve_host");
+}
+
+gn_status gn_profile(gn_ctx* c, int enable) {
+  if (!c) return GN_EINVAL;
+  c->profiling = enable != 0;
+  return GN_OK;
+}
+
+gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t* gemm_launches) {
+  if (!c) return GN_EINVAL;
+  GN_TRY(sync(c, "profile_read"));
+  double ms = 0.0, flop = 0.0;
+  for (size_t i = 0; i < c->ev_used; ++i) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, c->ev[i].a, c->ev[i].b) == cudaSuccess) ms += t;
+    flop += c->ev[i].flop;
+  }
+  if (gemm_ms) *gemm_ms = ms;
+  if (gemm_flop) *gemm_flop = flop;
+  if (gemm_launches) *gemm_launches = (int64_t)c->ev_used;
+  c->ev_used = 0;
+  cudaGetLastError();
+  return GN_OK;
 }
 
 gn_status gn_debug_activations(gn_ctx* c, int m, float* d_out) {
