@@ -283,10 +283,15 @@ def run_ours(args):
         peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
         roof = {"bound": "alu", "unit": "TFLOP/s", "peak": peak,
                 "peak_note": "148 SMs x 128 FP32 lanes x 2 FLOP x max SM clock"}
-    achieved = prof["gemm_flop"] / (prof["gemm_ms"] * 1e-3) / 1e12 if prof["gemm_ms"] > 0 else None
-    roof.update({"kernel": prof["kernel"], "achieved": achieved, "frac": achieved / peak if achieved else None,
-                 "traffic": None, "launches": prof["gemm_launches"], "avg_launch_us": 1e3 * prof["gemm_ms"] / max(1, prof["gemm_launches"]),
-                 "share_of_step": prof["gemm_ms"] / (ms / 1.0) if ms > 0 else None})
+    kern = prof["tensor"] if args.mode == "tf32" else prof["ffma"]
+    achieved = kern["flop"] / (kern["ms"] * 1e-3) / 1e12 if kern["ms"] > 0 else None
+    roof.update({"kernel": "gemm_tf32_kernel" if args.mode == "tf32" else "gemm_ffma_kernel",
+                 "achieved": achieved, "frac": achieved / peak if achieved else None, "traffic": None,
+                 "launches": kern["launches"], "avg_launch_us": 1e3 * kern["ms"] / max(1, kern["launches"]),
+                 "share_of_step": kern["ms"] / ms if ms > 0 else None,
+                 "other_gemm": {"kernel": "gemm_ffma_kernel" if args.mode == "tf32" else "gemm_tf32_kernel",
+                                "ms": (prof["ffma"] if args.mode == "tf32" else prof["tensor"])["ms"],
+                                "launches": (prof["ffma"] if args.mode == "tf32" else prof["tensor"])["launches"]}})
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:

@@ -37,6 +37,7 @@ _SIGNATURES = {
     "gn_debug_activations": (_i32, [_vp, _i32, _vp]),
     "gn_profile": (_i32, [_vp, _i32]),
     "gn_profile_read": (_i32, [_vp, C.POINTER(_dbl), C.POINTER(_dbl), C.POINTER(_i64)]),
+    "gn_debug_gemm": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64]),
 }
 
 
@@ -227,10 +228,22 @@ class GnContext:
         self._check(self._lib.gn_profile(self._h, int(bool(enable))))
 
     def profile_read(self):
-        ms, flop, cnt = _dbl(), _dbl(), _i64()
-        self._check(self._lib.gn_profile_read(self._h, C.byref(ms), C.byref(flop), C.byref(cnt)))
-        return {"gemm_ms": ms.value, "gemm_flop": flop.value, "gemm_launches": cnt.value,
-                "kernel": "gemm_ffma_kernel" if self.precision == GN_FP32_ACCURATE else "gemm_tf32_kernel"}
+        """Per-kernel GEMM timing since the last read: {"tensor": {...}, "ffma": {...}}."""
+        ms, flop, cnt = (_dbl * 2)(), (_dbl * 2)(), (_i64 * 2)()
+        self._check(self._lib.gn_profile_read(self._h, ms, flop, cnt))
+        return {name: {"ms": ms[k], "flop": flop[k], "launches": cnt[k]}
+                for k, name in enumerate(("tensor", "ffma"))}
+
+    def debug_gemm(self, kind, A, B, a_kmajor=True, b_kmajor=True):
+        """Test hook: D[M][N] from A ([M][K] or [K][M]) and B ([N][K] or [K][N]); kind 0 tensor-core, 1 FMA."""
+        import torch
+        M, K = (A.shape if a_kmajor else A.shape[::-1])
+        N = B.shape[0] if b_kmajor else B.shape[1]
+        D = torch.empty((M, N), dtype=torch.float32, device=A.device)
+        self._check(self._lib.gn_debug_gemm(self._h, int(kind), M, N, K, _dev_ptr(A, torch.float32), A.stride(0),
+                                            int(a_kmajor), _dev_ptr(B, torch.float32), B.stride(0), int(b_kmajor),
+                                            _dev_ptr(D, torch.float32), D.stride(0)))
+        return D
 
     def debug_activations(self, m):
         import torch

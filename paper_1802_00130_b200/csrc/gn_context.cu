@@ -41,8 +41,9 @@ struct gn_ctx {
   double* partial = nullptr; int64_t partial_cap = 0;
   double* dscal = nullptr;   // device: [0] loss, [1] theta^T theta, [2] cg sum rho, [3] cg active
   double* hscal = nullptr;   // pinned mirror
-  int* err_flag = nullptr;
-  int* h_err = nullptr;      // pinned
+  int* err_flag = nullptr;   // [0] gather index error, [1] tensor-core pipeline timeout code
+  int* h_err = nullptr;      // pinned mirror of err_flag
+  gn_status sticky = GN_OK;  // a launch-time failure that must surface at the next check
   // CG
   float* cg_r = nullptr; float* cg_p = nullptr; float* cg_q = nullptr;
   float* tmp_a = nullptr; float* tmp_b = nullptr;  // staging for *_host calls
@@ -50,7 +51,7 @@ struct gn_ctx {
   CgSeg* segs = nullptr;
 
   // optional per-GEMM timing
-  struct EvPair { cudaEvent_t a, b; double flop; };
+  struct EvPair { cudaEvent_t a, b; double flop; int kind; };
   std::vector<EvPair> ev;
   size_t ev_used = 0;
   bool profiling = false;
@@ -112,18 +113,27 @@ void dev_free(gn_ctx* c, T*& p, int64_t count) {
 }
 
 gn_status check_launch(gn_ctx* c, const char* where) {
+  if (c->sticky != GN_OK) { gn_status s = c->sticky; c->sticky = GN_OK; return s; }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(c, e, where);
   return GN_OK;
 }
 
+// Synchronise the stream; also fetch the tensor-core pipeline's timeout word.
 gn_status sync(gn_ctx* c, const char* where) {
-  cudaError_t e = cudaStreamSynchronize(c->st);
+  cudaError_t e = cudaMemcpyAsync(c->h_err + 1, c->err_flag + 1, sizeof(int), cudaMemcpyDeviceToHost, c->st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->st);
   if (e != cudaSuccess) return cuda_fail(c, e, where);
+  if (c->h_err[1] != 0) {
+    const int code = c->h_err[1];
+    cudaMemsetAsync(c->err_flag + 1, 0, sizeof(int), c->st);
+    return fail(c, GN_ETIMEOUT, std::string(where) + ": a bounded wait in the tensor-core pipeline ran out (role " +
+                                    std::to_string(code) + "); results are invalid");
+  }
   return GN_OK;
 }
 
-void run_gemm(gn_ctx* c, const GemmArgs& g) {
+void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
   gn_ctx::EvPair* e = nullptr;
   if (c->profiling) {
     if (c->ev_used == c->ev.size()) {
@@ -133,11 +143,22 @@ void run_gemm(gn_ctx* c, const GemmArgs& g) {
     if (c->ev_used < c->ev.size()) {
       e = &c->ev[c->ev_used++];
       e->flop = 2.0 * g.M * (double)g.N * ((double)g.K1 + (g.A2 ? (double)g.K2 : 0.0));
+      e->kind = kind;
       cudaEventRecord(e->a, c->st);
     }
   }
-  c->launches += launch_gemm_ffma(g, c->st);
+  if (kind == 0) {
+    const int r = launch_gemm_tf32(g, c->err_flag + 1, c->st);
+    if (r < 0) { c->sticky = GN_ECUDA; c->err = "cuTensorMapEncodeTiled failed"; }
+    else c->launches += r;
+  } else {
+    c->launches += launch_gemm_ffma(g, c->st);
+  }
   if (e) cudaEventRecord(e->b, c->st);
+}
+
+void run_gemm(gn_ctx* c, const GemmArgs& g) {
+  run_gemm_kind(c, g, (c->prec == GN_TF32 && gemm_tf32_eligible(g)) ? 0 : 1);
 }
 
 gn_status ensure_partials(gn_ctx* c, int64_t count) {
@@ -411,9 +432,11 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
     if ((s = dev_alloc(c, &c->cg_p, c->n)) != GN_OK) break;
     if ((s = dev_alloc(c, &c->cg_q, c->n)) != GN_OK) break;
     if ((s = dev_alloc(c, &c->dscal, 8)) != GN_OK) break;
-    if ((s = dev_alloc(c, &c->err_flag, 1)) != GN_OK) break;
+    if ((s = dev_alloc(c, &c->err_flag, 2)) != GN_OK) break;
+    if (cudaMemset(c->err_flag, 0, 2 * sizeof(int)) != cudaSuccess) { s = GN_ECUDA; break; }
     if (cudaMallocHost(&c->hscal, 8 * sizeof(double)) != cudaSuccess) { s = GN_ENOMEM; break; }
-    if (cudaMallocHost(&c->h_err, sizeof(int)) != cudaSuccess) { s = GN_ENOMEM; break; }
+    if (cudaMallocHost(&c->h_err, 2 * sizeof(int)) != cudaSuccess) { s = GN_ENOMEM; break; }
+    c->h_err[0] = c->h_err[1] = 0;
     if ((s = build_chunks(c)) != GN_OK) break;
     if ((s = ensure_partials(c, 2 * (int64_t)c->n_chunks[1] + 64)) != GN_OK) break;
   } while (0);
@@ -629,18 +652,38 @@ gn_status gn_profile(gn_ctx* c, int enable) {
 gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t* gemm_launches) {
   if (!c) return GN_EINVAL;
   GN_TRY(sync(c, "profile_read"));
-  double ms = 0.0, flop = 0.0;
+  double ms[2] = {0.0, 0.0}, flop[2] = {0.0, 0.0};
+  int64_t cnt[2] = {0, 0};
   for (size_t i = 0; i < c->ev_used; ++i) {
     float t = 0.f;
-    if (cudaEventElapsedTime(&t, c->ev[i].a, c->ev[i].b) == cudaSuccess) ms += t;
-    flop += c->ev[i].flop;
+    const int k = c->ev[i].kind ? 1 : 0;
+    if (cudaEventElapsedTime(&t, c->ev[i].a, c->ev[i].b) == cudaSuccess) ms[k] += t;
+    flop[k] += c->ev[i].flop;
+    cnt[k] += 1;
   }
-  if (gemm_ms) *gemm_ms = ms;
-  if (gemm_flop) *gemm_flop = flop;
-  if (gemm_launches) *gemm_launches = (int64_t)c->ev_used;
+  for (int k = 0; k < 2; ++k) {
+    if (gemm_ms) gemm_ms[k] = ms[k];
+    if (gemm_flop) gemm_flop[k] = flop[k];
+    if (gemm_launches) gemm_launches[k] = cnt[k];
+  }
   c->ev_used = 0;
   cudaGetLastError();
   return GN_OK;
+}
+
+gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* dA, int64_t lda, int a_kmajor,
+                        const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd) {
+  if (!c) return GN_EINVAL;
+  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || (kind != 0 && kind != 1)) return fail(c, GN_EINVAL, "bad GEMM arguments");
+  GemmArgs g;
+  g.M = M; g.N = N; g.K1 = K;
+  g.A1 = dA; g.lda1 = lda; g.a_kmajor = a_kmajor != 0;
+  g.B1 = dB; g.ldb1 = ldb; g.b_kmajor = b_kmajor != 0;
+  g.D = dD; g.ldd = ldd;
+  if (kind == 0 && !gemm_tf32_eligible(g)) return fail(c, GN_EINVAL, "operands do not qualify for the tensor-core kernel");
+  run_gemm_kind(c, g, kind);
+  GN_TRY(check_launch(c, "debug_gemm"));
+  return sync(c, "debug_gemm");
 }
 
 gn_status gn_debug_activations(gn_ctx* c, int m, float* d_out) {

@@ -34,6 +34,13 @@ struct GemmArgs {
 // FP32 fused-multiply-add GEMM (any shape, any alignment).  Returns launches made.
 int launch_gemm_ffma(const GemmArgs& g, cudaStream_t st);
 
+// TF32 tensor-core GEMM (tcgen05 + TMA).  Operands must be 16-byte aligned with leading dimensions
+// that are multiples of 4 floats (TMA strides); gemm_tf32_eligible says whether a problem qualifies.
+// *err_flag receives a non-zero code if a bounded device-side wait ran out.  Returns launches made,
+// or -1 if a tensor map could not be encoded.
+bool gemm_tf32_eligible(const GemmArgs& g);
+int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st);
+
 // ---- vector / memory-bound kernels -------------------------------------------------------------
 // Row gather dst[r][:] = src[idx[r]][:]; rows with idx outside [0, src_rows) are zero-filled and
 // *err_flag is set to 1.

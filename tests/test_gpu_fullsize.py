@@ -9,18 +9,19 @@ from test_gpu_parity import TOL, dev, make_ctx, rel
 pytestmark = pytest.mark.gpu
 
 
-def test_mnist300_products_and_gradient_on_all_rows():
+@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+def test_mnist300_products_and_gradient_on_all_rows(mode):
     p = wl.make("mnist300")
-    ctx = make_ctx(p)
+    ctx = make_ctx(p, mode)
     ctx.set_subsample(dev(p["idx"]))
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
     assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
-               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
     g, f = ctx.grad(with_f=True)
-    assert abs(f - orc.fun(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL["fp32"] * abs(f)
-    assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL["fp32"]
+    assert abs(f - orc.fun(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL[mode] * abs(f)
+    assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL[mode]
     ctx.close()
 
 
@@ -49,15 +50,16 @@ def test_svhn1000_products_and_cg():
     ctx.close()
 
 
-def test_mnist2000_headline_config_at_5_percent():
+@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+def test_mnist2000_headline_config_at_5_percent(mode):
     p = wl.make("mnist2000_5")
-    ctx = make_ctx(p)
+    ctx = make_ctx(p, mode)
     ctx.set_subsample(dev(p["idx"]))
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
     assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
-               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
     ctx.close()
 
 

@@ -1,0 +1,55 @@
+"""The two contraction kernels on their own, against a float64 matrix product (numpy)."""
+import numpy as np
+import pytest
+
+import gn_workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [(128, 256, 32), (128, 256, 64), (300, 520, 200), (1000, 300, 784), (37, 40, 12), (2500, 1000, 1000),
+          (260, 2000, 3000)]
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import torch
+    import paper_1802_00130_b200 as gn
+    p = wl.make("tiny")
+    X = torch.from_numpy(p["X"]).cuda()
+    Y = torch.from_numpy(p["Y"]).cuda()
+    c = gn.GnContext(p["widths"], p["C"], X, Y)
+    yield c
+    c.close()
+
+
+def operands(M, N, K, a_k, b_k, seed):
+    rng = np.random.Generator(np.random.PCG64(seed))
+    A = rng.standard_normal((M, K) if a_k else (K, M), dtype=np.float32)
+    B = rng.standard_normal((N, K) if b_k else (K, N), dtype=np.float32)
+    Am = A if a_k else A.T
+    Bm = B.T if b_k else B
+    ref = Am.astype(np.float64) @ Bm.astype(np.float64)
+    return A, B, ref
+
+
+@pytest.mark.parametrize("a_k,b_k", [(True, True), (True, False), (False, True), (False, False)])
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("kind,tol", [(1, 2e-6), (0, 1e-3)])
+def test_gemm_layouts(ctx, kind, tol, shape, a_k, b_k):
+    import torch
+    import paper_1802_00130_b200 as gn
+    M, N, K = shape
+    A, B, ref = operands(M, N, K, a_k, b_k, seed=M + 7 * N + 13 * K)
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    try:
+        D = ctx.debug_gemm(kind, dA, dB, a_kmajor=a_k, b_kmajor=b_k)
+    except gn.GnError as e:
+        # the tensor-core kernel refuses operands TMA cannot address (leading dimension not a multiple of 4)
+        assert kind == 0 and e.status == 1
+        lda, ldb = A.shape[1], B.shape[1]
+        assert lda % 4 or ldb % 4 or N < 32
+        return
+    err = np.linalg.norm(D.cpu().numpy() - ref) / np.linalg.norm(ref)
+    assert err <= tol, err
+    # element-wise too: a misplaced tile would hide in a norm of a large matrix
+    assert np.max(np.abs(D.cpu().numpy() - ref)) <= 50 * tol * np.sqrt(K)

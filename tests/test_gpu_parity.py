@@ -35,7 +35,7 @@ def dev(a):
 SMALL = ["tiny", "ragged", "single", "mid"]
 
 
-@pytest.mark.parametrize("mode", ["fp32"])
+@pytest.mark.parametrize("mode", ["fp32", "tf32"])
 @pytest.mark.parametrize("name", SMALL)
 def test_small_workloads_all_quantities(name, mode):
     p = wl.make(name)
