@@ -181,19 +181,20 @@ gn_status gn_debug_activations(gn_ctx* ctx, int m, float* d_out);
 /*
  * gn_profile - switch per-launch timing of the contraction kernels on (enable != 0) or off.  While on,
  * every GEMM launch is bracketed by a pair of CUDA events on the context's stream.
- * gn_profile_read - synchronise the stream and return, for the tensor-core kernel (index 0) and the
- * FP32 FMA kernel (index 1): summed device time in milliseconds, floating-point operations executed
- * (2 M N K per launch) and number of launches; then reset the counters.  Each output is an array of
- * two entries and may be NULL.
+ * gn_profile_read - synchronise the stream and return, for the tensor-core kernel (index 0), the
+ * FP32 FMA GEMM (index 1) and the streaming kernels for n_L-wide shapes (index 2): summed device time
+ * in milliseconds, floating-point operations executed (2 M N K per launch) and number of launches;
+ * then reset the counters.  Each output is an array of three entries and may be NULL.
  */
 gn_status gn_profile(gn_ctx* ctx, int enable);
 gn_status gn_profile_read(gn_ctx* ctx, double* gemm_ms, double* gemm_flop, int64_t* gemm_launches);
 
 /*
  * gn_debug_gemm - test hook: one contraction D[M][N] = sum_k A(m,k) B(k,n) on the context's stream
- * with the kernel of the given kind (0 = tensor-core TF32, 1 = FP32 FMA).  a_kmajor: A is [M][K]
+ * with the kernel of the given kind (0 = tensor-core TF32, 1 = FP32 FMA GEMM, 2 = streaming kernel for
+ * a dimension <= 16).  a_kmajor: A is [M][K]
  * (else [K][M]); b_kmajor: B is [N][K] (else [K][N]); all row-major with the given leading
- * dimensions.  GN_EINVAL if the tensor-core kernel cannot take the operands (alignment).
+ * dimensions.  GN_EINVAL if the chosen kernel cannot take the operands (alignment, shape).
  */
 gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float* dA, int64_t lda,
                         int a_kmajor, const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd);

@@ -229,10 +229,10 @@ class GnContext:
 
     def profile_read(self):
         """Per-kernel GEMM timing since the last read: {"tensor": {...}, "ffma": {...}}."""
-        ms, flop, cnt = (_dbl * 2)(), (_dbl * 2)(), (_i64 * 2)()
+        ms, flop, cnt = (_dbl * 3)(), (_dbl * 3)(), (_i64 * 3)()
         self._check(self._lib.gn_profile_read(self._h, ms, flop, cnt))
         return {name: {"ms": ms[k], "flop": flop[k], "launches": cnt[k]}
-                for k, name in enumerate(("tensor", "ffma"))}
+                for k, name in enumerate(("tensor", "ffma", "thin"))}
 
     def debug_gemm(self, kind, A, B, a_kmajor=True, b_kmajor=True):
         """Test hook: D[M][N] from A ([M][K] or [K][M]) and B ([N][K] or [K][N]); kind 0 tensor-core, 1 FMA."""

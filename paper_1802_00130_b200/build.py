@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgn_b200.so")
-SOURCES = ["gn_context.cu", "gemm_ffma.cu", "gemm_tf32.cu", "vector_ops.cu"]
+SOURCES = ["gn_context.cu", "gemm_ffma.cu", "gemm_tf32.cu", "gemm_thin.cu", "vector_ops.cu"]
 FLAGS = ["-shared", "-Xcompiler", "-fPIC", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
          "-O3", "-std=c++17"]
 

@@ -1,0 +1,305 @@
+// Contractions with one tiny dimension (the n_L-wide output layer): memory-bound, so they run as
+// streaming FP32 kernels instead of 128-wide GEMM tiles.
+//
+//   thin-N : D[M][N] = sum_k A[m][k] B[n][k] (+ second pair), N <= 16          (output-layer forward / R pass)
+//   thin-M : D[M][N] = alpha sum_r A[r][m] B[r][n] + beta cin, M <= 16          (output-layer weight block)
+//   thin-K : D[M][N] = (sum_k A[m][k] B[k][n]) * epilogue, K <= 16              (back-propagation out of layer L)
+//
+// All use the common epilogue of GemmArgs.  Deterministic: fixed-order reductions, no atomics.
+#include "gn_kernels.h"
+
+namespace gn {
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+struct Epi {
+  float* D; long long ldd;
+  const float* bias; int sigmoid;
+  const float* dsig; long long ld_dsig; int dsig_rows;
+  float alpha;
+  const float* cin; long long ld_cin; float beta;
+};
+
+Epi make_epi(const GemmArgs& g) {
+  Epi e;
+  e.D = g.D; e.ldd = g.ldd; e.bias = g.bias; e.sigmoid = g.sigmoid;
+  e.dsig = g.dsig; e.ld_dsig = g.ld_dsig; e.dsig_rows = g.dsig_rows > 0 ? g.dsig_rows : 1;
+  e.alpha = g.alpha; e.cin = g.cin; e.ld_cin = g.ld_cin; e.beta = g.beta;
+  return e;
+}
+
+__device__ __forceinline__ float apply_epi(const Epi& e, float x, int m, int n) {
+  if (e.bias) x += __ldg(e.bias + n);
+  if (e.sigmoid) x = 1.f / (1.f + expf(-x));
+  if (e.dsig) { const float z = __ldg(e.dsig + (long long)(m % e.dsig_rows) * e.ld_dsig + n); x *= z * (1.f - z); }
+  x *= e.alpha;
+  if (e.cin) x = fmaf(e.beta, __ldg(e.cin + (long long)m * e.ld_cin + n), x);
+  return x;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ------------------------------------------------------------------------------------ thin-N
+// One warp per group of TR rows; lanes stride K in float4 steps; B rows come through L1.
+constexpr int TR = 8;
+
+struct ThinNParams {
+  int M, N;
+  const float* A[2]; const float* B[2]; int K[2]; long long lda[2], ldb[2];
+  Epi e;
+};
+
+template <int NMAX>
+__global__ void __launch_bounds__(256) gemm_thin_n_kernel(const ThinNParams p) {
+  const int lane = threadIdx.x & 31;
+  const int warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int m0 = warp * TR;
+  if (m0 >= p.M) return;
+  float acc[TR][NMAX];
+#pragma unroll
+  for (int r = 0; r < TR; ++r)
+#pragma unroll
+    for (int n = 0; n < NMAX; ++n) acc[r][n] = 0.f;
+
+  for (int s = 0; s < 2; ++s) {
+    const float* __restrict__ A = p.A[s];
+    const float* __restrict__ B = p.B[s];
+    if (!A) continue;
+    const int K = p.K[s];
+    for (int k = lane * 4; k < K; k += 128) {
+      float4 a[TR];
+#pragma unroll
+      for (int r = 0; r < TR; ++r) {
+        const int m = min(m0 + r, p.M - 1);          // clamp: duplicate rows are never written
+        a[r] = __ldg(reinterpret_cast<const float4*>(A + (long long)m * p.lda[s] + k));
+      }
+#pragma unroll
+      for (int n = 0; n < NMAX; ++n) {
+        if (n < p.N) {
+          const float4 b = __ldg(reinterpret_cast<const float4*>(B + (long long)n * p.ldb[s] + k));
+#pragma unroll
+          for (int r = 0; r < TR; ++r) {
+            acc[r][n] = fmaf(a[r].x, b.x, acc[r][n]);
+            acc[r][n] = fmaf(a[r].y, b.y, acc[r][n]);
+            acc[r][n] = fmaf(a[r].z, b.z, acc[r][n]);
+            acc[r][n] = fmaf(a[r].w, b.w, acc[r][n]);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < TR; ++r) {
+    float mine = 0.f;
+#pragma unroll
+    for (int n = 0; n < NMAX; ++n) {
+      const float s = warp_sum(acc[r][n]);
+      if (lane == n) mine = s;
+    }
+    const int m = m0 + r;
+    if (m < p.M && lane < p.N) p.e.D[(long long)m * p.e.ldd + lane] = apply_epi(p.e, mine, m, lane);
+  }
+}
+
+// ------------------------------------------------------------------------------------ thin-M
+// grid (column tiles of 512, row chunks); thread = 4 consecutive columns; A rows staged in shared
+// memory 128 at a time; per-chunk partials go to scratch and are summed in chunk order.
+constexpr int TM_MAX = 16, TM_ROWS = 128;
+
+struct ThinMParams {
+  int M, N; long long rows, chunk_rows;
+  const float* A; long long lda;
+  const float* B; long long ldb;
+  float* scratch;  // [chunks][M][N]
+};
+
+template <int MMAX>
+__global__ void __launch_bounds__(128) gemm_thin_m_partial_kernel(const ThinMParams p) {
+  __shared__ float As[TM_ROWS][MMAX];
+  const int n = (blockIdx.x * 128 + threadIdx.x) * 4;
+  const long long r_begin = (long long)blockIdx.y * p.chunk_rows;
+  const long long r_end = min(p.rows, r_begin + p.chunk_rows);
+  float4 acc[MMAX];
+#pragma unroll
+  for (int m = 0; m < MMAX; ++m) acc[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (long long rb = r_begin; rb < r_end; rb += TM_ROWS) {
+    const int cnt = (int)min((long long)TM_ROWS, r_end - rb);
+    __syncthreads();
+    for (int i = threadIdx.x; i < cnt * MMAX; i += 128) {
+      const int r = i / MMAX, m = i % MMAX;
+      As[r][m] = m < p.M ? __ldg(p.A + (rb + r) * p.lda + m) : 0.f;
+    }
+    __syncthreads();
+    if (n < p.N) {
+#pragma unroll 4
+      for (int r = 0; r < cnt; ++r) {
+        const float4 b = __ldg(reinterpret_cast<const float4*>(p.B + (rb + r) * p.ldb + n));
+#pragma unroll
+        for (int m = 0; m < MMAX; ++m) {
+          const float a = As[r][m];
+          acc[m].x = fmaf(a, b.x, acc[m].x); acc[m].y = fmaf(a, b.y, acc[m].y);
+          acc[m].z = fmaf(a, b.z, acc[m].z); acc[m].w = fmaf(a, b.w, acc[m].w);
+        }
+      }
+    }
+  }
+  if (n < p.N) {
+#pragma unroll
+    for (int m = 0; m < MMAX; ++m)
+      if (m < p.M)
+        *reinterpret_cast<float4*>(p.scratch + ((long long)blockIdx.y * p.M + m) * p.N + n) = acc[m];
+  }
+}
+
+__global__ void __launch_bounds__(256) gemm_thin_m_final_kernel(const float* __restrict__ scratch, int chunks, int M, int N,
+                                                                const Epi e) {
+  const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= (long long)M * N) return;
+  const int m = (int)(i / N), n = (int)(i % N);
+  float s = 0.f;
+  for (int c = 0; c < chunks; ++c) s += scratch[((long long)c * M + m) * N + n];
+  e.D[(long long)m * e.ldd + n] = apply_epi(e, s, m, n);
+}
+
+// ------------------------------------------------------------------------------------ thin-K
+// thread = 4 consecutive columns, with its K x 4 slice of B in registers; blocks walk row chunks.
+constexpr int TK_MAX = 16;
+
+struct ThinKParams {
+  int M, N, K; int rows_per_block;
+  const float* A; long long lda;
+  const float* B; long long ldb;
+  Epi e;
+};
+
+template <int KMAX>
+__global__ void __launch_bounds__(128) gemm_thin_k_kernel(const ThinKParams p) {
+  const int n = (blockIdx.x * 128 + threadIdx.x) * 4;
+  if (n >= p.N) return;
+  float4 b[KMAX];
+#pragma unroll
+  for (int k = 0; k < KMAX; ++k)
+    b[k] = k < p.K ? __ldg(reinterpret_cast<const float4*>(p.B + (long long)k * p.ldb + n)) : make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (p.e.bias) bz = __ldg(reinterpret_cast<const float4*>(p.e.bias + n));
+  const int m_begin = blockIdx.y * p.rows_per_block;
+  const int m_end = min(p.M, m_begin + p.rows_per_block);
+  for (int m = m_begin; m < m_end; ++m) {
+    float4 acc = bz;
+#pragma unroll
+    for (int k = 0; k < KMAX; ++k) {
+      if (k < p.K) {
+        const float a = __ldg(p.A + (long long)m * p.lda + k);
+        acc.x = fmaf(a, b[k].x, acc.x); acc.y = fmaf(a, b[k].y, acc.y);
+        acc.z = fmaf(a, b[k].z, acc.z); acc.w = fmaf(a, b[k].w, acc.w);
+      }
+    }
+    float t[4] = {acc.x, acc.y, acc.z, acc.w};
+    if (p.e.sigmoid) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) t[j] = 1.f / (1.f + expf(-t[j]));
+    }
+    if (p.e.dsig) {
+      const float4 z = __ldg(reinterpret_cast<const float4*>(p.e.dsig + (long long)(m % p.e.dsig_rows) * p.e.ld_dsig + n));
+      t[0] *= z.x * (1.f - z.x); t[1] *= z.y * (1.f - z.y); t[2] *= z.z * (1.f - z.z); t[3] *= z.w * (1.f - z.w);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) t[j] *= p.e.alpha;
+    if (p.e.cin) {
+      const float4 c = __ldg(reinterpret_cast<const float4*>(p.e.cin + (long long)m * p.e.ld_cin + n));
+      t[0] = fmaf(p.e.beta, c.x, t[0]); t[1] = fmaf(p.e.beta, c.y, t[1]);
+      t[2] = fmaf(p.e.beta, c.z, t[2]); t[3] = fmaf(p.e.beta, c.w, t[3]);
+    }
+    *reinterpret_cast<float4*>(p.e.D + (long long)m * p.e.ldd + n) = make_float4(t[0], t[1], t[2], t[3]);
+  }
+}
+
+int thin_m_chunks(long long rows, int N) {
+  const int col_tiles = (N + 511) / 512;
+  long long chunks = (296 + col_tiles - 1) / col_tiles;
+  const long long max_chunks = (rows + 63) / 64;
+  if (chunks > max_chunks) chunks = max_chunks;
+  if (chunks < 1) chunks = 1;
+  return (int)chunks;
+}
+
+}  // namespace
+
+ThinKind gemm_thin_kind(const GemmArgs& g) {
+  if (g.M < 1 || g.N < 1) return THIN_NONE;
+  const bool pair2 = g.A2 != nullptr;
+  if (g.a_kmajor && g.b_kmajor && g.N <= 16 && g.K1 >= 64) {
+    bool ok = aligned16(g.A1) && aligned16(g.B1) && g.lda1 % 4 == 0 && g.ldb1 % 4 == 0 && g.K1 % 4 == 0;
+    if (pair2) ok = ok && aligned16(g.A2) && aligned16(g.B2) && g.lda2 % 4 == 0 && g.ldb2 % 4 == 0 && g.K2 % 4 == 0;
+    if (ok) return THIN_N;
+  }
+  if (!g.a_kmajor && !g.b_kmajor && !pair2 && g.M <= TM_MAX && g.N % 4 == 0 && aligned16(g.B1) && g.ldb1 % 4 == 0)
+    return THIN_M;
+  if (g.a_kmajor && !g.b_kmajor && !pair2 && g.K1 <= TK_MAX && g.N % 4 == 0 && aligned16(g.B1) && g.ldb1 % 4 == 0 &&
+      aligned16(g.D) && g.ldd % 4 == 0 && (!g.bias || aligned16(g.bias)) &&
+      (!g.dsig || (aligned16(g.dsig) && g.ld_dsig % 4 == 0)) && (!g.cin || (aligned16(g.cin) && g.ld_cin % 4 == 0)))
+    return THIN_K;
+  return THIN_NONE;
+}
+
+int64_t gemm_thin_scratch_floats(const GemmArgs& g) {
+  if (gemm_thin_kind(g) != THIN_M) return 0;
+  return (int64_t)thin_m_chunks(g.K1, g.N) * g.M * g.N;
+}
+
+int launch_gemm_thin(const GemmArgs& g, float* scratch, cudaStream_t st) {
+  const ThinKind kind = gemm_thin_kind(g);
+  if (kind == THIN_N) {
+    ThinNParams p{};
+    p.M = g.M; p.N = g.N;
+    p.A[0] = g.A1; p.B[0] = g.B1; p.K[0] = g.K1; p.lda[0] = g.lda1; p.ldb[0] = g.ldb1;
+    p.A[1] = g.A2; p.B[1] = g.B2; p.K[1] = g.A2 ? g.K2 : 0; p.lda[1] = g.lda2; p.ldb[1] = g.ldb2;
+    p.e = make_epi(g);
+    const int warps = (g.M + TR - 1) / TR;
+    const int grid = (warps + 7) / 8;
+    if (g.N <= 4) gemm_thin_n_kernel<4><<<grid, 256, 0, st>>>(p);
+    else if (g.N <= 8) gemm_thin_n_kernel<8><<<grid, 256, 0, st>>>(p);
+    else if (g.N <= 12) gemm_thin_n_kernel<12><<<grid, 256, 0, st>>>(p);
+    else gemm_thin_n_kernel<16><<<grid, 256, 0, st>>>(p);
+    return 1;
+  }
+  if (kind == THIN_M) {
+    ThinMParams p{};
+    p.M = g.M; p.N = g.N; p.rows = g.K1;
+    const int chunks = thin_m_chunks(g.K1, g.N);
+    p.chunk_rows = (g.K1 + chunks - 1) / chunks;
+    const int used = (int)((g.K1 + p.chunk_rows - 1) / p.chunk_rows);
+    p.A = g.A1; p.lda = g.lda1; p.B = g.B1; p.ldb = g.ldb1; p.scratch = scratch;
+    dim3 grid((g.N + 511) / 512, used);
+    if (g.M <= 4) gemm_thin_m_partial_kernel<4><<<grid, 128, 0, st>>>(p);
+    else if (g.M <= 8) gemm_thin_m_partial_kernel<8><<<grid, 128, 0, st>>>(p);
+    else if (g.M <= 12) gemm_thin_m_partial_kernel<12><<<grid, 128, 0, st>>>(p);
+    else gemm_thin_m_partial_kernel<16><<<grid, 128, 0, st>>>(p);
+    const long long total = (long long)g.M * g.N;
+    gemm_thin_m_final_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(scratch, used, g.M, g.N, make_epi(g));
+    return 2;
+  }
+  if (kind == THIN_K) {
+    ThinKParams p{};
+    p.M = g.M; p.N = g.N; p.K = g.K1;
+    p.A = g.A1; p.lda = g.lda1; p.B = g.B1; p.ldb = g.ldb1; p.e = make_epi(g);
+    const int col_tiles = (g.N + 511) / 512;
+    int row_blocks = (148 * 8 + col_tiles - 1) / col_tiles;
+    if (row_blocks > g.M) row_blocks = g.M;
+    p.rows_per_block = (g.M + row_blocks - 1) / row_blocks;
+    dim3 grid(col_tiles, (g.M + p.rows_per_block - 1) / p.rows_per_block);
+    if (g.K1 <= 4) gemm_thin_k_kernel<4><<<grid, 128, 0, st>>>(p);
+    else if (g.K1 <= 8) gemm_thin_k_kernel<8><<<grid, 128, 0, st>>>(p);
+    else if (g.K1 <= 12) gemm_thin_k_kernel<12><<<grid, 128, 0, st>>>(p);
+    else gemm_thin_k_kernel<16><<<grid, 128, 0, st>>>(p);
+    return 1;
+  }
+  return 0;
+}
+
+}  // namespace gn

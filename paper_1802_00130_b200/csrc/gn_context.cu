@@ -38,6 +38,7 @@ struct gn_ctx {
   std::vector<float*> Zb, Db;
   // reductions
   float* colsum_scratch = nullptr; int64_t colsum_cap = 0;
+  float* thin_scratch = nullptr; int64_t thin_cap = 0;
   double* partial = nullptr; int64_t partial_cap = 0;
   double* dscal = nullptr;   // device: [0] loss, [1] theta^T theta, [2] cg sum rho, [3] cg active
   double* hscal = nullptr;   // pinned mirror
@@ -151,13 +152,29 @@ void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
     const int r = launch_gemm_tf32(g, c->err_flag + 1, c->st);
     if (r < 0) { c->sticky = GN_ECUDA; c->err = "cuTensorMapEncodeTiled failed"; }
     else c->launches += r;
+  } else if (kind == 2) {
+    c->launches += launch_gemm_thin(g, c->thin_scratch, c->st);
   } else {
     c->launches += launch_gemm_ffma(g, c->st);
   }
   if (e) cudaEventRecord(e->b, c->st);
 }
 
+// Kernel choice: streaming kernels for the n_L-wide shapes (both precisions: they are exact FP32),
+// the tensor-core kernel in TF32 mode when TMA can address the operands, else the FP32 FMA GEMM.
 void run_gemm(gn_ctx* c, const GemmArgs& g) {
+  if (gemm_thin_kind(g) != THIN_NONE) {
+    const int64_t need = gemm_thin_scratch_floats(g);
+    if (need > c->thin_cap) {
+      cudaStreamSynchronize(c->st);
+      dev_free(c, c->thin_scratch, c->thin_cap);
+      c->thin_cap = 0;
+      if (dev_alloc(c, &c->thin_scratch, need) != GN_OK) { c->sticky = GN_ENOMEM; return; }
+      c->thin_cap = need;
+    }
+    run_gemm_kind(c, g, 2);
+    return;
+  }
   run_gemm_kind(c, g, (c->prec == GN_TF32 && gemm_tf32_eligible(g)) ? 0 : 1);
 }
 
@@ -652,16 +669,16 @@ gn_status gn_profile(gn_ctx* c, int enable) {
 gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t* gemm_launches) {
   if (!c) return GN_EINVAL;
   GN_TRY(sync(c, "profile_read"));
-  double ms[2] = {0.0, 0.0}, flop[2] = {0.0, 0.0};
-  int64_t cnt[2] = {0, 0};
+  double ms[3] = {0.0, 0.0, 0.0}, flop[3] = {0.0, 0.0, 0.0};
+  int64_t cnt[3] = {0, 0, 0};
   for (size_t i = 0; i < c->ev_used; ++i) {
     float t = 0.f;
-    const int k = c->ev[i].kind ? 1 : 0;
+    const int k = c->ev[i].kind < 0 || c->ev[i].kind > 2 ? 1 : c->ev[i].kind;
     if (cudaEventElapsedTime(&t, c->ev[i].a, c->ev[i].b) == cudaSuccess) ms[k] += t;
     flop[k] += c->ev[i].flop;
     cnt[k] += 1;
   }
-  for (int k = 0; k < 2; ++k) {
+  for (int k = 0; k < 3; ++k) {
     if (gemm_ms) gemm_ms[k] = ms[k];
     if (gemm_flop) gemm_flop[k] = flop[k];
     if (gemm_launches) gemm_launches[k] = cnt[k];
@@ -674,14 +691,19 @@ gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t
 gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* dA, int64_t lda, int a_kmajor,
                         const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd) {
   if (!c) return GN_EINVAL;
-  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || (kind != 0 && kind != 1)) return fail(c, GN_EINVAL, "bad GEMM arguments");
+  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 2) return fail(c, GN_EINVAL, "bad GEMM arguments");
   GemmArgs g;
   g.M = M; g.N = N; g.K1 = K;
   g.A1 = dA; g.lda1 = lda; g.a_kmajor = a_kmajor != 0;
   g.B1 = dB; g.ldb1 = ldb; g.b_kmajor = b_kmajor != 0;
   g.D = dD; g.ldd = ldd;
   if (kind == 0 && !gemm_tf32_eligible(g)) return fail(c, GN_EINVAL, "operands do not qualify for the tensor-core kernel");
-  run_gemm_kind(c, g, kind);
+  if (kind == 2) {
+    if (gemm_thin_kind(g) == THIN_NONE) return fail(c, GN_EINVAL, "operands do not qualify for a streaming kernel");
+    run_gemm(c, g);
+  } else {
+    run_gemm_kind(c, g, kind);
+  }
   GN_TRY(check_launch(c, "debug_gemm"));
   return sync(c, "debug_gemm");
 }

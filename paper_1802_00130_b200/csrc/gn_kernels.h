@@ -41,6 +41,14 @@ int launch_gemm_ffma(const GemmArgs& g, cudaStream_t st);
 bool gemm_tf32_eligible(const GemmArgs& g);
 int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st);
 
+// Streaming FP32 kernels for contractions with one dimension <= 16 (the n_L-wide output layer).
+// gemm_thin_kind says which of them (if any) takes a problem; THIN_M needs a scratch buffer of
+// gemm_thin_scratch_floats(g) floats.  launch_gemm_thin returns the launches made (0 = not taken).
+enum ThinKind { THIN_NONE = 0, THIN_N = 1, THIN_M = 2, THIN_K = 3 };
+ThinKind gemm_thin_kind(const GemmArgs& g);
+int64_t gemm_thin_scratch_floats(const GemmArgs& g);
+int launch_gemm_thin(const GemmArgs& g, float* scratch, cudaStream_t st);
+
 // ---- vector / memory-bound kernels -------------------------------------------------------------
 // Row gather dst[r][:] = src[idx[r]][:]; rows with idx outside [0, src_rows) are zero-filled and
 // *err_flag is set to 1.

@@ -46,7 +46,7 @@ def test_svhn1000_products_and_cg():
     # iterates follow the float64 ones to ~3e-4, the tiny configuration (test_gpu_parity) to 1e-4
     for k in range(10):
         assert rel(iterates[k].cpu().numpy(), its_ref[k]) <= 1e-3
-    assert all(b < a for a, b in zip(res[:-1], res[1:]) if a > 1e-6 * res[0])
+    assert res[-1] < 1e-4 * res[0]          # residual norms are not monotone in CG, but it has converged
     ctx.close()
 
 

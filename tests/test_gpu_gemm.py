@@ -53,3 +53,20 @@ def test_gemm_layouts(ctx, kind, tol, shape, a_k, b_k):
     assert err <= tol, err
     # element-wise too: a misplaced tile would hide in a norm of a large matrix
     assert np.max(np.abs(D.cpu().numpy() - ref)) <= 50 * tol * np.sqrt(K)
+
+
+THIN = [  # (M, N, K, a_kmajor, b_kmajor): one dimension <= 16, as at the n_L-wide output layer
+    (3000, 10, 2000, True, True), (131, 4, 64, True, True), (1000, 16, 300, True, True),
+    (10, 2000, 3000, False, False), (4, 16, 131, False, False), (16, 300, 70000, False, False),
+    (3000, 2000, 10, True, False), (131, 16, 4, True, False), (777, 300, 16, True, False),
+]
+
+
+@pytest.mark.parametrize("M,N,K,a_k,b_k", THIN)
+def test_streaming_kernels_for_thin_shapes(ctx, M, N, K, a_k, b_k):
+    import torch
+    A, B, ref = operands(M, N, K, a_k, b_k, seed=M + 7 * N + 13 * K)
+    D = ctx.debug_gemm(2, torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), a_kmajor=a_k, b_kmajor=b_k)
+    err = np.linalg.norm(D.cpu().numpy() - ref) / np.linalg.norm(ref)
+    assert err <= 2e-6, err
+    assert np.max(np.abs(D.cpu().numpy() - ref)) <= 1e-4 * np.sqrt(K)
