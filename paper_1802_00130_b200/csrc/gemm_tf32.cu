@@ -1,10 +1,13 @@
 // TF32 tensor-core GEMM for sm_100a: tcgen05.mma with the accumulator in tensor memory, operands
 // staged in shared memory by TMA (128-byte swizzle), fused epilogue read back with tcgen05.ld.
 //
-// One CTA computes one 128 x BN output tile.  Warp roles:
-//   warp 0      TMA producer (one elected lane): fills a ring of STAGES operand buffers
-//   warp 1      MMA issuer   (one elected lane): 4 x (128 x BN x 8) tcgen05.mma per ring slot
-//   warps 2..5  epilogue: each owns one 32-lane quadrant of tensor memory
+// Persistent kernel, one CTA per SM, each walking 128 x bn output tiles.  Warp roles:
+//   warp 0      TMA producer: fills a ring of STAGES operand buffers (issue spread over lanes)
+//   warp 1      MMA issuer   (one elected lane): 4 x (128 x bn x 8) tcgen05.mma per ring slot
+//   warps 2..9  epilogue: two warps per 32-lane quadrant of tensor memory, alternating over the
+//               tile's 32-column chunks; registers only (shared-memory bandwidth belongs to the
+//               MMA and TMA), all of a chunk's global reads issued before the accumulator is read
+// Two accumulators alternate in tensor memory, so a tile's epilogue overlaps the next tile's MMAs.
 // Up to two (A, B) operand pairs are accumulated into the same tile (the forward directional
 // derivative needs R z^{m-1} W^m + z^{m-1} V^m in one accumulator).
 //
@@ -27,7 +30,7 @@
 namespace gn {
 namespace {
 
-constexpr int BM = 128, BK = 32;
+constexpr int BM = 128, BK = 32, BN_MAX = 256;
 constexpr int A_STAGE_BYTES = BM * BK * 4;  // 16 KB
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
@@ -35,13 +38,15 @@ struct Tf32Params {
   int M, N;
   int kblocks[2];
   int a_mn, b_mn;
+  int a_3d, b_3d;       // MN-major operand fetched with one 3-D box per stage (needs a padded operand)
   float* D; long long ldd;
   const float* bias; int sigmoid;
   const float* dsig; long long ld_dsig; int dsig_rows;
   float alpha;
   const float* cin; long long ld_cin; float beta;
-  int vec_epi;
-  int tiles_n;
+  int vec_epi;          // D, bias, dsig, cin all 16-byte aligned with leading dimensions % 4 == 0
+  int bn;               // tile width: multiple of 32, 64 <= bn <= 256
+  int tiles_n, tiles;
   int* err;
 };
 
@@ -68,23 +73,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false (and records `code`) if the phase did not complete in time.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err, int code) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer();
-  while (!mbar_try_wait(bar, parity)) {
-    if (globaltimer() - t0 > WAIT_LIMIT_NS) {
-      atomicCAS(err, 0, code);
-      return false;
-    }
-  }
-  return true;
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
 }
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
       : "memory");
 }
 
@@ -128,32 +137,60 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-template <int BN, int STAGES>
-__global__ void __launch_bounds__(192, 1)
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Bounded wait that also gives up at once when another role of this CTA has already failed.
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* err, int code) {
+  if (mbar_test_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  unsigned spins = 0;
+  while (!mbar_test_wait(bar, parity)) {
+    if ((++spins & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer() - t0 > WAIT_LIMIT_NS) {
+        atomicCAS(err, 0, code);
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+// Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...  Tile = 128 rows x p.bn columns
+// (p.bn a multiple of 32, at most 256).  Two accumulators of 256 tensor-memory columns alternate so
+// that the epilogue of one tile overlaps the MMAs of the next.
+template <int STAGES>
+__global__ void __launch_bounds__(320, 1)
 gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
                  const Tf32Params p) {
-  constexpr int B_STAGE_BYTES = BN * BK * 4;
-  constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+  constexpr int B_STAGE_MAX = BN_MAX * BK * 4;
+  constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_MAX;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
   uint64_t* empty = full + STAGES;
-  uint64_t* tmem_full = empty + STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_full + 1);
+  uint64_t* acc_full = empty + STAGES;   // [2]
+  uint64_t* acc_empty = acc_full + 2;    // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile_m = blockIdx.x / p.tiles_n, tile_n = blockIdx.x % p.tiles_n;
-  const int m0 = tile_m * BM, n0 = tile_n * BN;
   const int total_kb = p.kblocks[0] + p.kblocks[1];
+  const int bn = p.bn;
+  const uint32_t stage_tx = A_STAGE_BYTES + (uint32_t)bn * BK * 4;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(tmem_full, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 8); }
+    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 2) {  // tensor-memory allocation: BN columns of 128 lanes x 32 bit
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN) : "memory");
+  if (warp == 2) {  // all 512 tensor-memory columns: two 128 x 256 FP32 accumulators
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -162,30 +199,40 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) {
-      // ---------------------------------------------------------------- producer
-      for (int kb = 0; kb < total_kb; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(&empty[s], ph ^ 1, p.err, 1)) break;
+    // ------------------------------------------------------------------ producer (TMA issue spread over lanes)
+    int it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < p.tiles && ok; t += gridDim.x) {
+      const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * bn;
+      for (int kb = 0; kb < total_kb; ++kb, ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1;
+        int good = 1;
+        if (lane == 0) good = wait_or_abort(&empty[s], ph ^ 1, abort_flag, p.err, 1) ? 1 : 0;
+        good = __shfl_sync(0xffffffffu, good, 0);
+        if (!good) { ok = false; break; }
+        if (lane == 0) mbar_expect_tx(&full[s], stage_tx);
+        __syncwarp();
         const int pair = kb < p.kblocks[0] ? 0 : 1;
         const int k0 = (pair == 0 ? kb : kb - p.kblocks[0]) * BK;
         const CUtensorMap* ma = pair == 0 ? &tmA0 : &tmA1;
         const CUtensorMap* mb = pair == 0 ? &tmB0 : &tmB1;
         uint8_t* sa = smem + s * STAGE_BYTES;
         uint8_t* sb = sa + A_STAGE_BYTES;
-        mbar_expect_tx(&full[s], STAGE_BYTES);
         if (!p.a_mn) {
-          tma_load_2d(sa, ma, k0, m0, &full[s]);
-        } else {
-#pragma unroll
-          for (int c = 0; c < BM / 32; ++c) tma_load_2d(sa + c * (BK * 128), ma, m0 + 32 * c, k0, &full[s]);
+          if (lane == 0) tma_load_2d(sa, ma, k0, m0, &full[s]);
+        } else if (p.a_3d) {
+          if (lane == 0) tma_load_3d(sa, ma, 0, k0, m0 / 32, &full[s]);
+        } else if (lane < BM / 32) {
+          tma_load_2d(sa + lane * (BK * 128), ma, m0 + 32 * lane, k0, &full[s]);
         }
         if (!p.b_mn) {
-          tma_load_2d(sb, mb, k0, n0, &full[s]);
-        } else {
-#pragma unroll
-          for (int c = 0; c < BN / 32; ++c) tma_load_2d(sb + c * (BK * 128), mb, n0 + 32 * c, k0, &full[s]);
+          if (lane == 8) tma_load_2d(sb, mb, k0, n0, &full[s]);
+        } else if (p.b_3d) {
+          if (lane == 8) tma_load_3d(sb, mb, 0, k0, n0 / 32, &full[s]);
+        } else if (lane >= 8 && lane < 8 + bn / 32) {
+          const int c = lane - 8;
+          tma_load_2d(sb + c * (BK * 128), mb, n0 + 32 * c, k0, &full[s]);
         }
       }
     }
@@ -194,87 +241,120 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant
       // ---------------------------------------------------------------- MMA issuer
       // instruction descriptor: D = F32, A = B = TF32, majors, N >> 3, M >> 4
       const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(p.a_mn ? 1 : 0) << 15) |
-                             ((uint32_t)(p.b_mn ? 1 : 0) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                             ((uint32_t)(p.b_mn ? 1 : 0) << 16) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
       const uint32_t a_step = p.a_mn ? 1024 : 32, b_step = p.b_mn ? 1024 : 32;
       const uint32_t a_sbo = p.a_mn ? 512 : 1024, b_sbo = p.b_mn ? 512 : 1024;
       const uint32_t a_lay = p.a_mn ? 1 : 2, b_lay = p.b_mn ? 1 : 2;
+      int it = 0, ti = 0;
       bool ok = true;
-      for (int kb = 0; kb < total_kb && ok; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        ok = mbar_wait(&full[s], ph, p.err, 2);
+      for (int t = blockIdx.x; t < p.tiles && ok; t += gridDim.x, ++ti) {
+        const int buf = ti & 1;
+        const uint32_t aph = (ti >> 1) & 1;
+        ok = wait_or_abort(&acc_empty[buf], aph ^ 1, abort_flag, p.err, 4);   // epilogue has drained this accumulator
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
-        const uint32_t sb = sa + A_STAGE_BYTES;
+        const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN_MAX);
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          ok = wait_or_abort(&full[s], ph, abort_flag, p.err, 2);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
+          const uint32_t sb = sa + A_STAGE_BYTES;
 #pragma unroll
-        for (int k = 0; k < BK / 8; ++k) {
-          const uint64_t ad = make_desc(sa + k * a_step, a_lbo, a_sbo, a_lay);
-          const uint64_t bd = make_desc(sb + k * b_step, b_lbo, b_sbo, b_lay);
-          mma_tf32(tmem_base, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < BK / 8; ++k) {
+            const uint64_t ad = make_desc(sa + k * a_step, a_lbo, a_sbo, a_lay);
+            const uint64_t bd = make_desc(sb + k * b_step, b_lbo, b_sbo, b_lay);
+            mma_tf32(tmem_d, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma_commit(&empty[s]);  // frees the slot once these MMAs have read it
         }
-        mma_commit(&empty[s]);  // frees the slot once these MMAs have read it
+        if (ok) mma_commit(&acc_full[buf]);
       }
-      mma_commit(tmem_full);    // accumulator complete (also reached after a timed-out wait)
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
-    const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 are this warp's
-    const bool ready = mbar_wait(tmem_full, 0, p.err, 3);
-    tc_fence_after();
-    const int m = m0 + quad * 32 + lane;
-    if (ready) {
-      const long long zrow = p.dsig ? (long long)(m % p.dsig_rows) * p.ld_dsig : 0;
-      for (int c = 0; c < BN / 32; ++c) {
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
+    // Two warps per tensor-memory quadrant; the pair alternates over the tile's 32-column chunks.
+    const int quad = warp & 3;            // tensor-memory lanes 32*quad .. 32*quad+31 are this warp's
+    const int half = (warp - 2) >> 2;     // 0 or 1: which chunks of the tile this warp takes
+    int ti = 0;
+    for (int t = blockIdx.x; t < p.tiles; t += gridDim.x, ++ti) {
+      const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * bn;
+      const int buf = ti & 1;
+      const uint32_t aph = (ti >> 1) & 1;
+      int good = 1;
+      if (lane == 0) good = wait_or_abort(&acc_full[buf], aph, abort_flag, p.err, 3) ? 1 : 0;
+      good = __shfl_sync(0xffffffffu, good, 0);
+      if (!good) break;
+      tc_fence_after();
+      // Registers only: the MMA's operand reads and the TMA writes already use all of the shared-memory
+      // bandwidth, so staging the tile through shared memory would starve.  Lane = row; every lane
+      // moves 16 bytes per access and a row's 128 bytes are completed by consecutive accesses.
+      const int m = m0 + quad * 32 + lane;
+      const bool m_ok = m < p.M;
+      const float* zrow = p.dsig ? p.dsig + (long long)(m % p.dsig_rows) * p.ld_dsig : nullptr;
+      const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
+      float* drow = p.D + (long long)m * p.ldd;
+      for (int c = half; c < bn / 32; c += 2) {
         const int nb = n0 + c * 32;
         if (nb >= p.N) break;               // warp-uniform
+        const bool full = p.vec_epi && nb + 32 <= p.N;   // warp-uniform: whole chunk in range and 16-byte aligned
+        float4 zc[8], ci[8];
+        if (full && m_ok) {                 // all global reads of the chunk in flight before anything waits
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            zc[q] = zrow ? __ldg(reinterpret_cast<const float4*>(zrow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            ci[q] = crow ? __ldg(reinterpret_cast<const float4*>(crow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
         float v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(c * 32), v);
-        if (m >= p.M) continue;
+        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
+        if (!m_ok) continue;
+        if (full) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const int n = nb + q * 4;
-          if (n >= p.N) break;
-          const int cnt = min(4, p.N - n);
-          const bool v4 = p.vec_epi && cnt == 4;
-          float bz[4] = {0.f, 0.f, 0.f, 0.f}, zc[4] = {0.f, 0.f, 0.f, 0.f}, ci[4] = {0.f, 0.f, 0.f, 0.f};
-          if (v4) {
-            if (p.bias) { const float4 x = __ldg(reinterpret_cast<const float4*>(p.bias + n)); bz[0] = x.x; bz[1] = x.y; bz[2] = x.z; bz[3] = x.w; }
-            if (p.dsig) { const float4 x = __ldg(reinterpret_cast<const float4*>(p.dsig + zrow + n)); zc[0] = x.x; zc[1] = x.y; zc[2] = x.z; zc[3] = x.w; }
-            if (p.cin)  { const float4 x = __ldg(reinterpret_cast<const float4*>(p.cin + (long long)m * p.ld_cin + n)); ci[0] = x.x; ci[1] = x.y; ci[2] = x.z; ci[3] = x.w; }
-          } else {
-            for (int j = 0; j < cnt; ++j) {
-              if (p.bias) bz[j] = __ldg(p.bias + n + j);
-              if (p.dsig) zc[j] = __ldg(p.dsig + zrow + n + j);
-              if (p.cin)  ci[j] = __ldg(p.cin + (long long)m * p.ld_cin + n + j);
+          for (int q = 0; q < 8; ++q) {
+            float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (p.bias) bz = __ldg(reinterpret_cast<const float4*>(p.bias + nb) + q);
+            float x[4] = {v[4 * q] + bz.x, v[4 * q + 1] + bz.y, v[4 * q + 2] + bz.z, v[4 * q + 3] + bz.w};
+            const float z[4] = {zc[q].x, zc[q].y, zc[q].z, zc[q].w};
+            const float cc[4] = {ci[q].x, ci[q].y, ci[q].z, ci[q].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (p.sigmoid) x[j] = 1.f / (1.f + __expf(-x[j]));
+              if (zrow) x[j] *= z[j] * (1.f - z[j]);
+              x[j] *= p.alpha;
+              if (crow) x[j] = fmaf(p.beta, cc[j], x[j]);
             }
+            reinterpret_cast<float4*>(drow + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
           }
-          float t[4];
+        } else {                             // ragged or unaligned chunk: element by element
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float x = v[q * 4 + j] + bz[j];
-            if (p.sigmoid) x = 1.f / (1.f + expf(-x));
-            if (p.dsig) x *= zc[j] * (1.f - zc[j]);
-            x *= p.alpha;
-            if (p.cin) x = fmaf(p.beta, ci[j], x);
-            t[j] = x;
-          }
-          float* dp = p.D + (long long)m * p.ldd + n;
-          if (v4) {
-            *reinterpret_cast<float4*>(dp) = make_float4(t[0], t[1], t[2], t[3]);
-          } else {
-            for (int j = 0; j < cnt; ++j) dp[j] = t[j];
+          for (int j = 0; j < 32; ++j) {
+            const int n = nb + j;
+            if (n < p.N) {
+              float x = v[j] + (p.bias ? __ldg(p.bias + n) : 0.f);
+              if (p.sigmoid) x = 1.f / (1.f + __expf(-x));
+              if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
+              x *= p.alpha;
+              if (crow) x = fmaf(p.beta, __ldg(crow + n), x);
+              drow[n] = x;
+            }
           }
         }
       }
+      // this warp has read its quadrant of the accumulator: let the MMA issuer reuse it
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
     }
-    tc_fence_before();
   }
+  tc_fence_before();
   __syncthreads();
   if (warp == 2) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
   }
 }
 
@@ -314,10 +394,54 @@ bool make_map(CUtensorMap* m, const float* base, long long rows, long long cols,
   return r == CUDA_SUCCESS;
 }
 
+// 3-D view of a row-major [K][MN] matrix (MN contiguous): (32 inner columns, K rows, MN/32 column chunks).
+// One box (32, BK, chunks) lands in shared memory as `chunks` consecutive [BK][32] blocks.  The last
+// chunk of a row may extend past MN (into the next row, or up to 124 bytes past the last row), so the
+// operand must be followed by that much readable memory.
+bool make_map_mn3d(CUtensorMap* m, const float* base, long long K, long long MN, long long ld, int chunks) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {32, (cuuint64_t)K, (cuuint64_t)((MN + 31) / 32)};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 4, 128};
+  cuuint32_t box[3] = {32, (cuuint32_t)BK, (cuuint32_t)chunks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_TFLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-constexpr int kBN = 256, kStages = 4;
-constexpr int kSmemBytes = kStages * (A_STAGE_BYTES + kBN * BK * 4) + 1024 + 256;
+constexpr int kStages = 4;
+constexpr int kSmemBytes = kStages * (A_STAGE_BYTES + BN_MAX * BK * 4) + 1024 + 256;
+
+int num_sms() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+// Tile width against wave quantisation: every CTA runs ceil(tiles / SMs) tiles.  Measured tile times
+// on B200 fit (320 + bn) units: the operand pipeline is latency-bound, so a narrower tile is only
+// slightly cheaper and the width that minimises the number of waves usually wins.
+int choose_bn(int M, int N) {
+  const long long tiles_m = (M + BM - 1) / BM;
+  const int sms = num_sms();
+  int best = 256;
+  long long best_cost = -1;
+  for (int bn = 256; bn >= 128; bn -= 32) {
+    const long long tiles = tiles_m * ((N + bn - 1) / bn);
+    const long long cost = ((tiles + sms - 1) / sms) * (320 + bn);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+  }
+  if (N <= 64) best = 64;
+  return best;
+}
 
 }  // namespace
 
@@ -332,9 +456,10 @@ bool gemm_tf32_eligible(const GemmArgs& g) {
 int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaFuncSetAttribute(gemm_tf32_kernel<kBN, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaFuncSetAttribute(gemm_tf32_kernel<kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     attr_set = true;
   }
+  const int bn = choose_bn(g.M, g.N);
   CUtensorMap maps[4];
   const float* As[2] = {g.A1, g.A2};
   const float* Bs[2] = {g.B1, g.B2};
@@ -344,10 +469,12 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
     const int src = As[s] ? s : 0;  // unused second pair: repeat the first (never dereferenced)
     bool ok;
     const CUtensorMapSwizzle kmaj = CU_TENSOR_MAP_SWIZZLE_128B, mnmaj = CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B;
-    if (g.a_kmajor) ok = make_map(&maps[2 * s], As[src], g.M, Ks[src], lda[src], BK, BM, kmaj);
-    else            ok = make_map(&maps[2 * s], As[src], Ks[src], g.M, lda[src], 32, BK, mnmaj);
-    if (g.b_kmajor) ok = ok && make_map(&maps[2 * s + 1], Bs[src], g.N, Ks[src], ldb[src], BK, kBN, kmaj);
-    else            ok = ok && make_map(&maps[2 * s + 1], Bs[src], Ks[src], g.N, ldb[src], 32, BK, mnmaj);
+    if (g.a_kmajor)      ok = make_map(&maps[2 * s], As[src], g.M, Ks[src], lda[src], BK, BM, kmaj);
+    else if (g.mn_padded) ok = make_map_mn3d(&maps[2 * s], As[src], Ks[src], g.M, lda[src], BM / 32);
+    else                 ok = make_map(&maps[2 * s], As[src], Ks[src], g.M, lda[src], 32, BK, mnmaj);
+    if (g.b_kmajor)      ok = ok && make_map(&maps[2 * s + 1], Bs[src], g.N, Ks[src], ldb[src], BK, bn, kmaj);
+    else if (g.mn_padded) ok = ok && make_map_mn3d(&maps[2 * s + 1], Bs[src], Ks[src], g.N, ldb[src], bn / 32);
+    else                 ok = ok && make_map(&maps[2 * s + 1], Bs[src], Ks[src], g.N, ldb[src], 32, BK, mnmaj);
     if (!ok) return -1;
   }
   Tf32Params p{};
@@ -355,6 +482,7 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   p.kblocks[0] = (Ks[0] + BK - 1) / BK;
   p.kblocks[1] = (Ks[1] + BK - 1) / BK;
   p.a_mn = g.a_kmajor ? 0 : 1; p.b_mn = g.b_kmajor ? 0 : 1;
+  p.a_3d = (p.a_mn && g.mn_padded) ? 1 : 0; p.b_3d = (p.b_mn && g.mn_padded) ? 1 : 0;
   p.D = g.D; p.ldd = g.ldd;
   p.bias = g.bias; p.sigmoid = g.sigmoid;
   p.dsig = g.dsig; p.ld_dsig = g.ld_dsig; p.dsig_rows = g.dsig_rows > 0 ? g.dsig_rows : 1;
@@ -363,10 +491,12 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   p.vec_epi = aligned16(g.D) && (g.ldd % 4 == 0) && (!g.bias || aligned16(g.bias)) &&
               (!g.dsig || (aligned16(g.dsig) && g.ld_dsig % 4 == 0)) &&
               (!g.cin || (aligned16(g.cin) && g.ld_cin % 4 == 0));
-  p.tiles_n = (g.N + kBN - 1) / kBN;
+  p.bn = bn;
+  p.tiles_n = (g.N + bn - 1) / bn;
+  p.tiles = ((g.M + BM - 1) / BM) * p.tiles_n;
   p.err = err_flag;
-  const long long tiles = (long long)((g.M + BM - 1) / BM) * p.tiles_n;
-  gemm_tf32_kernel<kBN, kStages><<<(unsigned)tiles, 192, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  const int grid = p.tiles < num_sms() ? p.tiles : num_sms();
+  gemm_tf32_kernel<kStages><<<grid, 320, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
   return 1;
 }
 

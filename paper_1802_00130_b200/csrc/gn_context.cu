@@ -92,7 +92,9 @@ gn_status dev_alloc(gn_ctx* c, T** p, int64_t count) {
   *p = nullptr;
   if (count <= 0) count = 1;
   void* q = nullptr;
-  cudaError_t e = cudaMalloc(&q, (size_t)count * sizeof(T));
+  // 256 bytes of slack: the tensor-core kernel's 3-D TMA boxes may read up to 124 bytes past the last
+  // row of an MN-major operand
+  cudaError_t e = cudaMalloc(&q, (size_t)count * sizeof(T) + 256);
   if (e != cudaSuccess) {
     cudaGetLastError();
     return fail(c, GN_ENOMEM, std::string("cudaMalloc of ") + std::to_string(count * (int64_t)sizeof(T)) + " bytes: " + cudaGetErrorString(e));
@@ -218,8 +220,9 @@ void forward_pass(gn_ctx* c, const float* Z0, int64_t rows, std::vector<float*>&
 // Parameter-space half of the backward pass for one layer (Eqs. xtow-g, xtow-g-bias, and their
 // Jacobian twins of Section 4.2): out_W = alpha ds^T Zprev + beta cin_W, out_b = alpha 1^T ds + beta cin_b.
 gn_status weight_block(gn_ctx* c, int m, const float* ds, const float* Zprev, int64_t rows, float alpha,
-                       const float* cin, float beta, float* out) {
+                       const float* cin, float beta, float* out, bool padded = true) {
   GemmArgs g;
+  g.mn_padded = padded;   // ds and Zprev are context-owned (padded) unless the caller says otherwise
   g.M = c->w[m]; g.N = c->w[m - 1];
   g.A1 = ds; g.lda1 = c->w[m]; g.a_kmajor = false;
   g.B1 = Zprev; g.ldb1 = c->w[m - 1]; g.b_kmajor = false;
@@ -244,6 +247,7 @@ void backward_data(gn_ctx* c, int m, const float* ds, int64_t rows, const float*
   g.K1 = c->w[m];
   g.dsig = Zprev; g.ld_dsig = c->w[m - 1]; g.dsig_rows = (int)z_rows;
   g.D = dst; g.ldd = c->w[m - 1];
+  g.mn_padded = true;     // B is the context's own (padded) copy of theta
   run_gemm(c, g);
 }
 
@@ -355,8 +359,17 @@ gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
     if (d_grad) {
       for (int m = L; m >= 1; --m) {
         const float* Zprev = m == 1 ? X0 : c->Zb[m - 1];
-        if (b == 0) GN_TRY(weight_block(c, m, c->Db[m], Zprev, rows, inv_l, c->theta, inv_C, d_grad));
-        else        GN_TRY(weight_block(c, m, c->Db[m], Zprev, rows, inv_l, d_grad, 1.f, d_grad));
+        const float* cin0 = b == 0 ? c->theta : d_grad;
+        const float beta0 = b == 0 ? inv_C : 1.f;
+        if (m == 1 && r0 + rows == c->l && rows > 64) {
+          // layer 1 reads the caller's X, which has no slack after its last row: all but the final 32
+          // rows use the padded fast path, the rest is added by a second, unpadded contraction
+          const int64_t head = rows - 32;
+          GN_TRY(weight_block(c, 1, c->Db[1], X0, head, inv_l, cin0, beta0, d_grad, true));
+          GN_TRY(weight_block(c, 1, c->Db[1] + head * c->w[1], X0 + head * c->w[0], 32, inv_l, d_grad, 1.f, d_grad, false));
+        } else {
+          GN_TRY(weight_block(c, m, c->Db[m], Zprev, rows, inv_l, cin0, beta0, d_grad, !(m == 1 && r0 + rows == c->l)));
+        }
         if (m > 1) backward_data(c, m, c->Db[m], rows, c->Zb[m - 1], rows, c->Db[m - 1]);
       }
     }
@@ -691,12 +704,14 @@ gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t
 gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* dA, int64_t lda, int a_kmajor,
                         const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd) {
   if (!c) return GN_EINVAL;
-  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 2) return fail(c, GN_EINVAL, "bad GEMM arguments");
+  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 3) return fail(c, GN_EINVAL, "bad GEMM arguments");
   GemmArgs g;
   g.M = M; g.N = N; g.K1 = K;
   g.A1 = dA; g.lda1 = lda; g.a_kmajor = a_kmajor != 0;
   g.B1 = dB; g.ldb1 = ldb; g.b_kmajor = b_kmajor != 0;
   g.D = dD; g.ldd = ldd;
+  g.mn_padded = (kind == 3);   // kind 3: tensor-core kernel, MN-major operands declared padded
+  if (kind == 3) kind = 0;
   if (kind == 0 && !gemm_tf32_eligible(g)) return fail(c, GN_EINVAL, "operands do not qualify for the tensor-core kernel");
   if (kind == 2) {
     if (gemm_thin_kind(g) == THIN_NONE) return fail(c, GN_EINVAL, "operands do not qualify for a streaming kernel");

@@ -23,6 +23,7 @@ struct GemmArgs {
   const float* A1 = nullptr; const float* B1 = nullptr; int K1 = 0; int64_t lda1 = 0, ldb1 = 0;
   const float* A2 = nullptr; const float* B2 = nullptr; int K2 = 0; int64_t lda2 = 0, ldb2 = 0;
   bool a_kmajor = true, b_kmajor = true;
+  bool mn_padded = false;  // every MN-major operand is followed by >= 128 readable bytes
   float* D = nullptr; int64_t ldd = 0;
   const float* bias = nullptr;
   bool sigmoid = false;
