@@ -201,6 +201,37 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
                         int a_kmajor, const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd);
 
 /*
+ * gn_thin_m_gemm_noalloc - D[M][N] = sum_r A[r][m] B[r][n] for M <= 16 (the shape of the output layer's
+ * weight block, rows = |S| or a row batch) without a context and without allocating anything.
+ * The paper has no counterpart to this call; it exists for callers that must not allocate device memory
+ * while they run: code living inside a host application whose own allocator holds all of the GPU's memory
+ * (a cudaMalloc from a library would fail or fragment it), jobs started under a fixed device-memory
+ * budget, and latency-critical loops that cannot take the device-wide synchronisation an allocation may
+ * cause.  It runs the same two kernels as the context's thin-M path (gn_debug_gemm kind 2 with both
+ * operands row-major over r); only the scratch differs: the per-row-chunk partial sums go to an 8 MiB
+ * array that is part of the library image (every GPU that loads the library holds it until the process
+ * exits) instead of a cudaMalloc'ed buffer.
+ *   M, N, rows     1 <= M <= 16; N a multiple of 4; rows >= 1.
+ *   dA             device [rows][lda], lda >= M: A[r][m].
+ *   dB             device [rows][ldb], ldb >= N, a multiple of 4, 16-byte aligned: B[r][n].
+ *   dD             device [M][ldd], ldd >= N: the result; must not overlap dA or dB.
+ *   cuda_stream    stream to enqueue on (NULL = legacy default stream); the call does not synchronise.
+ *   errbuf         optional host buffer of errbuf_len bytes that receives the reason for a failure.
+ * Limit: (row chunks) x M x N <= 2 097 152 floats, where row chunks = min(ceil(296 / ceil(N/512)),
+ * ceil(rows/64)); a larger problem returns GN_EINVAL and launches nothing (e.g. M = 10, N = 2000 fits for
+ * any rows; M = 16, N = 4096 does not once rows > 2048).
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress) with that
+ * device current; make that first call outside any stream capture.  No cudaMalloc, cudaFree or other
+ * allocating routine is called, on the first call or later.
+ * All calls share the one array, which keeps the previous call's partial sums: every element that a call
+ * reads it has written first, so nothing needs clearing, but two calls whose kernels may overlap on the
+ * GPU (different streams, or different host threads) race on it - serialise them.
+ */
+gn_status gn_thin_m_gemm_noalloc(int M, int N, int64_t rows, const float* dA, int64_t lda, const float* dB,
+                                 int64_t ldb, float* dD, int64_t ldd, void* cuda_stream, char* errbuf,
+                                 int64_t errbuf_len);
+
+/*
  * gn_kernel_launches - number of kernels this context has launched so far (all entry points).
  */
 int64_t gn_kernel_launches(const gn_ctx* ctx);

@@ -37,6 +37,7 @@ _SIGNATURES = {
     "gn_debug_activations": (_i32, [_vp, _i32, _vp]),
     "gn_profile": (_i32, [_vp, _i32]),
     "gn_profile_read": (_i32, [_vp, C.POINTER(_dbl), C.POINTER(_dbl), C.POINTER(_i64)]),
+    "gn_thin_m_gemm_noalloc": (_i32, [_i32, _i32, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp, C.c_char_p, _i64]),
     "gn_debug_gemm": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64]),
 }
 
@@ -88,6 +89,31 @@ def _host_ptr(a, dtype, count=None):
     if count is not None and a.size != count:
         raise ValueError(f"expected {count} elements, got {a.size}")
     return _vp(a.ctypes.data)
+
+
+def thin_m_gemm_noalloc(A, B, out, stream=None):
+    """out[M][N] = sum_r A[r][m] B[r][n], M <= 16, through gn_thin_m_gemm_noalloc.
+
+    For callers that cannot allocate device memory: the library call itself allocates nothing (its
+    scratch is a fixed array inside the library), and this wrapper allocates nothing either - the
+    caller brings `out`.  A [rows][M], B [rows][N], out [M][N]: CUDA float32, rows may be strided
+    (stride(0) is the leading dimension).  Raises GnError with the library's message on failure.
+    """
+    import torch
+    for t in (A, B, out):
+        if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.dim() == 2 and t.stride(1) == 1):
+            raise TypeError("expected 2-D CUDA float32 tensors with unit inner stride")
+    rows, M = A.shape
+    N = B.shape[1]
+    if B.shape[0] != rows or tuple(out.shape) != (M, N):
+        raise ValueError("shapes must be A [rows][M], B [rows][N], out [M][N]")
+    st = stream if stream is not None else torch.cuda.current_stream(A.device)
+    msg = C.create_string_buffer(256)
+    rc = lib().gn_thin_m_gemm_noalloc(M, N, rows, _vp(A.data_ptr()), A.stride(0), _vp(B.data_ptr()), B.stride(0),
+                                      _vp(out.data_ptr()), out.stride(0), _vp(st.cuda_stream), msg, 256)
+    if rc != 0:
+        raise GnError(rc, msg.value.decode())
+    return out
 
 
 class GnContext:

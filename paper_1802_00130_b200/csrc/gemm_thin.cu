@@ -6,6 +6,9 @@
 //   thin-K : D[M][N] = (sum_k A[m][k] B[k][n]) * epilogue, K <= 16              (back-propagation out of layer L)
 //
 // All use the common epilogue of GemmArgs.  Deterministic: fixed-order reductions, no atomics.
+#include <cstdio>
+
+#include "../../include/gn.h"
 #include "gn_kernels.h"
 
 namespace gn {
@@ -303,3 +306,68 @@ int launch_gemm_thin(const GemmArgs& g, float* scratch, cudaStream_t st) {
 }
 
 }  // namespace gn
+
+// ------------------------------------------------------------------------------------ allocation-free thin-M entry
+// Scratch for gn_thin_m_gemm_noalloc: a fixed array inside the library image instead of a buffer from
+// cudaMalloc.  Every device that loads the library carries these 8 MiB until the process exits.
+namespace {
+constexpr long long kNoAllocScratchFloats = 2097152;   // 8 MiB
+static __device__ __align__(256) float g_noalloc_scratch[kNoAllocScratchFloats];
+
+constexpr int kMaxDevices = 64;
+float* g_noalloc_ptr[kMaxDevices] = {};   // device address of the array, looked up once per device
+
+void put_msg(char* buf, int64_t len, const char* msg) {
+  if (buf && len > 0) snprintf(buf, (size_t)len, "%s", msg);
+}
+}  // namespace
+
+extern "C" gn_status gn_thin_m_gemm_noalloc(int M, int N, int64_t rows, const float* dA, int64_t lda, const float* dB,
+                                            int64_t ldb, float* dD, int64_t ldd, void* cuda_stream, char* errbuf,
+                                            int64_t errbuf_len) {
+  using namespace gn;
+  if (!dA || !dB || !dD || M < 1 || N < 1 || rows < 1 || lda < M || ldb < N || ldd < N) {
+    put_msg(errbuf, errbuf_len, "null pointer, non-positive size, or leading dimension smaller than the row length");
+    return GN_EINVAL;
+  }
+  if (rows > 0x7fffffffLL) { put_msg(errbuf, errbuf_len, "rows exceeds 2^31 - 1"); return GN_EINVAL; }
+  GemmArgs g;
+  g.M = M; g.N = N; g.K1 = (int)rows;
+  g.A1 = dA; g.lda1 = lda; g.a_kmajor = false;
+  g.B1 = dB; g.ldb1 = ldb; g.b_kmajor = false;
+  g.D = dD; g.ldd = ldd;
+  if (gemm_thin_kind(g) != THIN_M) {
+    put_msg(errbuf, errbuf_len, "shape not taken: needs M <= 16, N a multiple of 4, B 16-byte aligned with ldb a multiple of 4");
+    return GN_EINVAL;
+  }
+  const long long need = gemm_thin_scratch_floats(g);
+  if (need > kNoAllocScratchFloats) {
+    char msg[200];
+    snprintf(msg, sizeof msg, "problem needs %lld scratch floats (row chunks x M x N); the built-in scratch holds %lld",
+             need, kNoAllocScratchFloats);
+    put_msg(errbuf, errbuf_len, msg);
+    return GN_EINVAL;
+  }
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    put_msg(errbuf, errbuf_len, "no current CUDA device (or device ordinal >= 64)");
+    return GN_ECUDA;
+  }
+  if (!g_noalloc_ptr[dev]) {
+    // In host code the array's name is only a handle; the kernels need its address on this device.
+    float* ptr = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch);
+    if (e != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      put_msg(errbuf, errbuf_len, cudaGetErrorString(e));
+      return GN_ECUDA;
+    }
+    g_noalloc_ptr[dev] = ptr;
+  }
+  launch_gemm_thin(g, g_noalloc_ptr[dev], static_cast<cudaStream_t>(cuda_stream));
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { put_msg(errbuf, errbuf_len, cudaGetErrorString(e)); return GN_ECUDA; }
+  put_msg(errbuf, errbuf_len, "");
+  return GN_OK;
+}
