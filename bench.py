@@ -53,6 +53,21 @@ def mac_counts(widths):
     return dict(fwd=fwd, grad=grad, full=full, block_executed=b1, block_paper=paper_block)
 
 
+def max_over_ranks(value, dist, device):
+    """Slowest rank's time: the timed region of a multi-process run ends when the last rank ends."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(products_per_rank, world, ms):
+    """Replicas only: every rank does the same number of products; the job's rate uses the slowest rank."""
+    return products_per_rank * world / (ms * 1e-3)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks / throttle reasons for one GPU while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -212,12 +227,9 @@ def run_ours(args):
     ctx.profile(False)
     launches = ctx.kernel_launches - launches0
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
-    if dist:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, dev)
     matvecs = 2 * n_cg * args.steps * world
-    value = matvecs / (ms * 1e-3)
+    value = whole_job_rate(2 * n_cg * args.steps, world, ms)
 
     # ---- product-only rates (device-resident, outside the step timing)
     v = torch.from_numpy(p["v"]).to(dev)
@@ -261,10 +273,7 @@ def run_ours(args):
     e1.record()
     barrier()
     ms_e2e = e0.elapsed_time(e1)
-    if dist:
-        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    ms_e2e = max_over_ranks(ms_e2e, dist, dev)
     n4 = 4 * ctx.n
     e2e = {"value": matvecs / (ms_e2e * 1e-3), "unit": UNIT,
            "h2d_bytes_per_step": n4 + 4 * p["nS"] + 2 * n4, "d2h_bytes_per_step": n4 + 2 * n4}
