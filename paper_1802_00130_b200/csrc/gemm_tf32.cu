@@ -64,15 +64,6 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
 __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -358,6 +349,257 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Two-CTA variant: a cluster of two CTAs (two SMs) computes one 256 x bn tile with
+// tcgen05.mma.cta_group::2.  CTA r of the pair owns rows [128 r, 128 r + 128) of the tile (its A block
+// and its accumulator) and stages half of the B tile (bn/2 rows); the tensor cores of both SMs read
+// both halves.  Per k-block each SM therefore moves 16 KB + 16 KB instead of 16 KB + 32 KB through
+// shared memory, which is what limits the one-CTA kernel.
+// Protocol: both producers wait on their own empty[s] (released in both CTAs by a multicast commit),
+// only the leader (rank 0) arms full[s] with the bytes of both CTAs, and both CTAs' TMA loads complete
+// on the leader's full[s].  MMAs are issued by the leader only.  acc_full[b] is multicast to both
+// CTAs; all 16 epilogue warps of the pair arrive on the leader's acc_empty[b].
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+  return r;
+}
+// Cluster-wide barrier.  Warps may arrive here after divergent role code, so they reconverge first
+// and the non-aligned forms are used.
+__device__ __forceinline__ void cluster_sync_all() {
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma2_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ __forceinline__ void tma2_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ __forceinline__ void mma2_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
+}
+// commit of the pair's MMAs, arriving on the barrier at this offset in both CTAs
+__device__ __forceinline__ void mma2_commit_both(uint64_t* bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"(mask) : "memory");
+}
+
+constexpr int B2_STAGE_MAX = (BN_MAX / 2) * BK * 4;          // 16 KB: this CTA's half of the B tile
+constexpr int STAGE2_BYTES = A_STAGE_BYTES + B2_STAGE_MAX;   // 32 KB
+
+template <int STAGES>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(320, 1)
+gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                      const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
+                      const Tf32Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE2_BYTES);
+  uint64_t* empty = full + STAGES;
+  uint64_t* acc_full = empty + STAGES;   // [2]
+  uint64_t* acc_empty = acc_full + 2;    // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int total_kb = p.kblocks[0] + p.kblocks[1];
+  const int bn = p.bn, hb = p.bn >> 1;                       // hb: B rows staged by each CTA
+  const uint32_t pair_tx = 2u * (A_STAGE_BYTES + (uint32_t)hb * BK * 4);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 16); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 2) {  // both CTAs of the pair allocate all 512 columns, same warp, same destination offset
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  cluster_sync_all();      // barriers of both CTAs are initialised before anyone signals across the pair
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer (both CTAs)
+    int it = 0;
+    bool ok = true;
+    for (int t = pair; t < p.tiles && ok; t += n_pairs) {
+      const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM;
+      const int n0 = (t % p.tiles_n) * bn + (int)rank * hb;
+      for (int kb = 0; kb < total_kb; ++kb, ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1;
+        int good = 1;
+        if (lane == 0) good = wait_or_abort(&empty[s], ph ^ 1, abort_flag, p.err, 1) ? 1 : 0;
+        good = __shfl_sync(0xffffffffu, good, 0);
+        if (!good) { ok = false; break; }
+        if (rank == 0 && lane == 0) mbar_expect_tx(&full[s], pair_tx);
+        __syncwarp();
+        const uint32_t full_leader = map_to_cta(smem_u32(&full[s]), 0);
+        const int pr = kb < p.kblocks[0] ? 0 : 1;
+        const int k0 = (pr == 0 ? kb : kb - p.kblocks[0]) * BK;
+        const CUtensorMap* ma = pr == 0 ? &tmA0 : &tmA1;
+        const CUtensorMap* mb = pr == 0 ? &tmB0 : &tmB1;
+        uint8_t* sa = smem + s * STAGE2_BYTES;
+        uint8_t* sb = sa + A_STAGE_BYTES;
+        if (!p.a_mn) {
+          if (lane == 0) tma2_load_2d(sa, ma, k0, m0, full_leader);
+        } else if (p.a_3d) {
+          if (lane == 0) tma2_load_3d(sa, ma, 0, k0, m0 / 32, full_leader);
+        } else if (lane < BM / 32) {
+          tma2_load_2d(sa + lane * (BK * 128), ma, m0 + 32 * lane, k0, full_leader);
+        }
+        if (!p.b_mn) {
+          if (lane == 8) tma2_load_2d(sb, mb, k0, n0, full_leader);
+        } else if (p.b_3d) {
+          if (lane == 8) tma2_load_3d(sb, mb, 0, k0, n0 / 32, full_leader);
+        } else if (lane >= 8 && lane < 8 + hb / 32) {
+          const int c = lane - 8;
+          tma2_load_2d(sb + c * (BK * 128), mb, n0 + 32 * c, k0, full_leader);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0 && lane == 0) {
+      // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+      const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(p.a_mn ? 1 : 0) << 15) |
+                             ((uint32_t)(p.b_mn ? 1 : 0) << 16) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+      const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
+      const uint32_t a_step = p.a_mn ? 1024 : 32, b_step = p.b_mn ? 1024 : 32;
+      const uint32_t a_sbo = p.a_mn ? 512 : 1024, b_sbo = p.b_mn ? 512 : 1024;
+      const uint32_t a_lay = p.a_mn ? 1 : 2, b_lay = p.b_mn ? 1 : 2;
+      int it = 0, ti = 0;
+      bool ok = true;
+      for (int t = pair; t < p.tiles && ok; t += n_pairs, ++ti) {
+        const int buf = ti & 1;
+        const uint32_t aph = (ti >> 1) & 1;
+        ok = wait_or_abort(&acc_empty[buf], aph ^ 1, abort_flag, p.err, 4);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN_MAX);
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          ok = wait_or_abort(&full[s], ph, abort_flag, p.err, 2);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + s * STAGE2_BYTES);
+          const uint32_t sb = sa + A_STAGE_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 8; ++k) {
+            const uint64_t ad = make_desc(sa + k * a_step, a_lbo, a_sbo, a_lay);
+            const uint64_t bd = make_desc(sb + k * b_step, b_lbo, b_sbo, b_lay);
+            mma2_tf32(tmem_d, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma2_commit_both(&empty[s]);
+        }
+        if (ok) mma2_commit_both(&acc_full[buf]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
+    int ti = 0;
+    for (int t = pair; t < p.tiles; t += n_pairs, ++ti) {
+      const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM, n0 = (t % p.tiles_n) * bn;
+      const int buf = ti & 1;
+      const uint32_t aph = (ti >> 1) & 1;
+      int good = 1;
+      if (lane == 0) good = wait_or_abort(&acc_full[buf], aph, abort_flag, p.err, 3) ? 1 : 0;
+      good = __shfl_sync(0xffffffffu, good, 0);
+      if (!good) break;
+      tc_fence_after();
+      const int m = m0 + quad * 32 + lane;
+      const bool m_ok = m < p.M;
+      const float* zrow = p.dsig ? p.dsig + (long long)(m % p.dsig_rows) * p.ld_dsig : nullptr;
+      const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
+      float* drow = p.D + (long long)m * p.ldd;
+      for (int c = half; c < bn / 32; c += 2) {
+        const int nb = n0 + c * 32;
+        if (nb >= p.N) break;
+        const bool fullc = p.vec_epi && nb + 32 <= p.N;
+        float4 zc[8], ci[8];
+        if (fullc && m_ok) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            zc[q] = zrow ? __ldg(reinterpret_cast<const float4*>(zrow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            ci[q] = crow ? __ldg(reinterpret_cast<const float4*>(crow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
+        float v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
+        if (!m_ok) continue;
+        if (fullc) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (p.bias) bz = __ldg(reinterpret_cast<const float4*>(p.bias + nb) + q);
+            float x[4] = {v[4 * q] + bz.x, v[4 * q + 1] + bz.y, v[4 * q + 2] + bz.z, v[4 * q + 3] + bz.w};
+            const float z[4] = {zc[q].x, zc[q].y, zc[q].z, zc[q].w};
+            const float cc[4] = {ci[q].x, ci[q].y, ci[q].z, ci[q].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (p.sigmoid) x[j] = 1.f / (1.f + __expf(-x[j]));
+              if (zrow) x[j] *= z[j] * (1.f - z[j]);
+              x[j] *= p.alpha;
+              if (crow) x[j] = fmaf(p.beta, cc[j], x[j]);
+            }
+            reinterpret_cast<float4*>(drow + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int n = nb + j;
+            if (n < p.N) {
+              float x = v[j] + (p.bias ? __ldg(p.bias + n) : 0.f);
+              if (p.sigmoid) x = 1.f / (1.f + __expf(-x));
+              if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
+              x *= p.alpha;
+              if (crow) x = fmaf(p.beta, __ldg(crow + n), x);
+              drow[n] = x;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
+    }
+  }
+  tc_fence_before();
+  cluster_sync_all();      // neither CTA leaves (or frees tensor memory) while the other may still use it
+  if (warp == 2) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
 // ---- host side ---------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -453,13 +695,37 @@ bool gemm_tf32_eligible(const GemmArgs& g) {
   return true;
 }
 
+constexpr int kStages2 = 6;
+constexpr int kSmemBytes2 = kStages2 * STAGE2_BYTES + 1024 + 256;
+
+// Two-CTA tile width (a multiple of 64 so that each CTA's half is whole 32-column chunks).
+int choose_bn2(int M, int N) {
+  const long long tiles_m = (M + 2 * BM - 1) / (2 * BM);
+  const int pairs = num_sms() / 2;
+  int best = 256;
+  long long best_cost = -1;
+  for (int bn = 256; bn >= 128; bn -= 64) {
+    const long long tiles = tiles_m * ((N + bn - 1) / bn);
+    const long long cost = ((tiles + pairs - 1) / pairs) * (320 + bn);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+  }
+  return best;
+}
+
 int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaFuncSetAttribute(gemm_tf32_kernel<kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     attr_set = true;
   }
-  const int bn = choose_bn(g.M, g.N);
+  static bool attr2_set = false;
+  if (!attr2_set) {
+    cudaFuncSetAttribute(gemm_tf32_2cta_kernel<kStages2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+    attr2_set = true;
+  }
+  const bool two_cta = g.two_cta >= 0 ? g.two_cta != 0 : (g.M > BM && g.N >= 128);
+  const int bn = two_cta ? choose_bn2(g.M, g.N) : choose_bn(g.M, g.N);
+  const int b_rows = two_cta ? bn / 2 : bn;      // B rows staged per CTA
   CUtensorMap maps[4];
   const float* As[2] = {g.A1, g.A2};
   const float* Bs[2] = {g.B1, g.B2};
@@ -472,8 +738,8 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
     if (g.a_kmajor)      ok = make_map(&maps[2 * s], As[src], g.M, Ks[src], lda[src], BK, BM, kmaj);
     else if (g.mn_padded) ok = make_map_mn3d(&maps[2 * s], As[src], Ks[src], g.M, lda[src], BM / 32);
     else                 ok = make_map(&maps[2 * s], As[src], Ks[src], g.M, lda[src], 32, BK, mnmaj);
-    if (g.b_kmajor)      ok = ok && make_map(&maps[2 * s + 1], Bs[src], g.N, Ks[src], ldb[src], BK, bn, kmaj);
-    else if (g.mn_padded) ok = ok && make_map_mn3d(&maps[2 * s + 1], Bs[src], Ks[src], g.N, ldb[src], bn / 32);
+    if (g.b_kmajor)      ok = ok && make_map(&maps[2 * s + 1], Bs[src], g.N, Ks[src], ldb[src], BK, b_rows, kmaj);
+    else if (g.mn_padded) ok = ok && make_map_mn3d(&maps[2 * s + 1], Bs[src], Ks[src], g.N, ldb[src], b_rows / 32);
     else                 ok = ok && make_map(&maps[2 * s + 1], Bs[src], Ks[src], g.N, ldb[src], 32, BK, mnmaj);
     if (!ok) return -1;
   }
@@ -493,10 +759,17 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
               (!g.cin || (aligned16(g.cin) && g.ld_cin % 4 == 0));
   p.bn = bn;
   p.tiles_n = (g.N + bn - 1) / bn;
-  p.tiles = ((g.M + BM - 1) / BM) * p.tiles_n;
   p.err = err_flag;
-  const int grid = p.tiles < num_sms() ? p.tiles : num_sms();
-  gemm_tf32_kernel<kStages><<<grid, 320, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  if (two_cta) {
+    p.tiles = ((g.M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;   // tiles of 256 rows, one per CTA pair
+    const int pairs = num_sms() / 2;
+    const int grid = 2 * (p.tiles < pairs ? p.tiles : pairs);
+    gemm_tf32_2cta_kernel<kStages2><<<grid, 320, kSmemBytes2, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  } else {
+    p.tiles = ((g.M + BM - 1) / BM) * p.tiles_n;
+    const int grid = p.tiles < num_sms() ? p.tiles : num_sms();
+    gemm_tf32_kernel<kStages><<<grid, 320, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  }
   return 1;
 }
 

@@ -704,14 +704,18 @@ gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t
 gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* dA, int64_t lda, int a_kmajor,
                         const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd) {
   if (!c) return GN_EINVAL;
-  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 3) return fail(c, GN_EINVAL, "bad GEMM arguments");
+  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 5) return fail(c, GN_EINVAL, "bad GEMM arguments");
   GemmArgs g;
   g.M = M; g.N = N; g.K1 = K;
   g.A1 = dA; g.lda1 = lda; g.a_kmajor = a_kmajor != 0;
   g.B1 = dB; g.ldb1 = ldb; g.b_kmajor = b_kmajor != 0;
   g.D = dD; g.ldd = ldd;
-  g.mn_padded = (kind == 3);   // kind 3: tensor-core kernel, MN-major operands declared padded
-  if (kind == 3) kind = 0;
+  // kinds 3..5 are the tensor-core kernel with options: 3 = MN-major operands declared padded,
+  // 4 = one CTA per tile forced, 5 = CTA pair per tile forced (both with padded operands)
+  g.mn_padded = (kind >= 3);
+  if (kind == 4) g.two_cta = 0;
+  if (kind == 5) g.two_cta = 1;
+  if (kind >= 3) kind = 0;
   if (kind == 0 && !gemm_tf32_eligible(g)) return fail(c, GN_EINVAL, "operands do not qualify for the tensor-core kernel");
   if (kind == 2) {
     if (gemm_thin_kind(g) == THIN_NONE) return fail(c, GN_EINVAL, "operands do not qualify for a streaming kernel");

@@ -24,6 +24,7 @@ struct GemmArgs {
   const float* A2 = nullptr; const float* B2 = nullptr; int K2 = 0; int64_t lda2 = 0, ldb2 = 0;
   bool a_kmajor = true, b_kmajor = true;
   bool mn_padded = false;  // every MN-major operand is followed by >= 128 readable bytes
+  int two_cta = -1;        // tensor-core kernel: -1 choose, 0 one CTA per tile, 1 CTA pair per 256-row tile
   float* D = nullptr; int64_t ldd = 0;
   const float* bias = nullptr;
   bool sigmoid = false;
