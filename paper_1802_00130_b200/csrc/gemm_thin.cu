@@ -49,7 +49,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // ------------------------------------------------------------------------------------ thin-N
 // One warp per group of TR rows; lanes stride K in float4 steps; B rows come through L1.
-constexpr int TR = 8;
+constexpr int TR = 4;
 
 struct ThinNParams {
   int M, N;
@@ -58,7 +58,7 @@ struct ThinNParams {
 };
 
 template <int NMAX>
-__global__ void __launch_bounds__(256) gemm_thin_n_kernel(const ThinNParams p) {
+__global__ void __launch_bounds__(256, 2) gemm_thin_n_kernel(const ThinNParams p) {
   const int lane = threadIdx.x & 31;
   const int warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int m0 = warp * TR;
@@ -74,13 +74,18 @@ __global__ void __launch_bounds__(256) gemm_thin_n_kernel(const ThinNParams p) {
     const float* __restrict__ B = p.B[s];
     if (!A) continue;
     const int K = p.K[s];
-    for (int k = lane * 4; k < K; k += 128) {
-      float4 a[TR];
+    const float* arow[TR];
 #pragma unroll
-      for (int r = 0; r < TR; ++r) {
-        const int m = min(m0 + r, p.M - 1);          // clamp: duplicate rows are never written
-        a[r] = __ldg(reinterpret_cast<const float4*>(A + (long long)m * p.lda[s] + k));
-      }
+    for (int r = 0; r < TR; ++r) arow[r] = A + (long long)min(m0 + r, p.M - 1) * p.lda[s];   // clamped rows are never written
+    // software pipeline: the A rows of the next k-step are requested before this step's arithmetic
+    float4 a[TR], an[TR];
+    int k = lane * 4;
+#pragma unroll
+    for (int r = 0; r < TR; ++r) a[r] = k < K ? __ldg(reinterpret_cast<const float4*>(arow[r] + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (; k < K; k += 128) {
+      const int kn = k + 128;
+#pragma unroll
+      for (int r = 0; r < TR; ++r) an[r] = kn < K ? __ldg(reinterpret_cast<const float4*>(arow[r] + kn)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int n = 0; n < NMAX; ++n) {
         if (n < p.N) {
@@ -94,6 +99,8 @@ __global__ void __launch_bounds__(256) gemm_thin_n_kernel(const ThinNParams p) {
           }
         }
       }
+#pragma unroll
+      for (int r = 0; r < TR; ++r) a[r] = an[r];
     }
   }
 #pragma unroll
@@ -192,6 +199,7 @@ __global__ void __launch_bounds__(128) gemm_thin_k_kernel(const ThinKParams p) {
   if (p.e.bias) bz = __ldg(reinterpret_cast<const float4*>(p.e.bias + n));
   const int m_begin = blockIdx.y * p.rows_per_block;
   const int m_end = min(p.M, m_begin + p.rows_per_block);
+#pragma unroll 4
   for (int m = m_begin; m < m_end; ++m) {
     float4 acc = bz;
 #pragma unroll

@@ -59,9 +59,9 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const float* __restric
 }
 
 // ---------------------------------------------------------------------------------- column sums
-constexpr int CS_ROWS = 512;  // rows per block
+constexpr int CS_ROWS = 256;  // rows per block
 
-// grid (ceil(cols/32), ceil(rows/CS_ROWS)); 256 threads = 8 warps striding rows, lanes along columns.
+// Scalar version (any alignment): grid (ceil(cols/32), ceil(rows/CS_ROWS)); 8 warps stride rows.
 __global__ void __launch_bounds__(256) colsum_partial_kernel(const float* __restrict__ A, long long rows, int cols,
                                                              long long lda, float* __restrict__ scratch) {
   __shared__ float sh[8][33];
@@ -79,6 +79,41 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const float* __rest
 #pragma unroll
     for (int k = 0; k < 8; ++k) t += sh[k][lane];
     if (c < cols) scratch[(long long)blockIdx.y * cols + c] = t;
+  }
+}
+
+// 16-byte version: grid (ceil(cols/128), ceil(rows/CS_ROWS)); a warp covers 128 columns of a row,
+// 8 warps stride rows with four rows in flight per thread.
+__global__ void __launch_bounds__(256) colsum_partial_vec_kernel(const float* __restrict__ A, long long rows, int cols,
+                                                                 long long lda, float* __restrict__ scratch) {
+  __shared__ float4 sh[8][32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int c = (blockIdx.x * 32 + lane) * 4;
+  const long long r0 = (long long)blockIdx.y * CS_ROWS;
+  const long long r1 = min(rows, r0 + CS_ROWS);
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (c < cols) {
+    long long r = r0 + w;
+    for (; r + 24 < r1; r += 32) {
+      const float4 x0 = __ldg(reinterpret_cast<const float4*>(A + r * lda + c));
+      const float4 x1 = __ldg(reinterpret_cast<const float4*>(A + (r + 8) * lda + c));
+      const float4 x2 = __ldg(reinterpret_cast<const float4*>(A + (r + 16) * lda + c));
+      const float4 x3 = __ldg(reinterpret_cast<const float4*>(A + (r + 24) * lda + c));
+      s.x += (x0.x + x1.x) + (x2.x + x3.x); s.y += (x0.y + x1.y) + (x2.y + x3.y);
+      s.z += (x0.z + x1.z) + (x2.z + x3.z); s.w += (x0.w + x1.w) + (x2.w + x3.w);
+    }
+    for (; r < r1; r += 8) {
+      const float4 x = __ldg(reinterpret_cast<const float4*>(A + r * lda + c));
+      s.x += x.x; s.y += x.y; s.z += x.z; s.w += x.w;
+    }
+  }
+  sh[w][lane] = s;
+  __syncthreads();
+  if (w == 0 && c < cols) {
+    float4 t = sh[0][lane];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) { t.x += sh[k][lane].x; t.y += sh[k][lane].y; t.z += sh[k][lane].z; t.w += sh[k][lane].w; }
+    *reinterpret_cast<float4*>(scratch + (long long)blockIdx.y * cols + c) = t;
   }
 }
 
@@ -272,8 +307,15 @@ int64_t colsum_scratch_floats(int64_t rows, int cols) {
 int launch_colsum(const float* A, int64_t rows, int cols, int64_t lda, float alpha, const float* cin,
                   float beta, float* out, float* scratch, cudaStream_t st) {
   const int parts = (int)((rows + CS_ROWS - 1) / CS_ROWS);
-  dim3 grid((cols + 31) / 32, parts);
-  colsum_partial_kernel<<<grid, 256, 0, st>>>(A, rows, cols, lda, scratch);
+  const bool vec = (cols % 4 == 0) && (lda % 4 == 0) && ((reinterpret_cast<uintptr_t>(A) & 15) == 0) &&
+                   ((reinterpret_cast<uintptr_t>(scratch) & 15) == 0);
+  if (vec) {
+    dim3 grid((cols + 127) / 128, parts);
+    colsum_partial_vec_kernel<<<grid, 256, 0, st>>>(A, rows, cols, lda, scratch);
+  } else {
+    dim3 grid((cols + 31) / 32, parts);
+    colsum_partial_kernel<<<grid, 256, 0, st>>>(A, rows, cols, lda, scratch);
+  }
   colsum_final_kernel<<<(cols + 255) / 256, 256, 0, st>>>(scratch, parts, cols, alpha, cin, beta, out);
   return 2;
 }
