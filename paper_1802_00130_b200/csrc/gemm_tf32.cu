@@ -45,7 +45,7 @@ struct Tf32Params {
   float alpha;
   const float* cin; long long ld_cin; float beta;
   int vec_epi;          // D, bias, dsig, cin all 16-byte aligned with leading dimensions % 4 == 0
-  int bn;               // tile width: multiple of 32, 64 <= bn <= 256
+  int bn;               // tile width: multiple of 32, 32 <= bn <= 256
   int tiles_n, tiles;
   int* err;
 };
@@ -682,13 +682,14 @@ int choose_bn(int M, int N) {
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
   }
   if (N <= 64) best = 64;
+  if (N <= 32) best = 32;
   return best;
 }
 
 }  // namespace
 
 bool gemm_tf32_eligible(const GemmArgs& g) {
-  if (g.M < 1 || g.N < 32) return false;
+  if (g.M < 1 || g.N < 1) return false;
   if (!aligned16(g.A1) || !aligned16(g.B1) || g.lda1 % 4 || g.ldb1 % 4) return false;
   if (g.A2 && (!aligned16(g.A2) || !aligned16(g.B2) || g.lda2 % 4 || g.ldb2 % 4)) return false;
   if (!encode_fn()) return false;

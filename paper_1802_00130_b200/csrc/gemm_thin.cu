@@ -117,8 +117,9 @@ __global__ void __launch_bounds__(256, 2) gemm_thin_n_kernel(const ThinNParams p
 }
 
 // ------------------------------------------------------------------------------------ thin-M
-// grid (column tiles of 512, row chunks); thread = 4 consecutive columns; A rows staged in shared
-// memory 128 at a time; per-chunk partials go to scratch and are summed in chunk order.
+// grid (column tiles of 512, row chunks); a thread owns 4 consecutive columns and every other row of
+// the chunk; A rows staged in shared memory 128 at a time; per-chunk partials go to scratch and are
+// summed in chunk order.
 constexpr int TM_MAX = 16, TM_ROWS = 128;
 
 struct ThinMParams {
@@ -129,9 +130,13 @@ struct ThinMParams {
 };
 
 template <int MMAX>
-__global__ void __launch_bounds__(128) gemm_thin_m_partial_kernel(const ThinMParams p) {
+__global__ void __launch_bounds__(256) gemm_thin_m_partial_kernel(const ThinMParams p) {
+  // 256 threads = 2 row-halves x 128 column threads: half h takes rows h, h + 2, ... of the chunk, so
+  // that twice as many 16-byte loads of B are in flight; the halves are added at the end.
   __shared__ float As[TM_ROWS][MMAX];
-  const int n = (blockIdx.x * 128 + threadIdx.x) * 4;
+  __shared__ float4 Hs[MMAX][128];
+  const int ct = threadIdx.x & 127, half = threadIdx.x >> 7;
+  const int n = (blockIdx.x * 128 + ct) * 4;
   const long long r_begin = (long long)blockIdx.y * p.chunk_rows;
   const long long r_end = min(p.rows, r_begin + p.chunk_rows);
   float4 acc[MMAX];
@@ -140,14 +145,14 @@ __global__ void __launch_bounds__(128) gemm_thin_m_partial_kernel(const ThinMPar
   for (long long rb = r_begin; rb < r_end; rb += TM_ROWS) {
     const int cnt = (int)min((long long)TM_ROWS, r_end - rb);
     __syncthreads();
-    for (int i = threadIdx.x; i < cnt * MMAX; i += 128) {
+    for (int i = threadIdx.x; i < cnt * MMAX; i += 256) {
       const int r = i / MMAX, m = i % MMAX;
       As[r][m] = m < p.M ? __ldg(p.A + (rb + r) * p.lda + m) : 0.f;
     }
     __syncthreads();
     if (n < p.N) {
-#pragma unroll 4
-      for (int r = 0; r < cnt; ++r) {
+#pragma unroll 8
+      for (int r = half; r < cnt; r += 2) {
         const float4 b = __ldg(reinterpret_cast<const float4*>(p.B + (rb + r) * p.ldb + n));
 #pragma unroll
         for (int m = 0; m < MMAX; ++m) {
@@ -158,11 +163,19 @@ __global__ void __launch_bounds__(128) gemm_thin_m_partial_kernel(const ThinMPar
       }
     }
   }
-  if (n < p.N) {
+  if (half == 1) {
+#pragma unroll
+    for (int m = 0; m < MMAX; ++m) Hs[m][ct] = acc[m];
+  }
+  __syncthreads();
+  if (half == 0 && n < p.N) {
 #pragma unroll
     for (int m = 0; m < MMAX; ++m)
-      if (m < p.M)
-        *reinterpret_cast<float4*>(p.scratch + ((long long)blockIdx.y * p.M + m) * p.N + n) = acc[m];
+      if (m < p.M) {
+        const float4 o = Hs[m][ct];
+        *reinterpret_cast<float4*>(p.scratch + ((long long)blockIdx.y * p.M + m) * p.N + n) =
+            make_float4(acc[m].x + o.x, acc[m].y + o.y, acc[m].z + o.z, acc[m].w + o.w);
+      }
   }
 }
 
@@ -287,10 +300,10 @@ int launch_gemm_thin(const GemmArgs& g, float* scratch, cudaStream_t st) {
     const int used = (int)((g.K1 + p.chunk_rows - 1) / p.chunk_rows);
     p.A = g.A1; p.lda = g.lda1; p.B = g.B1; p.ldb = g.ldb1; p.scratch = scratch;
     dim3 grid((g.N + 511) / 512, used);
-    if (g.M <= 4) gemm_thin_m_partial_kernel<4><<<grid, 128, 0, st>>>(p);
-    else if (g.M <= 8) gemm_thin_m_partial_kernel<8><<<grid, 128, 0, st>>>(p);
-    else if (g.M <= 12) gemm_thin_m_partial_kernel<12><<<grid, 128, 0, st>>>(p);
-    else gemm_thin_m_partial_kernel<16><<<grid, 128, 0, st>>>(p);
+    if (g.M <= 4) gemm_thin_m_partial_kernel<4><<<grid, 256, 0, st>>>(p);
+    else if (g.M <= 8) gemm_thin_m_partial_kernel<8><<<grid, 256, 0, st>>>(p);
+    else if (g.M <= 12) gemm_thin_m_partial_kernel<12><<<grid, 256, 0, st>>>(p);
+    else gemm_thin_m_partial_kernel<16><<<grid, 256, 0, st>>>(p);
     const long long total = (long long)g.M * g.N;
     gemm_thin_m_final_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(scratch, used, g.M, g.N, make_epi(g));
     return 2;

@@ -165,7 +165,11 @@ void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
 // Kernel choice: streaming kernels for the n_L-wide shapes (both precisions: they are exact FP32),
 // the tensor-core kernel in TF32 mode when TMA can address the operands, else the FP32 FMA GEMM.
 void run_gemm(gn_ctx* c, const GemmArgs& g) {
-  if (gemm_thin_kind(g) != THIN_NONE) {
+  const ThinKind thin = gemm_thin_kind(g);
+  // In TF32 mode the n_L-wide forward products go to the tensor-core kernel as one 32- or 64-column
+  // tile: TMA streams A about 2.5x faster than the SIMT streaming kernel does (measured).
+  const bool thin_n_on_tensor = thin == THIN_N && c->prec == GN_TF32 && gemm_tf32_eligible(g);
+  if (thin != THIN_NONE && !thin_n_on_tensor) {
     const int64_t need = gemm_thin_scratch_floats(g);
     if (need > c->thin_cap) {
       cudaStreamSynchronize(c->st);

@@ -7,7 +7,7 @@ import gn_workloads as wl
 pytestmark = pytest.mark.gpu
 
 SHAPES = [(128, 256, 32), (128, 256, 64), (300, 520, 200), (1000, 300, 784), (37, 40, 12), (2500, 1000, 1000),
-          (260, 2000, 3000)]
+          (260, 2000, 3000), (3000, 10, 2000), (1000, 24, 520)]
 
 
 @pytest.fixture(scope="module")
