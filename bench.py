@@ -31,6 +31,10 @@ import gn_workloads as wl  # noqa: E402
 METRIC = "gauss_newton_matvecs_per_s"
 UNIT = "matvec/s"
 FP32_LANES_PER_SM, SMS = 128, 148
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant GEMM kernel, averaged over the
+# launches of one step (profiles/tf32_path_mnist2000_20_launches.md); unknown (None) for other cases
+TRAFFIC = {("tf32", "mnist2000_20"): {"bytes_per_launch": 318.5e6, "kernel": "gemm_tf32_2cta_kernel",
+                                      "source": "profiles/tf32_path_mnist2000_20_launches.md"}}
 
 
 def peaks():
@@ -295,7 +299,8 @@ def run_ours(args):
     kern = prof["tensor"] if args.mode == "tf32" else prof["ffma"]
     achieved = kern["flop"] / (kern["ms"] * 1e-3) / 1e12 if kern["ms"] > 0 else None
     roof.update({"kernel": "gemm_tf32_kernel" if args.mode == "tf32" else "gemm_ffma_kernel",
-                 "achieved": achieved, "frac": achieved / peak if achieved else None, "traffic": None,
+                 "achieved": achieved, "frac": achieved / peak if achieved else None,
+                 "traffic": TRAFFIC.get((args.mode, args.workload)),
                  "launches": kern["launches"], "avg_launch_us": 1e3 * kern["ms"] / max(1, kern["launches"]),
                  "share_of_step": kern["ms"] / ms if ms > 0 else None,
                  "other_gemm": {"kernel": "gemm_ffma_kernel" if args.mode == "tf32" else "gemm_tf32_kernel",
