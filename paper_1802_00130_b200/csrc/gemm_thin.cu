@@ -201,45 +201,71 @@ struct ThinKParams {
 };
 
 template <int KMAX>
-__global__ void __launch_bounds__(128) gemm_thin_k_kernel(const ThinKParams p) {
+__global__ void __launch_bounds__(128, 4) gemm_thin_k_kernel(const ThinKParams p) {
+  // Rows are taken 64 at a time: their A values are staged in shared memory, then groups of 8 rows
+  // first issue all their reads of the sigma' operand and only then compute and store, so
+  // that 8 independent 16-byte loads per thread are in flight (a store between two loads would
+  // otherwise pin their order, since D may alias the inputs as far as the compiler knows).
+  constexpr int RB = 64, RG = 8;
+  __shared__ float As[RB][KMAX];
   const int n = (blockIdx.x * 128 + threadIdx.x) * 4;
-  if (n >= p.N) return;
+  const bool n_ok = n < p.N;
   float4 b[KMAX];
 #pragma unroll
   for (int k = 0; k < KMAX; ++k)
-    b[k] = k < p.K ? __ldg(reinterpret_cast<const float4*>(p.B + (long long)k * p.ldb + n)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    b[k] = (n_ok && k < p.K) ? __ldg(reinterpret_cast<const float4*>(p.B + (long long)k * p.ldb + n)) : make_float4(0.f, 0.f, 0.f, 0.f);
   float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (p.e.bias) bz = __ldg(reinterpret_cast<const float4*>(p.e.bias + n));
+  if (p.e.bias && n_ok) bz = __ldg(reinterpret_cast<const float4*>(p.e.bias + n));
   const int m_begin = blockIdx.y * p.rows_per_block;
   const int m_end = min(p.M, m_begin + p.rows_per_block);
-#pragma unroll 4
-  for (int m = m_begin; m < m_end; ++m) {
-    float4 acc = bz;
+  for (int mb = m_begin; mb < m_end; mb += RB) {
+    const int cnt = min(RB, m_end - mb);
+    __syncthreads();
+    for (int i = threadIdx.x; i < cnt * KMAX; i += 128) {
+      const int r = i / KMAX, k = i % KMAX;
+      As[r][k] = k < p.K ? __ldg(p.A + (long long)(mb + r) * p.lda + k) : 0.f;
+    }
+    __syncthreads();
+    if (!n_ok) continue;
+    for (int r0 = 0; r0 < cnt; r0 += RG) {
+      float4 z[RG];
 #pragma unroll
-    for (int k = 0; k < KMAX; ++k) {
-      if (k < p.K) {
-        const float a = __ldg(p.A + (long long)m * p.lda + k);
-        acc.x = fmaf(a, b[k].x, acc.x); acc.y = fmaf(a, b[k].y, acc.y);
-        acc.z = fmaf(a, b[k].z, acc.z); acc.w = fmaf(a, b[k].w, acc.w);
+      for (int i = 0; i < RG; ++i) {
+        const int m = mb + r0 + i;
+        const bool ok = r0 + i < cnt;
+        z[i] = (p.e.dsig && ok) ? __ldg(reinterpret_cast<const float4*>(p.e.dsig + (long long)(m % p.e.dsig_rows) * p.e.ld_dsig + n))
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int i = 0; i < RG; ++i) {
+        if (r0 + i >= cnt) break;
+        const int m = mb + r0 + i;
+        float4 acc = bz;
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+          const float a = As[r0 + i][k];
+          acc.x = fmaf(a, b[k].x, acc.x); acc.y = fmaf(a, b[k].y, acc.y);
+          acc.z = fmaf(a, b[k].z, acc.z); acc.w = fmaf(a, b[k].w, acc.w);
+        }
+        float t[4] = {acc.x, acc.y, acc.z, acc.w};
+        if (p.e.sigmoid) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) t[j] = 1.f / (1.f + expf(-t[j]));
+        }
+        if (p.e.dsig) {
+          t[0] *= z[i].x * (1.f - z[i].x); t[1] *= z[i].y * (1.f - z[i].y);
+          t[2] *= z[i].z * (1.f - z[i].z); t[3] *= z[i].w * (1.f - z[i].w);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) t[j] *= p.e.alpha;
+        if (p.e.cin) {   // not on the path's hot use of this kernel: read in place
+          const float4 c = __ldg(reinterpret_cast<const float4*>(p.e.cin + (long long)m * p.e.ld_cin + n));
+          t[0] = fmaf(p.e.beta, c.x, t[0]); t[1] = fmaf(p.e.beta, c.y, t[1]);
+          t[2] = fmaf(p.e.beta, c.z, t[2]); t[3] = fmaf(p.e.beta, c.w, t[3]);
+        }
+        *reinterpret_cast<float4*>(p.e.D + (long long)m * p.e.ldd + n) = make_float4(t[0], t[1], t[2], t[3]);
       }
     }
-    float t[4] = {acc.x, acc.y, acc.z, acc.w};
-    if (p.e.sigmoid) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) t[j] = 1.f / (1.f + expf(-t[j]));
-    }
-    if (p.e.dsig) {
-      const float4 z = __ldg(reinterpret_cast<const float4*>(p.e.dsig + (long long)(m % p.e.dsig_rows) * p.e.ld_dsig + n));
-      t[0] *= z.x * (1.f - z.x); t[1] *= z.y * (1.f - z.y); t[2] *= z.z * (1.f - z.z); t[3] *= z.w * (1.f - z.w);
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) t[j] *= p.e.alpha;
-    if (p.e.cin) {
-      const float4 c = __ldg(reinterpret_cast<const float4*>(p.e.cin + (long long)m * p.e.ld_cin + n));
-      t[0] = fmaf(p.e.beta, c.x, t[0]); t[1] = fmaf(p.e.beta, c.y, t[1]);
-      t[2] = fmaf(p.e.beta, c.z, t[2]); t[3] = fmaf(p.e.beta, c.w, t[3]);
-    }
-    *reinterpret_cast<float4*>(p.e.D + (long long)m * p.e.ldd + n) = make_float4(t[0], t[1], t[2], t[3]);
   }
 }
 
