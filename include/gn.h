@@ -194,7 +194,8 @@ gn_status gn_profile_read(gn_ctx* ctx, double* gemm_ms, double* gemm_flop, int64
  * with the kernel of the given kind (0 = tensor-core TF32, 1 = FP32 FMA GEMM, 2 = streaming kernel for
  * a dimension <= 16, 3 = tensor-core TF32 with the promise that every [K][M] / [K][N] operand is
  * followed by at least 128 readable bytes, which lets it fetch them with one TMA box per stage;
- * 4 and 5 = as 3 with one CTA per 128-row tile, respectively a CTA pair per 256-row tile, forced).  a_kmajor: A is [M][K]
+ * 4 and 5 = as 3 with one CTA per 128-row tile, respectively a CTA pair per 256-row tile, forced;
+ * 6 = as 5 but whole tiles only, i.e. without the stream-K split of tiles between CTA pairs).  a_kmajor: A is [M][K]
  * (else [K][M]); b_kmajor: B is [N][K] (else [K][N]); all row-major with the given leading
  * dimensions.  GN_EINVAL if the chosen kernel cannot take the operands (alignment, shape).
  */

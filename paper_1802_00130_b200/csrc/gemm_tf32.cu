@@ -48,6 +48,12 @@ struct Tf32Params {
   int bn;               // tile width: multiple of 32, 32 <= bn <= 256
   int tiles_n, tiles;
   int* err;
+  // stream-K (two-CTA kernel): the tiles' k-blocks, flattened tile-major, are cut into sk_pairs equal
+  // ranges, one per CTA pair.  sk_split != 0 allows a range to start or end inside a tile.
+  int sk_pairs, sk_split;
+  int sk_W, sk_r;        // wave-major order of the flattened tiles (sk_W == 0: raster order), see sk_tile()
+  float* sk_ws;          // [sk_pairs][2][128][256] raw partial accumulators of split tiles
+  int* sk_flags;         // [sk_pairs + 1] arrival counters of those partials, zeroed before the launch
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -359,6 +365,13 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant
 // only the leader (rank 0) arms full[s] with the bytes of both CTAs, and both CTAs' TMA loads complete
 // on the leader's full[s].  MMAs are issued by the leader only.  acc_full[b] is multicast to both
 // CTAs; all 16 epilogue warps of the pair arrive on the leader's acc_empty[b].
+//
+// Work split: the k-blocks of all tiles, flattened in wave order, are divided over the CTA pairs in
+// contiguous ranges (tile-aligned unless the host allows splitting, which it does for under-filled
+// problems: two pairs per tile).  A pair's range may begin inside a tile (it then computes that tile's last k-blocks first in time, stores the raw
+// accumulator in a workspace slot and raises the slot's counter) and may end inside a tile (it
+// computes that tile's first k-blocks last in time, waits - bounded - for the next pair's slot, adds
+// it and runs the epilogue).  The sum order is fixed, so results are deterministic.
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -405,6 +418,19 @@ __device__ __forceinline__ void mma2_commit_both(uint64_t* bar) {
                ::"r"(smem_u32(bar)), "h"(mask) : "memory");
 }
 
+// Order in which the flattened work visits the tiles.  With T tiles on P pairs the tiles form W = ceil(T/P)
+// waves of P (the last holds r = T - (W-1) P); position L of the flattened order walks that grid column
+// by column (pair column first, wave index second) and lands on raster tile i * P + column.  A pair's
+// even share of the flattened work is then (about) one column, i.e. one tile of every wave, so that at
+// any moment all pairs work inside one or two waves of neighbouring tiles, which share A panels in L2.
+__device__ __forceinline__ int sk_tile(int L, int P, int W, int r) {
+  if (W == 0) return L;
+  int col, i;
+  if (L < r * W) { col = L / W; i = L - col * W; }
+  else { const int L2 = L - r * W; col = r + L2 / (W - 1); i = L2 - (col - r) * (W - 1); }
+  return i * P + col;
+}
+
 constexpr int B2_STAGE_MAX = (BN_MAX / 2) * BK * 4;          // 16 KB: this CTA's half of the B tile
 constexpr int STAGE2_BYTES = A_STAGE_BYTES + B2_STAGE_MAX;   // 32 KB
 
@@ -428,6 +454,23 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
   const int total_kb = p.kblocks[0] + p.kblocks[1];
   const int bn = p.bn, hb = p.bn >> 1;                       // hb: B rows staged by each CTA
   const uint32_t pair_tx = 2u * (A_STAGE_BYTES + (uint32_t)hb * BK * 4);
+  // this pair's range of k-block units [u_begin, u_end)
+  long long u_begin, u_end;
+  if (p.sk_split) {
+    const long long U = (long long)p.tiles * total_kb;
+    u_begin = U * pair / p.sk_pairs;
+    u_end = U * (pair + 1) / p.sk_pairs;
+  } else if (p.sk_W > 0) {
+    // whole tiles, one column of the wave grid per pair: pair p runs raster tiles p, p + P, p + 2P, ...
+    const int c0 = pair < p.sk_r ? pair * p.sk_W : p.sk_r * p.sk_W + (pair - p.sk_r) * (p.sk_W - 1);
+    const int c1 = pair + 1 <= p.sk_r ? (pair + 1) * p.sk_W : p.sk_r * p.sk_W + (pair + 1 - p.sk_r) * (p.sk_W - 1);
+    u_begin = (long long)c0 * total_kb;
+    u_end = (long long)c1 * total_kb;
+  } else {
+    u_begin = ((long long)p.tiles * pair / p.sk_pairs) * total_kb;
+    u_end = ((long long)p.tiles * (pair + 1) / p.sk_pairs) * total_kb;
+  }
+  (void)n_pairs;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -448,10 +491,15 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
     // ------------------------------------------------------------------ producer (both CTAs)
     int it = 0;
     bool ok = true;
-    for (int t = pair; t < p.tiles && ok; t += n_pairs) {
+    for (long long u = u_begin; u < u_end && ok;) {
+      const int tl = (int)(u / total_kb);                      // position in the flattened order
+      const int kb0 = (int)(u - (long long)tl * total_kb);
+      const int t = sk_tile(tl, p.sk_pairs, p.sk_W, p.sk_r);
+      const int kb1 = (int)min((long long)total_kb, kb0 + (u_end - u));
+      u += kb1 - kb0;
       const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM;
       const int n0 = (t % p.tiles_n) * bn + (int)rank * hb;
-      for (int kb = 0; kb < total_kb; ++kb, ++it) {
+      for (int kb = kb0; kb < kb1; ++kb, ++it) {
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1;
         int good = 1;
@@ -495,14 +543,18 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
       const uint32_t a_lay = p.a_mn ? 1 : 2, b_lay = p.b_mn ? 1 : 2;
       int it = 0, ti = 0;
       bool ok = true;
-      for (int t = pair; t < p.tiles && ok; t += n_pairs, ++ti) {
+      for (long long u = u_begin; u < u_end && ok; ++ti) {
+        const int tl = (int)(u / total_kb);
+        const int kb0 = (int)(u - (long long)tl * total_kb);
+        const int kb1 = (int)min((long long)total_kb, kb0 + (u_end - u));
+        u += kb1 - kb0;
         const int buf = ti & 1;
         const uint32_t aph = (ti >> 1) & 1;
         ok = wait_or_abort(&acc_empty[buf], aph ^ 1, abort_flag, p.err, 4);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN_MAX);
-        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           ok = wait_or_abort(&full[s], ph, abort_flag, p.err, 2);
@@ -514,7 +566,7 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
           for (int k = 0; k < BK / 8; ++k) {
             const uint64_t ad = make_desc(sa + k * a_step, a_lbo, a_sbo, a_lay);
             const uint64_t bd = make_desc(sb + k * b_step, b_lbo, b_sbo, b_lay);
-            mma2_tf32(tmem_d, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+            mma2_tf32(tmem_d, ad, bd, idesc, (kb > kb0 || k != 0) ? 1u : 0u);
           }
           mma2_commit_both(&empty[s]);
         }
@@ -525,8 +577,16 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
     // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
     const int quad = warp & 3;
     const int half = (warp - 2) >> 2;
+    const int row = quad * 32 + lane;                          // row of this CTA's 128-row block
     int ti = 0;
-    for (int t = pair; t < p.tiles; t += n_pairs, ++ti) {
+    for (long long u = u_begin; u < u_end; ++ti) {
+      const int tl = (int)(u / total_kb);                      // position in the flattened order
+      const int kb0 = (int)(u - (long long)tl * total_kb);
+      const int t = sk_tile(tl, p.sk_pairs, p.sk_W, p.sk_r);
+      const int kb1 = (int)min((long long)total_kb, kb0 + (u_end - u));
+      u += kb1 - kb0;
+      const bool is_tail = kb0 > 0;                            // partial: last k-blocks of a tile another pair begins
+      const bool is_head = kb0 == 0 && kb1 < total_kb;         // partial: first k-blocks; pair + 1 holds the rest
       const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM, n0 = (t % p.tiles_n) * bn;
       const int buf = ti & 1;
       const uint32_t aph = (ti >> 1) & 1;
@@ -535,54 +595,93 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
       good = __shfl_sync(0xffffffffu, good, 0);
       if (!good) break;
       tc_fence_after();
-      const int m = m0 + quad * 32 + lane;
-      const bool m_ok = m < p.M;
-      const float* zrow = p.dsig ? p.dsig + (long long)(m % p.dsig_rows) * p.ld_dsig : nullptr;
-      const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
-      float* drow = p.D + (long long)m * p.ldd;
-      for (int c = half; c < bn / 32; c += 2) {
-        const int nb = n0 + c * 32;
-        if (nb >= p.N) break;
-        const bool fullc = p.vec_epi && nb + 32 <= p.N;
-        float4 zc[8], ci[8];
-        if (fullc && m_ok) {
+      if (is_tail) {
+        // raw accumulator to this pair's workspace slot, then count this warp in
+        float* ws = p.sk_ws + (((long long)pair * 2 + rank) * BM + row) * BN_MAX;
+        for (int c = half; c < bn / 32; c += 2) {
+          if (n0 + c * 32 >= p.N) break;
+          float v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            zc[q] = zrow ? __ldg(reinterpret_cast<const float4*>(zrow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-            ci[q] = crow ? __ldg(reinterpret_cast<const float4*>(crow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-          }
+          for (int q = 0; q < 8; ++q)
+            __stcg(reinterpret_cast<float4*>(ws + c * 32) + q, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
         }
-        float v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
-        if (!m_ok) continue;
-        if (fullc) {
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (p.bias) bz = __ldg(reinterpret_cast<const float4*>(p.bias + nb) + q);
-            float x[4] = {v[4 * q] + bz.x, v[4 * q + 1] + bz.y, v[4 * q + 2] + bz.z, v[4 * q + 3] + bz.w};
-            const float z[4] = {zc[q].x, zc[q].y, zc[q].z, zc[q].w};
-            const float cc[4] = {ci[q].x, ci[q].y, ci[q].z, ci[q].w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              if (p.sigmoid) x[j] = 1.f / (1.f + __expf(-x[j]));
-              if (zrow) x[j] *= z[j] * (1.f - z[j]);
-              x[j] *= p.alpha;
-              if (crow) x[j] = fmaf(p.beta, cc[j], x[j]);
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(p.sk_flags + pair, 1);
+      } else {
+        const float* ws = nullptr;
+        if (is_head) {
+          // the rest of this tile was computed (earlier in time) by pair + 1: wait for its 16 warps
+          ws = p.sk_ws + (((long long)(pair + 1) * 2 + rank) * BM + row) * BN_MAX;
+          if (lane == 0) {
+            const volatile int* flag = p.sk_flags + pair + 1;
+            const unsigned long long t0 = globaltimer();
+            while (*flag < 16) {
+              if (*abort_flag || globaltimer() - t0 > WAIT_LIMIT_NS) { atomicCAS(p.err, 0, 5); *abort_flag = 1; good = 0; break; }
             }
-            reinterpret_cast<float4*>(drow + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
+            __threadfence();
           }
-        } else {
+          good = __shfl_sync(0xffffffffu, good, 0);
+          if (!good) break;
+        }
+        const int m = m0 + row;
+        const bool m_ok = m < p.M;
+        const float* zrow = p.dsig ? p.dsig + (long long)(m % p.dsig_rows) * p.ld_dsig : nullptr;
+        const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
+        float* drow = p.D + (long long)m * p.ldd;
+        for (int c = half; c < bn / 32; c += 2) {
+          const int nb = n0 + c * 32;
+          if (nb >= p.N) break;
+          const bool fullc = p.vec_epi && nb + 32 <= p.N;
+          float4 zc[8], ci[8], pw[8];
+          if (fullc && m_ok) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int n = nb + j;
-            if (n < p.N) {
-              float x = v[j] + (p.bias ? __ldg(p.bias + n) : 0.f);
-              if (p.sigmoid) x = 1.f / (1.f + __expf(-x));
-              if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
-              x *= p.alpha;
-              if (crow) x = fmaf(p.beta, __ldg(crow + n), x);
-              drow[n] = x;
+            for (int q = 0; q < 8; ++q) {
+              zc[q] = zrow ? __ldg(reinterpret_cast<const float4*>(zrow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+              ci[q] = crow ? __ldg(reinterpret_cast<const float4*>(crow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+          }
+          if (ws) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) pw[q] = __ldcg(reinterpret_cast<const float4*>(ws + c * 32) + q);
+          }
+          float v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
+          if (ws) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { v[4 * q] += pw[q].x; v[4 * q + 1] += pw[q].y; v[4 * q + 2] += pw[q].z; v[4 * q + 3] += pw[q].w; }
+          }
+          if (!m_ok) continue;
+          if (fullc) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (p.bias) bz = __ldg(reinterpret_cast<const float4*>(p.bias + nb) + q);
+              float x[4] = {v[4 * q] + bz.x, v[4 * q + 1] + bz.y, v[4 * q + 2] + bz.z, v[4 * q + 3] + bz.w};
+              const float z[4] = {zc[q].x, zc[q].y, zc[q].z, zc[q].w};
+              const float cc[4] = {ci[q].x, ci[q].y, ci[q].z, ci[q].w};
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                if (p.sigmoid) x[j] = 1.f / (1.f + __expf(-x[j]));
+                if (zrow) x[j] *= z[j] * (1.f - z[j]);
+                x[j] *= p.alpha;
+                if (crow) x[j] = fmaf(p.beta, cc[j], x[j]);
+              }
+              reinterpret_cast<float4*>(drow + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int n = nb + j;
+              if (n < p.N) {
+                float x = v[j] + (p.bias ? __ldg(p.bias + n) : 0.f);
+                if (p.sigmoid) x = 1.f / (1.f + __expf(-x));
+                if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
+                x *= p.alpha;
+                if (crow) x = fmaf(p.beta, __ldg(crow + n), x);
+                drow[n] = x;
+              }
             }
           }
         }
@@ -699,21 +798,27 @@ bool gemm_tf32_eligible(const GemmArgs& g) {
 constexpr int kStages2 = 6;
 constexpr int kSmemBytes2 = kStages2 * STAGE2_BYTES + 1024 + 256;
 
-// Two-CTA tile width (a multiple of 64 so that each CTA's half is whole 32-column chunks).
-int choose_bn2(int M, int N) {
+// Two-CTA tile width (a multiple of 64 so that each CTA's half is whole 32-column chunks).  With the
+// work split evenly over the pairs (stream-K) only the padding of N to whole tiles costs anything;
+// without it the number of waves decides as well.
+int choose_bn2(int M, int N, bool stream_k) {
   const long long tiles_m = (M + 2 * BM - 1) / (2 * BM);
   const int pairs = num_sms() / 2;
   int best = 256;
   long long best_cost = -1;
   for (int bn = 256; bn >= 128; bn -= 64) {
-    const long long tiles = tiles_m * ((N + bn - 1) / bn);
-    const long long cost = ((tiles + pairs - 1) / pairs) * (320 + bn);
+    const long long tiles_n = (N + bn - 1) / bn;
+    const long long tiles = tiles_m * tiles_n;
+    const long long cost = (stream_k ? tiles_n : (tiles + pairs - 1) / pairs) * (320 + bn);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
   }
   return best;
 }
 
-int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
+int64_t gemm_tf32_workspace_floats() { return (int64_t)(num_sms() / 2) * 2 * BM * BN_MAX; }
+int gemm_tf32_workspace_flags() { return num_sms() / 2 + 1; }
+
+int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaFuncSetAttribute(gemm_tf32_kernel<kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -725,7 +830,8 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
     attr2_set = true;
   }
   const bool two_cta = g.two_cta >= 0 ? g.two_cta != 0 : (g.M > BM && g.N >= 128);
-  const int bn = two_cta ? choose_bn2(g.M, g.N) : choose_bn(g.M, g.N);
+  const bool stream_k = two_cta && sk_ws && sk_flags;
+  const int bn = two_cta ? choose_bn2(g.M, g.N, stream_k) : choose_bn(g.M, g.N);
   const int b_rows = two_cta ? bn / 2 : bn;      // B rows staged per CTA
   CUtensorMap maps[4];
   const float* As[2] = {g.A1, g.A2};
@@ -764,8 +870,25 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   if (two_cta) {
     p.tiles = ((g.M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;   // tiles of 256 rows, one per CTA pair
     const int pairs = num_sms() / 2;
-    const int grid = 2 * (p.tiles < pairs ? p.tiles : pairs);
-    gemm_tf32_2cta_kernel<kStages2><<<grid, 320, kSmemBytes2, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+    // active pairs: all of them when there is at least a tile each; two per tile (each tile cut once in
+    // the middle) when that still fits; else one per tile.  A range never holds less than half a tile,
+    // so no tile is cut more than once per pair boundary.
+    p.sk_ws = sk_ws; p.sk_flags = sk_flags;
+    p.sk_split = 0;
+    p.sk_pairs = p.tiles < pairs ? p.tiles : pairs;
+    if (p.tiles >= pairs) {
+      p.sk_W = (p.tiles + pairs - 1) / pairs;
+      p.sk_r = p.tiles - (p.sk_W - 1) * pairs;
+    }
+    if (stream_k) {
+      const int total_kb = p.kblocks[0] + p.kblocks[1];
+      // Splitting is used only for under-filled problems (each tile cut once in the middle, two pairs per
+      // tile).  With more tiles than pairs an even split was measured to lose: the pairs drift apart
+      // over the waves, tiles of one A panel are then processed at different times and miss in L2.
+      if (2 * p.tiles <= pairs && total_kb >= 2) { p.sk_pairs = 2 * p.tiles; p.sk_split = 1; }
+      if (p.sk_split) cudaMemsetAsync(sk_flags, 0, sizeof(int) * (pairs + 1), st);
+    }
+    gemm_tf32_2cta_kernel<kStages2><<<2 * p.sk_pairs, 320, kSmemBytes2, st>>>(maps[0], maps[1], maps[2], maps[3], p);
   } else {
     p.tiles = ((g.M + BM - 1) / BM) * p.tiles_n;
     const int grid = p.tiles < num_sms() ? p.tiles : num_sms();

@@ -39,6 +39,8 @@ struct gn_ctx {
   // reductions
   float* colsum_scratch = nullptr; int64_t colsum_cap = 0;
   float* thin_scratch = nullptr; int64_t thin_cap = 0;
+  float* sk_ws = nullptr; int* sk_flags = nullptr;   // stream-K workspace of the tensor-core kernel
+  bool sk_enabled = true;
   double* partial = nullptr; int64_t partial_cap = 0;
   double* dscal = nullptr;   // device: [0] loss, [1] theta^T theta, [2] cg sum rho, [3] cg active
   double* hscal = nullptr;   // pinned mirror
@@ -151,7 +153,16 @@ void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
     }
   }
   if (kind == 0) {
-    const int r = launch_gemm_tf32(g, c->err_flag + 1, c->st);
+    if (!c->sk_ws && c->sk_enabled) {   // first tensor-core launch of this context: stream-K workspace
+      if (dev_alloc(c, &c->sk_ws, gemm_tf32_workspace_floats()) != GN_OK ||
+          dev_alloc(c, &c->sk_flags, (int64_t)gemm_tf32_workspace_flags()) != GN_OK) {
+        c->sk_ws = nullptr; c->sk_flags = nullptr; c->sk_enabled = false;
+      }
+    }
+    const bool sk = c->sk_enabled && g.two_cta != 2;
+    GemmArgs g2 = g;
+    if (g2.two_cta == 2) g2.two_cta = 1;
+    const int r = launch_gemm_tf32(g2, c->err_flag + 1, sk ? c->sk_ws : nullptr, sk ? c->sk_flags : nullptr, c->st);
     if (r < 0) { c->sticky = GN_ECUDA; c->err = "cuTensorMapEncodeTiled failed"; }
     else c->launches += r;
   } else if (kind == 2) {
@@ -708,17 +719,19 @@ gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t
 gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* dA, int64_t lda, int a_kmajor,
                         const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd) {
   if (!c) return GN_EINVAL;
-  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 5) return fail(c, GN_EINVAL, "bad GEMM arguments");
+  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 6) return fail(c, GN_EINVAL, "bad GEMM arguments");
   GemmArgs g;
   g.M = M; g.N = N; g.K1 = K;
   g.A1 = dA; g.lda1 = lda; g.a_kmajor = a_kmajor != 0;
   g.B1 = dB; g.ldb1 = ldb; g.b_kmajor = b_kmajor != 0;
   g.D = dD; g.ldd = ldd;
-  // kinds 3..5 are the tensor-core kernel with options: 3 = MN-major operands declared padded,
-  // 4 = one CTA per tile forced, 5 = CTA pair per tile forced (both with padded operands)
+  // kinds 3..6 are the tensor-core kernel with options: 3 = MN-major operands declared padded,
+  // 4 = one CTA per tile forced, 5 = CTA pair per tile forced, 6 = as 5 without splitting tiles
+  // between pairs (all with padded operands)
   g.mn_padded = (kind >= 3);
   if (kind == 4) g.two_cta = 0;
   if (kind == 5) g.two_cta = 1;
+  if (kind == 6) g.two_cta = 2;   // CTA pair per tile, whole tiles only (no stream-K split)
   if (kind >= 3) kind = 0;
   if (kind == 0 && !gemm_tf32_eligible(g)) return fail(c, GN_EINVAL, "operands do not qualify for the tensor-core kernel");
   if (kind == 2) {

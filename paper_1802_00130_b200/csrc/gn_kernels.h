@@ -40,8 +40,13 @@ int launch_gemm_ffma(const GemmArgs& g, cudaStream_t st);
 // that are multiples of 4 floats (TMA strides); gemm_tf32_eligible says whether a problem qualifies.
 // *err_flag receives a non-zero code if a bounded device-side wait ran out.  Returns launches made,
 // or -1 if a tensor map could not be encoded.
+// sk_ws / sk_flags: optional workspace of gemm_tf32_workspace_floats() floats and
+// gemm_tf32_workspace_flags() ints that lets the two-CTA kernel split tiles between CTA pairs
+// (stream-K); pass nullptr to keep whole tiles.
 bool gemm_tf32_eligible(const GemmArgs& g);
-int launch_gemm_tf32(const GemmArgs& g, int* err_flag, cudaStream_t st);
+int64_t gemm_tf32_workspace_floats();
+int gemm_tf32_workspace_flags();
+int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st);
 
 // Streaming FP32 kernels for contractions with one dimension <= 16 (the n_L-wide output layer).
 // gemm_thin_kind says which of them (if any) takes a problem; THIN_M needs a scratch buffer of
