@@ -48,12 +48,11 @@ struct Tf32Params {
   int bn;               // tile width: multiple of 32, 32 <= bn <= 256
   int tiles_n, tiles;
   int* err;
-  // stream-K (two-CTA kernel): the tiles' k-blocks, flattened tile-major, are cut into sk_pairs equal
-  // ranges, one per CTA pair.  sk_split != 0 allows a range to start or end inside a tile.
-  int sk_pairs, sk_split;
-  int sk_W, sk_r;        // wave-major order of the flattened tiles (sk_W == 0: raster order), see sk_tile()
-  float* sk_ws;          // [sk_pairs][2][128][256] raw partial accumulators of split tiles
-  int* sk_flags;         // [sk_pairs + 1] arrival counters of those partials, zeroed before the launch
+  // work list of the two-CTA kernel: pair q runs tiles q, q + P, ... for `waves` full waves of P tiles;
+  // the `rem` tiles left over are each cut along K into `slices` parts, one per pair (slices == 1: whole)
+  int P, waves, rem, slices;
+  float* sk_ws;          // [P][2][128][256] raw partial accumulators of the sliced tiles, slot = pair
+  int* sk_flags;         // [P] arrival counters, one per sliced tile, zeroed before the launch
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -366,12 +365,13 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant
 // on the leader's full[s].  MMAs are issued by the leader only.  acc_full[b] is multicast to both
 // CTAs; all 16 epilogue warps of the pair arrive on the leader's acc_empty[b].
 //
-// Work split: the k-blocks of all tiles, flattened in wave order, are divided over the CTA pairs in
-// contiguous ranges (tile-aligned unless the host allows splitting, which it does for under-filled
-// problems: two pairs per tile).  A pair's range may begin inside a tile (it then computes that tile's last k-blocks first in time, stores the raw
-// accumulator in a workspace slot and raises the slot's counter) and may end inside a tile (it
-// computes that tile's first k-blocks last in time, waits - bounded - for the next pair's slot, adds
-// it and runs the epilogue).  The sum order is fixed, so results are deterministic.
+// Work list: with T tiles on P pairs, pair q runs tiles q, q + P, ... for the floor(T / P) full waves, so
+// that all pairs move through neighbouring tiles together (tiles of one A panel are read at the same
+// time and hit in L2).  The T mod P tiles of the last, partial wave are each cut along K into up to 8
+// slices, one per otherwise idle pair.  The pairs of a sliced tile store their raw accumulators in a
+// workspace, count themselves in on the tile's flag, wait (bounded) until all slices have arrived, and
+// then each sums one share of the tile's column chunks over all slices, in slice order, and runs the
+// epilogue on it.  The order of every sum is fixed, so results are deterministic.
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -418,17 +418,24 @@ __device__ __forceinline__ void mma2_commit_both(uint64_t* bar) {
                ::"r"(smem_u32(bar)), "h"(mask) : "memory");
 }
 
-// Order in which the flattened work visits the tiles.  With T tiles on P pairs the tiles form W = ceil(T/P)
-// waves of P (the last holds r = T - (W-1) P); position L of the flattened order walks that grid column
-// by column (pair column first, wave index second) and lands on raster tile i * P + column.  A pair's
-// even share of the flattened work is then (about) one column, i.e. one tile of every wave, so that at
-// any moment all pairs work inside one or two waves of neighbouring tiles, which share A panels in L2.
-__device__ __forceinline__ int sk_tile(int L, int P, int W, int r) {
-  if (W == 0) return L;
-  int col, i;
-  if (L < r * W) { col = L / W; i = L - col * W; }
-  else { const int L2 = L - r * W; col = r + L2 / (W - 1); i = L2 - (col - r) * (W - 1); }
-  return i * P + col;
+struct Work { int tile, kb0, kb1, sliced; };
+
+// idx-th piece of work of CTA pair `pair` (see Tf32Params); false when the pair has no more.
+__device__ __forceinline__ bool next_work(const Tf32Params& p, int pair, int total_kb, int idx, Work& w) {
+  if (idx < p.waves) { w.tile = idx * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0; return true; }
+  if (idx > p.waves || p.rem == 0) return false;
+  if (p.slices < 2) {
+    if (pair >= p.rem) return false;
+    w.tile = p.waves * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0;
+    return true;
+  }
+  if (pair >= p.rem * p.slices) return false;
+  const int j = pair / p.slices, sl = pair - j * p.slices;
+  w.tile = p.waves * p.P + j;
+  w.kb0 = (int)((long long)total_kb * sl / p.slices);
+  w.kb1 = (int)((long long)total_kb * (sl + 1) / p.slices);
+  w.sliced = 1;
+  return true;
 }
 
 constexpr int B2_STAGE_MAX = (BN_MAX / 2) * BK * 4;          // 16 KB: this CTA's half of the B tile
@@ -454,22 +461,6 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
   const int total_kb = p.kblocks[0] + p.kblocks[1];
   const int bn = p.bn, hb = p.bn >> 1;                       // hb: B rows staged by each CTA
   const uint32_t pair_tx = 2u * (A_STAGE_BYTES + (uint32_t)hb * BK * 4);
-  // this pair's range of k-block units [u_begin, u_end)
-  long long u_begin, u_end;
-  if (p.sk_split) {
-    const long long U = (long long)p.tiles * total_kb;
-    u_begin = U * pair / p.sk_pairs;
-    u_end = U * (pair + 1) / p.sk_pairs;
-  } else if (p.sk_W > 0) {
-    // whole tiles, one column of the wave grid per pair: pair p runs raster tiles p, p + P, p + 2P, ...
-    const int c0 = pair < p.sk_r ? pair * p.sk_W : p.sk_r * p.sk_W + (pair - p.sk_r) * (p.sk_W - 1);
-    const int c1 = pair + 1 <= p.sk_r ? (pair + 1) * p.sk_W : p.sk_r * p.sk_W + (pair + 1 - p.sk_r) * (p.sk_W - 1);
-    u_begin = (long long)c0 * total_kb;
-    u_end = (long long)c1 * total_kb;
-  } else {
-    u_begin = ((long long)p.tiles * pair / p.sk_pairs) * total_kb;
-    u_end = ((long long)p.tiles * (pair + 1) / p.sk_pairs) * total_kb;
-  }
   (void)n_pairs;
 
   if (threadIdx.x == 0) {
@@ -491,12 +482,9 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
     // ------------------------------------------------------------------ producer (both CTAs)
     int it = 0;
     bool ok = true;
-    for (long long u = u_begin; u < u_end && ok;) {
-      const int tl = (int)(u / total_kb);                      // position in the flattened order
-      const int kb0 = (int)(u - (long long)tl * total_kb);
-      const int t = sk_tile(tl, p.sk_pairs, p.sk_W, p.sk_r);
-      const int kb1 = (int)min((long long)total_kb, kb0 + (u_end - u));
-      u += kb1 - kb0;
+    Work w;
+    for (int wi = 0; ok && next_work(p, pair, total_kb, wi, w); ++wi) {
+      const int t = w.tile, kb0 = w.kb0, kb1 = w.kb1;
       const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM;
       const int n0 = (t % p.tiles_n) * bn + (int)rank * hb;
       for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -543,11 +531,9 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
       const uint32_t a_lay = p.a_mn ? 1 : 2, b_lay = p.b_mn ? 1 : 2;
       int it = 0, ti = 0;
       bool ok = true;
-      for (long long u = u_begin; u < u_end && ok; ++ti) {
-        const int tl = (int)(u / total_kb);
-        const int kb0 = (int)(u - (long long)tl * total_kb);
-        const int kb1 = (int)min((long long)total_kb, kb0 + (u_end - u));
-        u += kb1 - kb0;
+      Work w;
+      for (int wi = 0; ok && next_work(p, pair, total_kb, wi, w); ++wi, ++ti) {
+        const int kb0 = w.kb0, kb1 = w.kb1;
         const int buf = ti & 1;
         const uint32_t aph = (ti >> 1) & 1;
         ok = wait_or_abort(&acc_empty[buf], aph ^ 1, abort_flag, p.err, 4);
@@ -579,14 +565,9 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
     const int half = (warp - 2) >> 2;
     const int row = quad * 32 + lane;                          // row of this CTA's 128-row block
     int ti = 0;
-    for (long long u = u_begin; u < u_end; ++ti) {
-      const int tl = (int)(u / total_kb);                      // position in the flattened order
-      const int kb0 = (int)(u - (long long)tl * total_kb);
-      const int t = sk_tile(tl, p.sk_pairs, p.sk_W, p.sk_r);
-      const int kb1 = (int)min((long long)total_kb, kb0 + (u_end - u));
-      u += kb1 - kb0;
-      const bool is_tail = kb0 > 0;                            // partial: last k-blocks of a tile another pair begins
-      const bool is_head = kb0 == 0 && kb1 < total_kb;         // partial: first k-blocks; pair + 1 holds the rest
+    Work w;
+    for (int wi = 0; next_work(p, pair, total_kb, wi, w); ++wi, ++ti) {
+      const int t = w.tile;
       const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM, n0 = (t % p.tiles_n) * bn;
       const int buf = ti & 1;
       const uint32_t aph = (ti >> 1) & 1;
@@ -595,46 +576,53 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
       good = __shfl_sync(0xffffffffu, good, 0);
       if (!good) break;
       tc_fence_after();
-      if (is_tail) {
-        // raw accumulator to this pair's workspace slot, then count this warp in
-        float* ws = p.sk_ws + (((long long)pair * 2 + rank) * BM + row) * BN_MAX;
-        for (int c = half; c < bn / 32; c += 2) {
-          if (n0 + c * 32 >= p.N) break;
+      const int n_chunks = min(bn / 32, (p.N - n0 + 31) / 32);   // column chunks of this tile that exist
+      int sl = 0, grp = 0;                                       // slice index and first pair of the tile's group
+      if (w.sliced) {
+        grp = (pair / p.slices) * p.slices;
+        sl = pair - grp;
+        // 1. raw accumulator of this slice to the workspace slot of this pair
+        float* wsw = p.sk_ws + (((long long)pair * 2 + rank) * BM + row) * BN_MAX;
+        for (int c = half; c < n_chunks; c += 2) {
           float v[32];
           tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
 #pragma unroll
           for (int q = 0; q < 8; ++q)
-            __stcg(reinterpret_cast<float4*>(ws + c * 32) + q, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
+            __stcg(reinterpret_cast<float4*>(wsw + c * 32) + q, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
         }
+        // the accumulator is free again; the tensor pipe has no further use for it in this pair
+        tc_fence_before();
         __threadfence();
         __syncwarp();
-        if (lane == 0) atomicAdd(p.sk_flags + pair, 1);
-      } else {
-        const float* ws = nullptr;
-        if (is_head) {
-          // the rest of this tile was computed (earlier in time) by pair + 1: wait for its 16 warps
-          ws = p.sk_ws + (((long long)(pair + 1) * 2 + rank) * BM + row) * BN_MAX;
-          if (lane == 0) {
-            const volatile int* flag = p.sk_flags + pair + 1;
-            const unsigned long long t0 = globaltimer();
-            while (*flag < 16) {
-              if (*abort_flag || globaltimer() - t0 > WAIT_LIMIT_NS) { atomicCAS(p.err, 0, 5); *abort_flag = 1; good = 0; break; }
-            }
-            __threadfence();
+        if (lane == 0) {
+          mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
+          atomicAdd(p.sk_flags + pair / p.slices, 1);
+          // 2. wait until the 16 warps of every slice of this tile have stored theirs
+          const volatile int* flag = p.sk_flags + pair / p.slices;
+          const int want = 16 * p.slices;
+          const unsigned long long t0 = globaltimer();
+          while (*flag < want) {
+            if (*abort_flag || globaltimer() - t0 > WAIT_LIMIT_NS) { atomicCAS(p.err, 0, 5); *abort_flag = 1; good = 0; break; }
           }
-          good = __shfl_sync(0xffffffffu, good, 0);
-          if (!good) break;
+          __threadfence();
         }
+        good = __shfl_sync(0xffffffffu, good, 0);
+        if (!good) break;
+      }
+      {
         const int m = m0 + row;
         const bool m_ok = m < p.M;
         const float* zrow = p.dsig ? p.dsig + (long long)(m % p.dsig_rows) * p.ld_dsig : nullptr;
         const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
         float* drow = p.D + (long long)m * p.ldd;
-        for (int c = half; c < bn / 32; c += 2) {
+        // whole tile: this warp's chunks are half, half + 2, ...; sliced tile: the pair's share of the
+        // chunks is sl, sl + slices, ..., dealt alternately to the two warps of a quadrant
+        const int c_first = w.sliced ? sl + half * p.slices : half;
+        const int c_step = w.sliced ? 2 * p.slices : 2;
+        for (int c = c_first; c < n_chunks; c += c_step) {
           const int nb = n0 + c * 32;
-          if (nb >= p.N) break;
           const bool fullc = p.vec_epi && nb + 32 <= p.N;
-          float4 zc[8], ci[8], pw[8];
+          float4 zc[8], ci[8];
           if (fullc && m_ok) {
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
@@ -642,15 +630,21 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
               ci[q] = crow ? __ldg(reinterpret_cast<const float4*>(crow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
           }
-          if (ws) {
-#pragma unroll
-            for (int q = 0; q < 8; ++q) pw[q] = __ldcg(reinterpret_cast<const float4*>(ws + c * 32) + q);
-          }
           float v[32];
-          tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
-          if (ws) {
+          if (!w.sliced) {
+            tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
+          } else {
+            // sum of the slices' partials, slice 0 first
 #pragma unroll
-            for (int q = 0; q < 8; ++q) { v[4 * q] += pw[q].x; v[4 * q + 1] += pw[q].y; v[4 * q + 2] += pw[q].z; v[4 * q + 3] += pw[q].w; }
+            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+            for (int s2 = 0; s2 < p.slices; ++s2) {
+              const float* wsr = p.sk_ws + (((long long)(grp + s2) * 2 + rank) * BM + row) * BN_MAX + c * 32;
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                const float4 x = __ldcg(reinterpret_cast<const float4*>(wsr) + q);
+                v[4 * q] += x.x; v[4 * q + 1] += x.y; v[4 * q + 2] += x.z; v[4 * q + 3] += x.w;
+              }
+            }
           }
           if (!m_ok) continue;
           if (fullc) {
@@ -686,9 +680,11 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
+      if (!w.sliced) {       // (a sliced tile released its accumulator right after storing it)
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
+      }
     }
   }
   tc_fence_before();
@@ -816,7 +812,7 @@ int choose_bn2(int M, int N, bool stream_k) {
 }
 
 int64_t gemm_tf32_workspace_floats() { return (int64_t)(num_sms() / 2) * 2 * BM * BN_MAX; }
-int gemm_tf32_workspace_flags() { return num_sms() / 2 + 1; }
+int gemm_tf32_workspace_flags() { return num_sms() / 2; }
 
 int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st) {
   static bool attr_set = false;
@@ -870,25 +866,27 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
   if (two_cta) {
     p.tiles = ((g.M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;   // tiles of 256 rows, one per CTA pair
     const int pairs = num_sms() / 2;
-    // active pairs: all of them when there is at least a tile each; two per tile (each tile cut once in
-    // the middle) when that still fits; else one per tile.  A range never holds less than half a tile,
-    // so no tile is cut more than once per pair boundary.
+    const int total_kb = p.kblocks[0] + p.kblocks[1];
     p.sk_ws = sk_ws; p.sk_flags = sk_flags;
-    p.sk_split = 0;
-    p.sk_pairs = p.tiles < pairs ? p.tiles : pairs;
-    if (p.tiles >= pairs) {
-      p.sk_W = (p.tiles + pairs - 1) / pairs;
-      p.sk_r = p.tiles - (p.sk_W - 1) * pairs;
+    p.P = p.tiles < pairs ? p.tiles : pairs;
+    p.waves = p.tiles / p.P;
+    p.rem = p.tiles - p.waves * p.P;
+    p.slices = 1;
+    int launch_pairs = p.P;
+    if (stream_k && p.tiles < pairs) {
+      // fewer tiles than pairs: there is no full wave; every tile is cut along K over pairs / tiles pairs
+      p.P = pairs; p.waves = 0; p.rem = p.tiles;
     }
-    if (stream_k) {
-      const int total_kb = p.kblocks[0] + p.kblocks[1];
-      // Splitting is used only for under-filled problems (each tile cut once in the middle, two pairs per
-      // tile).  With more tiles than pairs an even split was measured to lose: the pairs drift apart
-      // over the waves, tiles of one A panel are then processed at different times and miss in L2.
-      if (2 * p.tiles <= pairs && total_kb >= 2) { p.sk_pairs = 2 * p.tiles; p.sk_split = 1; }
-      if (p.sk_split) cudaMemsetAsync(sk_flags, 0, sizeof(int) * (pairs + 1), st);
+    if (stream_k && p.rem > 0) {
+      int sl = pairs / p.rem;
+      if (sl > 8) sl = 8;
+      if (sl > total_kb) sl = total_kb;
+      // a slice costs a store and a re-read of the tile on top of its MMAs: not worth it for short K
+      if (sl >= 2 && total_kb / sl >= 4) p.slices = sl;
     }
-    gemm_tf32_2cta_kernel<kStages2><<<2 * p.sk_pairs, 320, kSmemBytes2, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+    if (p.waves == 0) launch_pairs = p.rem * p.slices;
+    if (p.slices >= 2) cudaMemsetAsync(sk_flags, 0, sizeof(int) * pairs, st);
+    gemm_tf32_2cta_kernel<kStages2><<<2 * launch_pairs, 320, kSmemBytes2, st>>>(maps[0], maps[1], maps[2], maps[3], p);
   } else {
     p.tiles = ((g.M + BM - 1) / BM) * p.tiles_n;
     const int grid = p.tiles < num_sms() ? p.tiles : num_sms();

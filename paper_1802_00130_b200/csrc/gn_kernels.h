@@ -41,8 +41,8 @@ int launch_gemm_ffma(const GemmArgs& g, cudaStream_t st);
 // *err_flag receives a non-zero code if a bounded device-side wait ran out.  Returns launches made,
 // or -1 if a tensor map could not be encoded.
 // sk_ws / sk_flags: optional workspace of gemm_tf32_workspace_floats() floats and
-// gemm_tf32_workspace_flags() ints that lets the two-CTA kernel split tiles between CTA pairs
-// (stream-K); pass nullptr to keep whole tiles.
+// gemm_tf32_workspace_flags() ints that lets the two-CTA kernel cut the tiles of its last, partial
+// wave along K over the idle CTA pairs; pass nullptr to keep whole tiles.
 bool gemm_tf32_eligible(const GemmArgs& g);
 int64_t gemm_tf32_workspace_floats();
 int gemm_tf32_workspace_flags();
