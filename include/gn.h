@@ -173,6 +173,14 @@ gn_status gn_cg_solve_host(gn_ctx* ctx, const float* h_g, double lambda, int blo
                            double* resnorm_host);
 
 /*
+ * gn_debug_timeout_probe - test hook for the failure path of the tensor-core pipeline: launches one
+ * CTA that waits, with the pipeline's bounded-wait code and the given limit (0 < limit_ms <= 1000), on a
+ * barrier nothing arrives on.  The wait runs out, the kernel records its code and returns, and the call
+ * reports GN_ETIMEOUT like any synchronising call would after a timed-out GEMM.  The context stays usable.
+ */
+gn_status gn_debug_timeout_probe(gn_ctx* ctx, double limit_ms);
+
+/*
  * gn_debug_activations - copy the stored Z_m (m in 1..L, [|S|][n_m]) of the current subsample to a
  * device buffer; a test hook for the stored forward pass (Eq. xtoz).
  */

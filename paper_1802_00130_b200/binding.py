@@ -35,6 +35,7 @@ _SIGNATURES = {
     "gn_cg_solve": (_i32, [_vp, _vp, _dbl, _i32, _i32, _dbl, _vp, C.POINTER(_i32), _vp, C.POINTER(_dbl)]),
     "gn_cg_solve_host": (_i32, [_vp, _vp, _dbl, _i32, _i32, _dbl, _vp, C.POINTER(_i32), C.POINTER(_dbl)]),
     "gn_debug_activations": (_i32, [_vp, _i32, _vp]),
+    "gn_debug_timeout_probe": (_i32, [_vp, _dbl]),
     "gn_profile": (_i32, [_vp, _i32]),
     "gn_profile_read": (_i32, [_vp, C.POINTER(_dbl), C.POINTER(_dbl), C.POINTER(_i64)]),
     "gn_thin_m_gemm_noalloc": (_i32, [_i32, _i32, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp, C.c_char_p, _i64]),
@@ -270,6 +271,10 @@ class GnContext:
                                             int(a_kmajor), _dev_ptr(B, torch.float32), B.stride(0), int(b_kmajor),
                                             _dev_ptr(D, torch.float32), D.stride(0)))
         return D
+
+    def debug_timeout_probe(self, limit_ms=1.0):
+        """Test hook: raises GnError(GN_ETIMEOUT) after a bounded device wait has run out."""
+        self._check(self._lib.gn_debug_timeout_probe(self._h, float(limit_ms)))
 
     def debug_activations(self, m):
         import torch

@@ -695,6 +695,22 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
   }
 }
 
+// One CTA waits on an mbarrier that nothing ever arrives on, with the same bounded-wait code the GEMM
+// roles use but a caller-chosen limit; it must record its code and return.  Exercises the path from a
+// timed-out device wait to GN_ETIMEOUT on the host without hanging anything.
+__global__ void timeout_probe_kernel(int* err, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const unsigned long long t0 = globaltimer();
+    bool done = false;
+    while (!(done = mbar_test_wait(&bar, 0))) {
+      if (globaltimer() - t0 > limit_ns) { atomicCAS(err, 0, 9); break; }
+    }
+  }
+}
+
 // ---- host side ---------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -782,6 +798,11 @@ int choose_bn(int M, int N) {
 }
 
 }  // namespace
+
+int launch_timeout_probe(int* err_flag, unsigned long long limit_ns, cudaStream_t st) {
+  timeout_probe_kernel<<<1, 32, 0, st>>>(err_flag, limit_ns);
+  return 1;
+}
 
 bool gemm_tf32_eligible(const GemmArgs& g) {
   if (g.M < 1 || g.N < 1) return false;

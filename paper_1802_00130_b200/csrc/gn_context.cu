@@ -744,6 +744,14 @@ gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* d
   return sync(c, "debug_gemm");
 }
 
+gn_status gn_debug_timeout_probe(gn_ctx* c, double limit_ms) {
+  if (!c) return GN_EINVAL;
+  if (!(limit_ms > 0.0) || limit_ms > 1000.0) return fail(c, GN_EINVAL, "limit must be in (0, 1000] ms");
+  c->launches += launch_timeout_probe(c->err_flag + 1, (unsigned long long)(limit_ms * 1e6), c->st);
+  GN_TRY(check_launch(c, "timeout probe"));
+  return sync(c, "timeout probe");
+}
+
 gn_status gn_debug_activations(gn_ctx* c, int m, float* d_out) {
   if (!c) return GN_EINVAL;
   if (!d_out || m < 1 || m > c->L) return fail(c, GN_EINVAL, "bad layer / NULL output");

@@ -56,6 +56,9 @@ ThinKind gemm_thin_kind(const GemmArgs& g);
 int64_t gemm_thin_scratch_floats(const GemmArgs& g);
 int launch_gemm_thin(const GemmArgs& g, float* scratch, cudaStream_t st);
 
+// A one-CTA kernel whose bounded wait (limit_ns) can never be satisfied: writes code 9 to *err_flag.
+int launch_timeout_probe(int* err_flag, unsigned long long limit_ns, cudaStream_t st);
+
 // ---- vector / memory-bound kernels -------------------------------------------------------------
 // Row gather dst[r][:] = src[idx[r]][:]; rows with idx outside [0, src_rows) are zero-filled and
 // *err_flag is set to 1.

@@ -211,3 +211,20 @@ def test_symmetry_and_positive_definiteness_on_device():
         assert abs(u @ Gv - v @ Gu) <= 1e-4 * abs(u @ Gv)
         assert v @ Gv >= v.astype(np.float64) @ v / p["C"]
     ctx.close()
+
+
+def test_a_timed_out_device_wait_is_reported_and_the_context_survives():
+    import paper_1802_00130_b200 as gn
+    p = wl.make("mid")
+    ctx = make_ctx(p, "tf32")
+    ctx.set_subsample(dev(p["idx"]))
+    before = ctx.Gv(dev(p["v"])).clone()
+    with pytest.raises(gn.GnError) as e:
+        ctx.debug_timeout_probe(1.0)                 # a barrier nothing arrives on, 1 ms limit
+    assert e.value.status == 5 and "bounded wait" in str(e.value)
+    # the error word was cleared and the device context is intact: same product, bit for bit
+    import torch
+    assert torch.equal(ctx.Gv(dev(p["v"])), before)
+    g, f = ctx.grad(with_f=True)                     # a synchronising call reports no stale error
+    assert np.isfinite(f)
+    ctx.close()
