@@ -302,3 +302,58 @@ def cg_solve(theta, widths, C, XS, g, lam, blockdiag, max_iter, tol):
         return cg(lambda p: Gv_blockdiag(theta, widths, C, XS, p), g, lam, max_iter, tol,
                   segments=block_slices(widths))
     return cg(lambda p: Gv(theta, widths, C, XS, p), g, lam, max_iter, tol)
+
+
+# --------------------------------------------------------------------------- Newton iteration (Algorithm 3 on one node)
+def combine_directions(a, b, c, r1, r2, eps):
+    """Two-variable system of Eq. (sol-comp): [[a, b], [b, c]] (beta1, beta2) = (r1, r2) with
+    a = d^T G d, b = dbar^T G d, c = dbar^T G dbar, r1 = -g^T d, r2 = -g^T dbar.
+    Eq. (determinant): beta = (1, 0) when the determinant is at most eps."""
+    det = a * c - b * b
+    if det <= eps:
+        return 1.0, 0.0
+    return (r1 * c - b * r2) / det, (a * r2 - b * r1) / det
+
+
+def lm_update(lam, rho, drop, boost):
+    """Eq. (LM-rules)."""
+    if rho > 0.75:
+        return lam * drop
+    if rho >= 0.25:
+        return lam
+    return lam * boost
+
+
+def newton_iteration(theta, widths, C, X, Y, idx, dprev, lam, sigma=1e-3, eta=1e-4, cg_max=250, eps=1e-5,
+                     drop=2.0 / 3.0, boost=1.5, blockdiag=True, max_backtrack=30):
+    """One pass of the loop body of Algorithm 3 with a single partition holding everything.
+
+    g on all rows; CG on the (block-diagonal or full) subsampled system with lambda (Eq. block-gaussnewton);
+    direction combination with the previous direction on the full G^S (Eq. linear-comb-now); back-tracking
+    line search alpha in {1, 1/2, ...} (Eq. linesearch-condition); rho and the next lambda (Eq. LM-rules).
+    Returns (theta_next, d, lam_next, report).
+    """
+    theta = np.asarray(theta, dtype=np.float64)
+    dprev = np.asarray(dprev, dtype=np.float64)
+    XS = np.asarray(X)[np.asarray(idx)]
+    f0 = fun(theta, widths, C, X, Y)
+    g = grad(theta, widths, C, X, Y)
+    d, its, _ = cg_solve(theta, widths, C, XS, g, lam, blockdiag, cg_max, sigma)
+    Gd = Gv(theta, widths, C, XS, d)
+    Gdb = Gv(theta, widths, C, XS, dprev)
+    a, b, c = d @ Gd, dprev @ Gd, dprev @ Gdb
+    beta1, beta2 = combine_directions(a, b, c, -(g @ d), -(g @ dprev), eps)
+    dnew = beta1 * d + beta2 * dprev
+    gTd = g @ dnew
+    dGd = beta1 * beta1 * a + 2.0 * beta1 * beta2 * b + beta2 * beta2 * c
+    alpha, backtracks = 1.0, 0
+    f1 = fun(theta + alpha * dnew, widths, C, X, Y)
+    while f1 > f0 + eta * alpha * gTd and backtracks < max_backtrack:
+        alpha *= 0.5
+        backtracks += 1
+        f1 = fun(theta + alpha * dnew, widths, C, X, Y)
+    rho = (f1 - f0) / (alpha * gTd + 0.5 * alpha * alpha * dGd)
+    lam_next = lm_update(lam, rho, drop, boost)
+    report = dict(f_before=f0, f_after=f1, alpha=alpha, beta1=beta1, beta2=beta2, rho=rho, gTd=gTd, dGd=dGd,
+                  cg_iters=len(its), backtracks=backtracks, lambda_next=lam_next)
+    return theta + alpha * dnew, dnew, lam_next, report
