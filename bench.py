@@ -257,6 +257,17 @@ def run_ours(args):
                            "executed_tflops": 2.0 * mac_exec * p["nS"] / t / 1e12,
                            "algorithmic_tflops": 2.0 * mac_alg * p["nS"] / t / 1e12}
 
+    # ---- one Newton iteration of Algorithm 3 (block-diagonal CG capped at n_cg steps), for context
+    th_n, dir_n = theta.clone(), torch.zeros_like(theta)
+    prm = gn.NewtonParams(lam=1.0, sigma=1e-3, cg_max=n_cg, blockdiag=1)
+    ctx.newton_iter(th_n, idx_dev[0], dir_n, prm)
+    torch.cuda.synchronize()
+    t0n = time.perf_counter()
+    rep_n = ctx.newton_iter(th_n, idx_dev[1], dir_n, prm)
+    torch.cuda.synchronize()
+    breakdown["newton_iter"] = {"ms": 1e3 * (time.perf_counter() - t0n), "cg_iters": rep_n["cg_iters"],
+                                "backtracks": rep_n["backtracks"], "f_before": rep_n["f_before"], "f_after": rep_n["f_after"]}
+
     # ---- end to end through the host-buffer entry points (pinned host memory)
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory().numpy()
     h_theta, h_g, h_d = pin(p["theta"]), pin(np.zeros(ctx.n, np.float32)), pin(np.zeros(ctx.n, np.float32))

@@ -173,6 +173,44 @@ gn_status gn_cg_solve_host(gn_ctx* ctx, const float* h_g, double lambda, int blo
                            double* resnorm_host);
 
 /*
+ * gn_newton_iter - one iteration of the subsampled Newton method of Algorithm 3 with everything on this
+ * GPU (no partitions, no communication):
+ *   1. g = grad f(theta) over all rows, f(theta);
+ *   2. CG for d on (Ghat^S + lambda I) d = -g (blockdiag != 0, Eq. block-gaussnewton) or on the full
+ *      system (Eq. sample-gaussnewton), stop rule of Eq. (CG-stopping-cond) with sigma, at most cg_max steps;
+ *   3. d <- beta1 d + beta2 dbar with dbar the previous direction, (beta1, beta2) from the two-variable
+ *      system of Eq. (sol-comp) on the full G^S; (1, 0) if its determinant is <= eps (Eq. determinant);
+ *   4. back-tracking line search: largest alpha in {1, 1/2, 1/4, ...} with
+ *      f(theta + alpha d) <= f(theta) + eta alpha g^T d (Eq. linesearch-condition), at most max_backtrack halvings;
+ *   5. rho = (f(theta + alpha d) - f(theta)) / (alpha g^T d + alpha^2/2 d^T G^S d) and the next lambda by
+ *      Eq. (LM-rules) with (drop, boost).
+ * d_theta [n] is updated in place to theta + alpha d; d_dir [n] holds dbar on entry (all zeros at the first
+ * iteration, as the paper prescribes) and the new direction d on return; d_idx / nS choose S_k (Section 4.3).
+ * The paper's constants: sigma = 0.001, cg_max = 250, lambda_1 = 1, (drop, boost) = (2/3, 3/2), eps = 1e-5;
+ * it leaves eta in (0, 1) open.  Synchronises the stream; the context's theta is the new theta on return and
+ * the subsample must be set again before products are asked for.
+ */
+typedef struct {
+  double lambda;      /* lambda_k */
+  double sigma;       /* CG tolerance; <= 0 runs exactly cg_max steps */
+  double eta;         /* sufficient-decrease constant */
+  double eps;         /* determinant guard */
+  double drop, boost; /* Levenberg-Marquardt factors */
+  int32_t cg_max;
+  int32_t blockdiag;
+  int32_t max_backtrack;
+  int32_t reserved;
+} gn_newton_params;
+
+typedef struct {
+  double f_before, f_after, alpha, beta1, beta2, rho, gTd, dGd, lambda_next;
+  int32_t cg_iters, backtracks;
+} gn_newton_report;
+
+gn_status gn_newton_iter(gn_ctx* ctx, float* d_theta, const int32_t* d_idx, int64_t nS, float* d_dir,
+                         const gn_newton_params* params, gn_newton_report* report);
+
+/*
  * gn_debug_timeout_probe - test hook for the failure path of the tensor-core pipeline: launches one
  * CTA that waits, with the pipeline's bounded-wait code and the given limit (0 < limit_ms <= 1000), on a
  * barrier nothing arrives on.  The wait runs out, the kernel records its code and returns, and the call

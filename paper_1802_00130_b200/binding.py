@@ -35,12 +35,31 @@ _SIGNATURES = {
     "gn_cg_solve": (_i32, [_vp, _vp, _dbl, _i32, _i32, _dbl, _vp, C.POINTER(_i32), _vp, C.POINTER(_dbl)]),
     "gn_cg_solve_host": (_i32, [_vp, _vp, _dbl, _i32, _i32, _dbl, _vp, C.POINTER(_i32), C.POINTER(_dbl)]),
     "gn_debug_activations": (_i32, [_vp, _i32, _vp]),
+    "gn_newton_iter": (_i32, [_vp, _vp, _vp, _i64, _vp, _vp, _vp]),
     "gn_debug_timeout_probe": (_i32, [_vp, _dbl]),
     "gn_profile": (_i32, [_vp, _i32]),
     "gn_profile_read": (_i32, [_vp, C.POINTER(_dbl), C.POINTER(_dbl), C.POINTER(_i64)]),
     "gn_thin_m_gemm_noalloc": (_i32, [_i32, _i32, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp, C.c_char_p, _i64]),
     "gn_debug_gemm": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64]),
 }
+
+
+class NewtonParams(C.Structure):
+    """gn_newton_params; defaults are the paper's constants (eta is left open there)."""
+    _fields_ = [("lam", _dbl), ("sigma", _dbl), ("eta", _dbl), ("eps", _dbl), ("drop", _dbl), ("boost", _dbl),
+                ("cg_max", _i32), ("blockdiag", _i32), ("max_backtrack", _i32), ("reserved", _i32)]
+
+    def __init__(self, lam=1.0, sigma=1e-3, eta=1e-4, eps=1e-5, drop=2.0 / 3.0, boost=1.5, cg_max=250, blockdiag=1,
+                 max_backtrack=30):
+        super().__init__(lam, sigma, eta, eps, drop, boost, cg_max, blockdiag, max_backtrack, 0)
+
+
+class NewtonReport(C.Structure):
+    _fields_ = [("f_before", _dbl), ("f_after", _dbl), ("alpha", _dbl), ("beta1", _dbl), ("beta2", _dbl), ("rho", _dbl),
+                ("gTd", _dbl), ("dGd", _dbl), ("lambda_next", _dbl), ("cg_iters", _i32), ("backtracks", _i32)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
 
 
 class GnError(RuntimeError):
@@ -271,6 +290,15 @@ class GnContext:
                                             int(a_kmajor), _dev_ptr(B, torch.float32), B.stride(0), int(b_kmajor),
                                             _dev_ptr(D, torch.float32), D.stride(0)))
         return D
+
+    def newton_iter(self, theta, idx, direction, params):
+        """One iteration of Algorithm 3 on this GPU; theta and direction are updated in place.  Returns the report."""
+        import torch
+        rep = NewtonReport()
+        self._check(self._lib.gn_newton_iter(self._h, _dev_ptr(theta, torch.float32, self.n), _dev_ptr(idx, torch.int32),
+                                             idx.numel(), _dev_ptr(direction, torch.float32, self.n), C.byref(params),
+                                             C.byref(rep)))
+        return rep.as_dict()
 
     def debug_timeout_probe(self, limit_ms=1.0):
         """Test hook: raises GnError(GN_ETIMEOUT) after a bounded device wait has run out."""

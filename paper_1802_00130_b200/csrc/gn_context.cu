@@ -50,6 +50,7 @@ struct gn_ctx {
   // CG
   float* cg_r = nullptr; float* cg_p = nullptr; float* cg_q = nullptr;
   float* tmp_a = nullptr; float* tmp_b = nullptr;  // staging for *_host calls
+  float* nt[4] = {nullptr, nullptr, nullptr, nullptr};  // Newton iteration: g, d, G d / G dbar, trial theta
   CgChunk* chunks[2] = {nullptr, nullptr}; int n_chunks[2] = {0, 0};
   CgSeg* segs = nullptr;
 
@@ -476,10 +477,10 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
     if ((s = dev_alloc(c, &c->cg_r, c->n)) != GN_OK) break;
     if ((s = dev_alloc(c, &c->cg_p, c->n)) != GN_OK) break;
     if ((s = dev_alloc(c, &c->cg_q, c->n)) != GN_OK) break;
-    if ((s = dev_alloc(c, &c->dscal, 8)) != GN_OK) break;
+    if ((s = dev_alloc(c, &c->dscal, 16)) != GN_OK) break;
     if ((s = dev_alloc(c, &c->err_flag, 2)) != GN_OK) break;
     if (cudaMemset(c->err_flag, 0, 2 * sizeof(int)) != cudaSuccess) { s = GN_ECUDA; break; }
-    if (cudaMallocHost(&c->hscal, 8 * sizeof(double)) != cudaSuccess) { s = GN_ENOMEM; break; }
+    if (cudaMallocHost(&c->hscal, 16 * sizeof(double)) != cudaSuccess) { s = GN_ENOMEM; break; }
     if (cudaMallocHost(&c->h_err, 2 * sizeof(int)) != cudaSuccess) { s = GN_ENOMEM; break; }
     c->h_err[0] = c->h_err[1] = 0;
     if ((s = build_chunks(c)) != GN_OK) break;
@@ -742,6 +743,73 @@ gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* d
   }
   GN_TRY(check_launch(c, "debug_gemm"));
   return sync(c, "debug_gemm");
+}
+
+// x^T y into device scalar slot (fixed-order double-precision sum of per-chunk partials)
+static void dot_to_slot(gn_ctx* c, const float* x, const float* y, int slot) {
+  c->launches += launch_cg_dot(x, y, c->chunks[0], c->n_chunks[0], c->partial, c->st);
+  c->launches += launch_sum_partials(c->partial, c->n_chunks[0], c->dscal + slot, false, c->st);
+}
+
+gn_status gn_newton_iter(gn_ctx* c, float* d_theta, const int32_t* d_idx, int64_t nS, float* d_dir,
+                         const gn_newton_params* prm, gn_newton_report* rep) {
+  if (!c) return GN_EINVAL;
+  if (!d_theta || !d_idx || !d_dir || !prm || !rep) return fail(c, GN_EINVAL, "NULL argument");
+  if (!(prm->lambda >= 0.0) || prm->cg_max < 1 || !(prm->eta > 0.0 && prm->eta < 1.0) || prm->max_backtrack < 0 ||
+      !(prm->drop > 0.0) || !(prm->boost > 0.0))
+    return fail(c, GN_EINVAL, "bad Newton parameters");
+  for (int i = 0; i < 4; ++i)
+    if (!c->nt[i]) GN_TRY(dev_alloc(c, &c->nt[i], c->n));
+  float* g = c->nt[0]; float* d = c->nt[1]; float* Gx = c->nt[2]; float* trial = c->nt[3];
+  const float inv_C = (float)(1.0 / c->C);
+  std::memset(rep, 0, sizeof(*rep));
+
+  GN_TRY(gn_set_theta(c, d_theta));
+  GN_TRY(gn_set_subsample(c, d_idx, nS));
+  double f0 = 0.0;
+  GN_TRY(fun_grad(c, g, &f0));
+  int its = 0;
+  GN_TRY(gn_cg_solve(c, g, prm->lambda, prm->blockdiag, prm->cg_max, prm->sigma, d, &its, nullptr, nullptr));
+  // entries of the two-variable system on the full G^S (Eq. sol-comp)
+  GN_TRY(product_full(c, d, Gx, inv_C));
+  dot_to_slot(c, d, Gx, 4);          // a  = d^T G d
+  dot_to_slot(c, d_dir, Gx, 5);      // b  = dbar^T G d
+  GN_TRY(product_full(c, d_dir, Gx, inv_C));
+  dot_to_slot(c, d_dir, Gx, 6);      // c  = dbar^T G dbar
+  dot_to_slot(c, g, d, 7);           // g^T d
+  dot_to_slot(c, g, d_dir, 8);       // g^T dbar
+  GN_CUDA(c, cudaMemcpyAsync(c->hscal + 4, c->dscal + 4, 5 * sizeof(double), cudaMemcpyDeviceToHost, c->st));
+  GN_TRY(check_launch(c, "newton: direction combination"));
+  GN_TRY(sync(c, "newton: direction combination"));
+  const double a = c->hscal[4], b = c->hscal[5], cc = c->hscal[6], gd = c->hscal[7], gdb = c->hscal[8];
+  double beta1 = 1.0, beta2 = 0.0;
+  const double det = a * cc - b * b;
+  if (det > prm->eps) { beta1 = (-gd * cc + b * gdb) / det; beta2 = (-a * gdb + b * gd) / det; }
+  // d <- beta1 d + beta2 dbar, kept in d_dir (it is the next iteration's dbar)
+  c->launches += launch_axpby(c->n, (float)beta1, d, (float)beta2, d_dir, d_dir, c->st);
+  const double gTd = beta1 * gd + beta2 * gdb;
+  const double dGd = beta1 * beta1 * a + 2.0 * beta1 * beta2 * b + beta2 * beta2 * cc;
+  // back-tracking line search (Eq. linesearch-condition)
+  double alpha = 1.0, f1 = 0.0;
+  int backtracks = 0;
+  for (;;) {
+    c->launches += launch_axpby(c->n, 1.f, d_theta, (float)alpha, d_dir, trial, c->st);
+    GN_TRY(gn_set_theta(c, trial));
+    GN_TRY(fun_grad(c, nullptr, &f1));
+    if (f1 <= f0 + prm->eta * alpha * gTd || backtracks >= prm->max_backtrack) break;
+    alpha *= 0.5;
+    ++backtracks;
+  }
+  GN_CUDA(c, cudaMemcpyAsync(d_theta, trial, c->n * sizeof(float), cudaMemcpyDeviceToDevice, c->st));
+  GN_TRY(sync(c, "newton: update"));
+  const double rho = (f1 - f0) / (alpha * gTd + 0.5 * alpha * alpha * dGd);
+  double lam = prm->lambda;
+  if (rho > 0.75) lam *= prm->drop;
+  else if (!(rho >= 0.25)) lam *= prm->boost;
+  rep->f_before = f0; rep->f_after = f1; rep->alpha = alpha; rep->beta1 = beta1; rep->beta2 = beta2;
+  rep->rho = rho; rep->gTd = gTd; rep->dGd = dGd; rep->lambda_next = lam;
+  rep->cg_iters = its; rep->backtracks = backtracks;
+  return GN_OK;
 }
 
 gn_status gn_debug_timeout_probe(gn_ctx* c, double limit_ms) {

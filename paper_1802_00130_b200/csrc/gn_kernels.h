@@ -80,6 +80,9 @@ int launch_loss_delta(const float* Z, const float* Y, int64_t count, float* delt
 // Fixed-order double-precision sum of `count` partials: *out (+)= sum.
 int launch_sum_partials(const double* partial, int count, double* out, bool accumulate, cudaStream_t st);
 
+// out[i] = a x[i] + b y[i]; out may be x or y.
+int launch_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out, cudaStream_t st);
+
 // Transposed copy dst[c][r] = src[r][c] (src rows x cols).
 int launch_transpose(const float* src, int rows, int cols, float* dst, cudaStream_t st);
 

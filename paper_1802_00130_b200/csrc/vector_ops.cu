@@ -158,6 +158,14 @@ __global__ void __launch_bounds__(256) sum_partials_kernel(const double* __restr
   if (threadIdx.x == 0) *out = accumulate ? *out + t : t;
 }
 
+// ---------------------------------------------------------------------------------- out = a x + b y
+__global__ void __launch_bounds__(256) axpby_kernel(long long n, float a, const float* x, float b, const float* y,
+                                                    float* out) {
+  // out may be x or y (same index read and written by the same thread)
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256)
+    out[i] = fmaf(a, x[i], b * y[i]);
+}
+
 // ---------------------------------------------------------------------------------- transpose
 __global__ void __launch_bounds__(256) transpose_kernel(const float* __restrict__ src, int rows, int cols,
                                                         float* __restrict__ dst) {
@@ -330,6 +338,13 @@ int launch_loss_delta(const float* Z, const float* Y, int64_t count, float* delt
 
 int launch_sum_partials(const double* partial, int count, double* out, bool accumulate, cudaStream_t st) {
   sum_partials_kernel<<<1, 256, 0, st>>>(partial, count, out, accumulate ? 1 : 0);
+  return 1;
+}
+
+int launch_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out, cudaStream_t st) {
+  long long blocks = (n + 255) / 256;
+  if (blocks > 148LL * 16) blocks = 148LL * 16;
+  axpby_kernel<<<(unsigned)blocks, 256, 0, st>>>(n, a, x, b, y, out);
   return 1;
 }
 
