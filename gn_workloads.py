@@ -8,7 +8,8 @@ Every workload is a dict of numpy arrays in the layouts the C ABI expects:
 
     X      float32 [l][n_0]   row-major feature rows
     labels int64   [l]        class of each row
-    Y      float32 [l][n_L]   one-hot label rows (Section 1 of the paper)
+    Y      float32 [l][n_L]   one-hot label rows (Section 1 of the paper), or one column of -1 / +1
+                              for the two-class, scalar-output setting (Section 8.3)
     theta  float32 [n]        model vector, per layer: columns of W^m concatenated,
                               then b^m (Section 2.1)
     idx    int32   [|S|]      subsample, drawn without replacement
@@ -38,6 +39,8 @@ WORKLOADS = {
     "ragged": dict(widths=[37, 53, 19, 7], l=333, nS=131, C=3.0, x="sparse80", seed=1011),
     "mid": dict(widths=[200, 260, 140, 10], l=3000, nS=700, C=30.0, x="sparse80", seed=1012),
     "single": dict(widths=[50, 6], l=400, nS=150, C=2.0, x="normal", seed=1013),
+    # scalar output with labels -1 / +1 (the paper's two-class setting of Section 8.3), HIGGS-like shape
+    "binary300": dict(widths=[28, 300, 300, 1], l=20000, nS=2000, C=20000.0, x="normal", seed=1014, y="pm1"),
 }
 
 
@@ -89,9 +92,13 @@ def make(name, l=None, nS=None, with_v=True):
         raise ValueError("need 0 < nS <= l")
     rng = np.random.Generator(np.random.PCG64(rec["seed"]))
     X = draw_rows(rng, rec["x"], l, widths[0])
-    labels = rng.integers(0, widths[-1], size=l)
-    Y = np.zeros((l, widths[-1]), dtype=np.float32)
-    Y[np.arange(l), labels] = 1.0
+    if rec.get("y") == "pm1":
+        labels = rng.integers(0, 2, size=l)
+        Y = (2.0 * labels - 1.0).astype(np.float32).reshape(l, 1)
+    else:
+        labels = rng.integers(0, widths[-1], size=l)
+        Y = np.zeros((l, widths[-1]), dtype=np.float32)
+        Y[np.arange(l), labels] = 1.0
     theta = draw_theta(rng, widths)
     idx = rng.permutation(l)[:nS].astype(np.int32)
     n = num_params(widths)

@@ -32,7 +32,7 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).to("cuda:0")
 
 
-SMALL = ["tiny", "ragged", "single", "mid"]
+SMALL = ["tiny", "ragged", "single", "mid", "binary300"]
 
 
 @pytest.mark.parametrize("mode", ["fp32", "tf32"])

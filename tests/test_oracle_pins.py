@@ -354,3 +354,18 @@ def test_cost_formula_fixture():
         assert sum(g) == int(fwd)
         assert 2 * g[0] + 4 * sum(g[1:]) == int(full)
         assert sum(2 * g[m - 1] + 2 * w[-1] * w[m] for m in range(1, len(w))) == int(paper_block)
+
+
+def test_scalar_output_with_plus_minus_one_labels():
+    # Section 8.3: n_L = 1, y in {-1, +1}.  f(0) = mean y^2 = 1 again, and the gradient still matches differences of f
+    p = wl.make("binary300", l=40, nS=10)
+    assert set(np.unique(p["Y"]).tolist()) <= {-1.0, 1.0} and p["Y"].shape == (40, 1)
+    assert orc.fun(np.zeros(p["n"]), p["widths"], p["C"], p["X"], p["Y"]) == pytest.approx(1.0)
+    th = p["theta"].astype(np.float64)
+    g = orc.grad(th, p["widths"], p["C"], p["X"], p["Y"])
+    rng = np.random.Generator(np.random.PCG64(3))
+    for _ in range(5):
+        e = rng.standard_normal(p["n"])
+        h = 1e-6
+        fd = (orc.fun(th + h * e, p["widths"], p["C"], p["X"], p["Y"]) - orc.fun(th - h * e, p["widths"], p["C"], p["X"], p["Y"])) / (2 * h)
+        assert fd == pytest.approx(g @ e, rel=1e-6)
