@@ -75,3 +75,55 @@ def test_wide4096_reduced_rows_and_properties_at_full_size():
     g = ctx.grad()
     assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL["fp32"]
     ctx.close()
+
+
+@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+def test_bench_configuration_at_20_percent(mode):
+    # the workload bench.py times by default: 784-2000-2000-2000-10, |S| = 12000 (fewer rows only for the gradient)
+    p = wl.make("mnist2000_20", l=12000)
+    ctx = make_ctx(p, mode)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    v = dev(p["v"])
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
+    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
+               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
+    ctx.close()
+
+
+def properties_at_any_size(p, mode):
+    """Checks that need no oracle run: symmetry, the I/C lower bound, and the block-diagonal product agreeing with
+    the full one on a direction supported on a single layer (then J_m v_m = J v)."""
+    import torch
+    ctx = make_ctx(p, mode)
+    ctx.set_subsample(dev(p["idx"]))
+    rng = np.random.Generator(np.random.PCG64(123))
+    n = p["n"]
+    u = rng.standard_normal(n, dtype=np.float32)
+    v = p["v"]
+    tol = 5 * TOL[mode]
+    for fn in (ctx.Gv, ctx.Gv_blockdiag):
+        Gu = fn(dev(u)).double()
+        Gv_ = fn(dev(v)).double()
+        du, dv = dev(u).double(), dev(v).double()
+        a, b = float(du @ Gv_), float(dv @ Gu)
+        assert abs(a - b) <= tol * max(abs(a), abs(b), float(Gv_.norm() * du.norm()) * 1e-3)
+        assert float(dv @ Gv_) >= float(dv @ dv) / p["C"] * (1 - 1e-3)
+        assert bool(torch.isfinite(Gv_).all())
+    offs = wl.layer_offsets(p["widths"])
+    for (w_off, b_off, end) in (offs[0], offs[-1], offs[len(offs) // 2]):
+        vm = np.zeros(n, dtype=np.float32)
+        vm[w_off:end] = v[w_off:end]
+        full = ctx.Gv(dev(vm))[w_off:end].double()
+        hat = ctx.Gv_blockdiag(dev(vm))[w_off:end].double()
+        assert float((full - hat).norm() / full.norm()) <= tol
+    ctx.close()
+
+
+@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+def test_wide4096_full_size_properties(mode):
+    properties_at_any_size(wl.make("wide4096", l=20000), mode)       # all 20000 subsample rows of the recipe
+
+
+def test_mnist2000_all_rows_properties():
+    properties_at_any_size(wl.make("mnist2000_100"), "tf32")          # |S| = l = 60000
