@@ -704,8 +704,7 @@ __global__ void timeout_probe_kernel(int* err, unsigned long long limit_ns) {
     mbar_init(&bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     const unsigned long long t0 = globaltimer();
-    bool done = false;
-    while (!(done = mbar_test_wait(&bar, 0))) {
+    while (!mbar_test_wait(&bar, 0)) {
       if (globaltimer() - t0 > limit_ns) { atomicCAS(err, 0, 9); break; }
     }
   }
