@@ -357,3 +357,39 @@ def newton_iteration(theta, widths, C, X, Y, idx, dprev, lam, sigma=1e-3, eta=1e
     report = dict(f_before=f0, f_after=f1, alpha=alpha, beta1=beta1, beta2=beta2, rho=rho, gTd=gTd, dGd=dGd,
                   cg_iters=len(its), backtracks=backtracks, lambda_next=lam_next)
     return theta + alpha * dnew, dnew, lam_next, report
+
+
+# --------------------------------------------------------------------------- stored Jacobian factors (Section 3.3.1 / 4.2)
+def jacobian_factors(theta, widths, Z):
+    """D^m[i, u, j] = d z^{L,i}_u / d s^{m,i}_j for every row i, m = 1..L (Eq. Jelement-store).
+
+    Backward recurrence of Section 3.3 for all rows at once: D^L = I (the output layer is linear),
+    D^{m-1} = (D^m W^{mT}) * sigma'(z^{m-1}) (Eq. communi-jaco followed by Eq. ztox-jaco).  Returns [D^1, ..., D^L].
+    """
+    layers = unpack(theta, widths)
+    L = len(layers)
+    rows, nL = Z[0].shape[0], widths[-1]
+    D = [None] * (L + 1)
+    D[L] = np.broadcast_to(np.eye(nL), (rows, nL, nL)).copy()
+    for m in range(L, 1, -1):
+        W, _ = layers[m - 1]
+        D[m - 1] = (D[m] @ W.T) * act_derivative(Z, m - 1, L)[:, None, :]
+    return D[1:]
+
+
+def Gv_blockdiag_stored(theta, widths, C, XS, v):
+    """Block-diagonal product the way Section 4.2 orders it: for block m, u_i = V^{mT} z^{m-1,i} + c^m
+    (the inner sum of Eq. direct-JV-cost), J_m v_m = D^m_i u_i, then D^{mT}_i (2 J_m v_m) (Eq. JTv), and the
+    outer product with z^{m-1,i} summed over rows (Eq. JTV-independent)."""
+    v = np.asarray(v, dtype=np.float64)
+    Z = forward(theta, widths, XS)
+    D = jacobian_factors(theta, widths, Z)
+    dirs = unpack(v, widths)
+    rows = Z[0].shape[0]
+    out = []
+    for m, (V, c) in enumerate(dirs, start=1):
+        U = Z[m - 1] @ V + c                                  # rows x n_m
+        P = np.einsum("iuj,ij->iu", D[m - 1], U)              # J_m v_m per row
+        Q = np.einsum("iuj,iu->ij", D[m - 1], 2.0 * P)        # D^T (B J_m v_m), B = 2I
+        out.append((Z[m - 1].T @ Q / rows, Q.sum(axis=0) / rows))
+    return v / C + pack(out)

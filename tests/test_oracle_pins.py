@@ -369,3 +369,21 @@ def test_scalar_output_with_plus_minus_one_labels():
         h = 1e-6
         fd = (orc.fun(th + h * e, p["widths"], p["C"], p["X"], p["Y"]) - orc.fun(th - h * e, p["widths"], p["C"], p["X"], p["Y"])) / (2 * h)
         assert fd == pytest.approx(g @ e, rel=1e-6)
+
+
+@pytest.mark.parametrize("widths", [(5, 4, 3, 2), (3, 5, 1), (2, 3, 3, 3, 2), (4, 3)])
+def test_stored_factor_form_of_the_blockdiag_product(widths):
+    # Section 3.3.1 / 4.2: the product through stored d z^L / d s^m equals the explicit-Jacobian definition,
+    # and the factors are the Jacobian's bias columns (Eq. xtow-jaco-bias: d z^L_u / d b^m_j = d z^L_u / d s^m_j)
+    p = tiny(widths=widths, seed=29)
+    XS = p["X"][p["idx"]]
+    v = p["v"].astype(np.float64)
+    a = orc.Gv_blockdiag_stored(p["theta"], p["widths"], p["C"], XS, v)
+    b = orc.Gv_blockdiag_definition(p["theta"], p["widths"], p["C"], XS, v)
+    assert np.linalg.norm(a - b) <= 1e-12 * np.linalg.norm(b)
+    Z = orc.forward(p["theta"], p["widths"], XS)
+    D = orc.jacobian_factors(p["theta"], p["widths"], Z)
+    J = orc.jacobian(p["theta"], p["widths"], XS[2])
+    for m, sl in enumerate(orc.block_slices(p["widths"]), start=1):
+        nm = p["widths"][m]
+        assert np.allclose(D[m - 1][2], J[:, sl.stop - nm: sl.stop], rtol=1e-12, atol=1e-15)
