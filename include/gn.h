@@ -102,6 +102,23 @@ int64_t gn_workspace_bytes(const gn_ctx* ctx);
 gn_status gn_set_batch_rows(gn_ctx* ctx, int64_t rows);
 
 /*
+ * gn_set_blockdiag_method - how gn_Gv_blockdiag (and block-diagonal CG) forms its product.
+ *   1  propagate: the perturbation of each layer block is pushed through the layers above it and pulled
+ *      back (R-operator form, L streams stacked along rows); no extra memory.
+ *   2  stored factors, the paper's own mechanism: d z^L / d s^m is computed once per (theta, subsample) by
+ *      the backward recurrence of Section 3.3 and kept (|S| n_L n_m floats per layer, Eq. Jelement-store);
+ *      a block product is then the two re-ordered contractions of Section 4.2 around it.  Needs L >= 2 and
+ *      n_L <= 16 (GN_EINVAL otherwise).  Fewer operations than 1 when n_L is small, more memory traffic.
+ *   0  choose (default): where 2 applies and its factors take at most 32 GB, the factors are built when a
+ *      solver may run 8 or more products (gn_cg_solve's max_iter, gn_newton_iter's cg_max) or on the
+ *      8th single product on one (theta, subsample), and every later product uses them; building them costs
+ *      about as much as five to six products of form 1 and saves about a third of each later product.
+ *      Otherwise 1.
+ * Both give the same product up to rounding.
+ */
+gn_status gn_set_blockdiag_method(gn_ctx* ctx, int method);
+
+/*
  * gn_set_theta - copy the model vector (Section 2.1 layout) into the context.  Activations stored
  * by an earlier gn_set_subsample become stale: products return GN_ESTATE until the subsample is
  * set again.

@@ -21,6 +21,7 @@ _SIGNATURES = {
     "gn_workspace_bytes": (_i64, [_vp]),
     "gn_kernel_launches": (_i64, [_vp]),
     "gn_set_batch_rows": (_i32, [_vp, _i64]),
+    "gn_set_blockdiag_method": (_i32, [_vp, _i32]),
     "gn_set_theta": (_i32, [_vp, _vp]),
     "gn_set_theta_host": (_i32, [_vp, _vp]),
     "gn_set_subsample": (_i32, [_vp, _vp, _i64]),
@@ -191,6 +192,10 @@ class GnContext:
     # ------------------------------------------------------------------ entry points
     def set_batch_rows(self, rows):
         self._check(self._lib.gn_set_batch_rows(self._h, int(rows)))
+
+    def set_blockdiag_method(self, method):
+        """0 choose, 1 propagate stacked streams, 2 stored Jacobian factors (Section 3.3.1)."""
+        self._check(self._lib.gn_set_blockdiag_method(self._h, int(method)))
 
     def set_theta(self, theta):
         import torch

@@ -18,7 +18,7 @@ struct FfmaParams {
   int vecA[2], vecB[2];
   float* D; long long ldd;
   const float* bias; int sigmoid;
-  const float* dsig; long long ld_dsig; int dsig_rows;
+  const float* dsig; long long ld_dsig; int dsig_rows, dsig_div;
   float alpha;
   const float* cin; long long ld_cin; float beta;
   int vec_epi;
@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(NT, 2) gemm_ffma_kernel(const FfmaParams p) {
   for (int i = 0; i < 8; ++i) {
     const int m = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
     if (m >= p.M) continue;
-    const long long zrow = p.dsig ? (long long)(m % p.dsig_rows) * p.ld_dsig : 0;
+    const long long zrow = p.dsig ? (long long)((m / p.dsig_div) % p.dsig_rows) * p.ld_dsig : 0;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const int n = n0 + h * 64 + tx * 4;
@@ -187,7 +187,7 @@ int launch_gemm_ffma(const GemmArgs& g, cudaStream_t st) {
   }
   p.D = g.D; p.ldd = g.ldd;
   p.bias = g.bias; p.sigmoid = g.sigmoid;
-  p.dsig = g.dsig; p.ld_dsig = g.ld_dsig; p.dsig_rows = g.dsig_rows > 0 ? g.dsig_rows : 1;
+  p.dsig = g.dsig; p.ld_dsig = g.ld_dsig; p.dsig_rows = g.dsig_rows > 0 ? g.dsig_rows : 1; p.dsig_div = g.dsig_div > 0 ? g.dsig_div : 1;
   p.alpha = g.alpha;
   p.cin = g.cin; p.ld_cin = g.ld_cin; p.beta = g.beta;
   p.vec_epi = aligned16(g.D) && (g.ldd % 4 == 0) && (!g.bias || aligned16(g.bias)) &&

@@ -41,7 +41,7 @@ struct Tf32Params {
   int a_3d, b_3d;       // MN-major operand fetched with one 3-D box per stage (needs a padded operand)
   float* D; long long ldd;
   const float* bias; int sigmoid;
-  const float* dsig; long long ld_dsig; int dsig_rows;
+  const float* dsig; long long ld_dsig; int dsig_rows, dsig_div;
   float alpha;
   const float* cin; long long ld_cin; float beta;
   int vec_epi;          // D, bias, dsig, cin all 16-byte aligned with leading dimensions % 4 == 0
@@ -290,7 +290,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant
       // moves 16 bytes per access and a row's 128 bytes are completed by consecutive accesses.
       const int m = m0 + quad * 32 + lane;
       const bool m_ok = m < p.M;
-      const float* zrow = p.dsig ? p.dsig + (long long)(m % p.dsig_rows) * p.ld_dsig : nullptr;
+      const float* zrow = p.dsig ? p.dsig + (long long)((m / p.dsig_div) % p.dsig_rows) * p.ld_dsig : nullptr;
       const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
       float* drow = p.D + (long long)m * p.ldd;
       for (int c = half; c < bn / 32; c += 2) {
@@ -612,7 +612,7 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
       {
         const int m = m0 + row;
         const bool m_ok = m < p.M;
-        const float* zrow = p.dsig ? p.dsig + (long long)(m % p.dsig_rows) * p.ld_dsig : nullptr;
+        const float* zrow = p.dsig ? p.dsig + (long long)((m / p.dsig_div) % p.dsig_rows) * p.ld_dsig : nullptr;
         const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
         float* drow = p.D + (long long)m * p.ldd;
         // whole tile: this warp's chunks are half, half + 2, ...; sliced tile: the pair's share of the
@@ -874,7 +874,7 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
   p.a_3d = (p.a_mn && g.mn_padded) ? 1 : 0; p.b_3d = (p.b_mn && g.mn_padded) ? 1 : 0;
   p.D = g.D; p.ldd = g.ldd;
   p.bias = g.bias; p.sigmoid = g.sigmoid;
-  p.dsig = g.dsig; p.ld_dsig = g.ld_dsig; p.dsig_rows = g.dsig_rows > 0 ? g.dsig_rows : 1;
+  p.dsig = g.dsig; p.ld_dsig = g.ld_dsig; p.dsig_rows = g.dsig_rows > 0 ? g.dsig_rows : 1; p.dsig_div = g.dsig_div > 0 ? g.dsig_div : 1;
   p.alpha = g.alpha;
   p.cin = g.cin; p.ld_cin = g.ld_cin; p.beta = g.beta;
   p.vec_epi = aligned16(g.D) && (g.ldd % 4 == 0) && (!g.bias || aligned16(g.bias)) &&

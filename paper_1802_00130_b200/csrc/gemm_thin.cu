@@ -19,7 +19,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 struct Epi {
   float* D; long long ldd;
   const float* bias; int sigmoid;
-  const float* dsig; long long ld_dsig; int dsig_rows;
+  const float* dsig; long long ld_dsig; int dsig_rows, dsig_div;
   float alpha;
   const float* cin; long long ld_cin; float beta;
 };
@@ -27,7 +27,7 @@ struct Epi {
 Epi make_epi(const GemmArgs& g) {
   Epi e;
   e.D = g.D; e.ldd = g.ldd; e.bias = g.bias; e.sigmoid = g.sigmoid;
-  e.dsig = g.dsig; e.ld_dsig = g.ld_dsig; e.dsig_rows = g.dsig_rows > 0 ? g.dsig_rows : 1;
+  e.dsig = g.dsig; e.ld_dsig = g.ld_dsig; e.dsig_rows = g.dsig_rows > 0 ? g.dsig_rows : 1; e.dsig_div = g.dsig_div > 0 ? g.dsig_div : 1;
   e.alpha = g.alpha; e.cin = g.cin; e.ld_cin = g.ld_cin; e.beta = g.beta;
   return e;
 }
@@ -35,7 +35,7 @@ Epi make_epi(const GemmArgs& g) {
 __device__ __forceinline__ float apply_epi(const Epi& e, float x, int m, int n) {
   if (e.bias) x += __ldg(e.bias + n);
   if (e.sigmoid) x = 1.f / (1.f + expf(-x));
-  if (e.dsig) { const float z = __ldg(e.dsig + (long long)(m % e.dsig_rows) * e.ld_dsig + n); x *= z * (1.f - z); }
+  if (e.dsig) { const float z = __ldg(e.dsig + (long long)((m / e.dsig_div) % e.dsig_rows) * e.ld_dsig + n); x *= z * (1.f - z); }
   x *= e.alpha;
   if (e.cin) x = fmaf(e.beta, __ldg(e.cin + (long long)m * e.ld_cin + n), x);
   return x;
@@ -233,7 +233,7 @@ __global__ void __launch_bounds__(128, 4) gemm_thin_k_kernel(const ThinKParams p
       for (int i = 0; i < RG; ++i) {
         const int m = mb + r0 + i;
         const bool ok = r0 + i < cnt;
-        z[i] = (p.e.dsig && ok) ? __ldg(reinterpret_cast<const float4*>(p.e.dsig + (long long)(m % p.e.dsig_rows) * p.e.ld_dsig + n))
+        z[i] = (p.e.dsig && ok) ? __ldg(reinterpret_cast<const float4*>(p.e.dsig + (long long)((m / p.e.dsig_div) % p.e.dsig_rows) * p.e.ld_dsig + n))
                                 : make_float4(0.f, 0.f, 0.f, 0.f);
       }
 #pragma unroll

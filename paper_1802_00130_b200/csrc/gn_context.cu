@@ -33,6 +33,13 @@ struct gn_ctx {
   std::vector<float*> Z;    // Z[0] = X_S, Z[m] = [nS][n_m]
   std::vector<float*> RZ;   // RZ[m] = [m * nS][n_m]: forward directional derivatives (stacked streams)
   std::vector<float*> DS;   // DS[m] = [m * nS][n_m]: backward quantities d(.)/d s^m
+  // stored Jacobian factors d z^L / d s^m on the subsample (block-diagonal product, Section 3.3.1)
+  std::vector<float*> DF;   // DF[m] = [nS * n_L][n_m], m = 1..L-1
+  int64_t capF = 0;         // rows of S the factor buffers hold
+  bool factors_valid = false;
+  int bd_method = 0;        // 0 choose, 1 propagate L stacked streams, 2 stored factors
+  int bd_expect = 0;        // products the running solver may still ask for (0 outside a solver)
+  int bd_count = 0;         // propagate-form products since the factors were last invalidated
   // row-batch workspace of f / grad
   int64_t capB = 0;
   std::vector<float*> Zb, Db;
@@ -336,6 +343,83 @@ gn_status product_blockdiag(gn_ctx* c, const float* v, float* out, float coef) {
   return check_launch(c, "block-diagonal G v");
 }
 
+// ---- block-diagonal product through stored factors (the paper's own mechanism, Sections 3.3.1 and 4.2)
+bool stored_factors_applicable(const gn_ctx* c) {
+  if (c->L < 2 || c->w[c->L] > 16) return false;
+  if ((int64_t)c->w[c->L] * c->nS > 65535LL * 128) return false;
+  int64_t bytes = 0;
+  for (int m = 1; m < c->L; ++m) bytes += (int64_t)c->nS * c->w[c->L] * c->w[m] * 4;
+  return bytes <= 32LL * 1000 * 1000 * 1000;
+}
+
+// D^{L-1} from the linear output layer, then D^{m-1} = (D^m W^{mT}) * sigma'(z^{m-1}) on |S| n_L rows
+// (Eqs. communi-jaco, ztox-jaco, Jelement-store).  Done once per (theta, S).
+gn_status ensure_factors(gn_ctx* c) {
+  if (c->factors_valid) return GN_OK;
+  const int L = c->L, nL = c->w[L];
+  const int64_t nS = c->nS;
+  if (nS > c->capF) {
+    GN_TRY(sync(c, "factors"));
+    for (int m = 1; m < L; ++m) dev_free(c, c->DF[m], c->capF * nL * c->w[m]);
+    c->capF = 0;
+    for (int m = 1; m < L; ++m) GN_TRY(dev_alloc(c, &c->DF[m], nS * nL * c->w[m]));
+    c->capF = nS;
+  }
+  c->launches += launch_factor_last(Wm(c, c->theta, L), c->Z[L - 1], nS, nL, c->w[L - 1], c->DF[L - 1], c->st);
+  for (int m = L - 1; m >= 2; --m) {
+    GemmArgs g;
+    g.M = (int)(nS * nL); g.N = c->w[m - 1];
+    g.A1 = c->DF[m]; g.lda1 = c->w[m]; g.a_kmajor = true;
+    g.B1 = Wm(c, c->theta, m); g.ldb1 = c->w[m - 1]; g.b_kmajor = false;
+    g.K1 = c->w[m];
+    g.dsig = c->Z[m - 1]; g.ld_dsig = c->w[m - 1]; g.dsig_rows = (int)nS; g.dsig_div = nL;
+    g.D = c->DF[m - 1]; g.ldd = c->w[m - 1];
+    g.mn_padded = true;
+    run_gemm(c, g);
+  }
+  c->factors_valid = true;
+  return check_launch(c, "Jacobian factors");
+}
+
+gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float coef) {
+  GN_TRY(ensure_factors(c));
+  const int L = c->L, nL = c->w[L];
+  const int64_t nS = c->nS;
+  const float inv = (float)(1.0 / (double)nS);
+  for (int m = 1; m <= L; ++m) {
+    // u_i = V^{mT} z^{m-1,i} + c^m for every row (the inner sum of Eq. direct-JV-cost); at m = L, D = I and B = 2I
+    GemmArgs g;
+    g.M = (int)nS; g.N = c->w[m];
+    g.A1 = c->Z[m - 1]; g.lda1 = c->w[m - 1]; g.B1 = Wm(c, v, m); g.ldb1 = c->w[m - 1]; g.K1 = c->w[m - 1];
+    g.bias = bm(c, v, m);
+    if (m == L) g.alpha = 2.f;
+    g.D = c->RZ[m]; g.ldd = c->w[m];
+    run_gemm(c, g);
+    const float* ds = c->RZ[m];
+    if (m < L) {
+      c->launches += launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], c->DS[m], c->st);
+      ds = c->DS[m];
+    }
+    GN_TRY(weight_block(c, m, ds, c->Z[m - 1], nS, inv, v, coef, out));
+  }
+  return check_launch(c, "block-diagonal G v (stored factors)");
+}
+
+// Choosing between the two forms when the caller has not: building the factors costs about as much as
+// five to six propagate-form products and saves about a third of each later one, so they are built when
+// a solver announces at least kFactorBreakEven products, or once that many single products have been
+// asked for on the same (theta, S), counting the one at hand; after that every product uses them.
+constexpr int kFactorBreakEven = 8;
+
+gn_status product_blockdiag_any(gn_ctx* c, const float* v, float* out, float coef) {
+  bool stored = c->bd_method == 2;
+  if (c->bd_method == 0 && stored_factors_applicable(c))
+    stored = c->factors_valid || c->bd_expect >= kFactorBreakEven || c->bd_count + 1 >= kFactorBreakEven;
+  if (stored && c->L >= 2 && c->w[c->L] <= 16) return product_blockdiag_stored(c, v, out, coef);
+  ++c->bd_count;
+  return product_blockdiag(c, v, out, coef);
+}
+
 gn_status ensure_batch(gn_ctx* c) {
   const int64_t rows = c->batch_rows < c->l ? c->batch_rows : c->l;
   if (rows <= c->capB) return GN_OK;
@@ -470,6 +554,7 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
   }
   c->n = off;
   c->Z.assign(L + 1, nullptr); c->RZ.assign(L + 1, nullptr); c->DS.assign(L + 1, nullptr);
+  c->DF.assign(L + 1, nullptr);
   c->Zb.assign(L + 1, nullptr); c->Db.assign(L + 1, nullptr);
   gn_status s = GN_OK;
   do {
@@ -522,6 +607,15 @@ gn_status gn_set_batch_rows(gn_ctx* c, int64_t rows) {
   return GN_OK;
 }
 
+gn_status gn_set_blockdiag_method(gn_ctx* c, int method) {
+  if (!c) return GN_EINVAL;
+  if (method < 0 || method > 2) return fail(c, GN_EINVAL, "method must be 0 (choose), 1 (propagate) or 2 (stored factors)");
+  if (method == 2 && (c->L < 2 || c->w[c->L] > 16))
+    return fail(c, GN_EINVAL, "stored factors need at least two layers and n_L <= 16");
+  c->bd_method = method;
+  return GN_OK;
+}
+
 gn_status gn_set_theta(gn_ctx* c, const float* d_theta) {
   if (!c) return GN_EINVAL;
   if (!d_theta) return fail(c, GN_EINVAL, "theta is NULL");
@@ -548,6 +642,8 @@ static gn_status set_subsample_impl(gn_ctx* c, const int32_t* idx, int64_t nS, c
   if (!c->have_theta) return fail(c, GN_ESTATE, "theta has not been set");
   if ((int64_t)c->L * nS > 65535LL * 128) return fail(c, GN_EINVAL, "L * |S| exceeds 8 388 480 rows");
   c->have_sub = false;
+  c->factors_valid = false;
+  c->bd_count = 0;
   if (nS > c->capS) {
     GN_TRY(sync(c, "set_subsample"));
     dev_free(c, c->idx, c->capS);
@@ -619,7 +715,7 @@ gn_status gn_Gv_blockdiag(gn_ctx* c, const float* d_v, float* d_out) {
   if (!d_v || !d_out) return fail(c, GN_EINVAL, "v / out is NULL");
   if (d_v == d_out) return fail(c, GN_EINVAL, "v and out must not overlap");
   GN_TRY(need_product_state(c));
-  return product_blockdiag(c, d_v, d_out, (float)(1.0 / c->C));
+  return product_blockdiag_any(c, d_v, d_out, (float)(1.0 / c->C));
 }
 
 static gn_status product_host(gn_ctx* c, const float* h_v, float* h_out, bool blockdiag) {
@@ -629,7 +725,7 @@ static gn_status product_host(gn_ctx* c, const float* h_v, float* h_out, bool bl
   GN_TRY(ensure_tmp(c));
   GN_CUDA(c, cudaMemcpyAsync(c->tmp_a, h_v, c->n * sizeof(float), cudaMemcpyHostToDevice, c->st));
   const float coef = (float)(1.0 / c->C);
-  GN_TRY(blockdiag ? product_blockdiag(c, c->tmp_a, c->tmp_b, coef) : product_full(c, c->tmp_a, c->tmp_b, coef));
+  GN_TRY(blockdiag ? product_blockdiag_any(c, c->tmp_a, c->tmp_b, coef) : product_full(c, c->tmp_a, c->tmp_b, coef));
   GN_CUDA(c, cudaMemcpyAsync(h_out, c->tmp_b, c->n * sizeof(float), cudaMemcpyDeviceToHost, c->st));
   return sync(c, "product_host");
 }
@@ -658,8 +754,10 @@ gn_status gn_cg_solve(gn_ctx* c, const float* d_g, double lambda, int blockdiag,
   GN_TRY(sync(c, "cg init"));
   if (resnorm_host) resnorm_host[0] = sqrt(c->hscal[2]);
   int it = 0;
+  c->bd_expect = blockdiag ? max_iter : 0;
+  struct Reset { int* p; ~Reset() { *p = 0; } } reset_expect{&c->bd_expect};
   while (it < max_iter && c->hscal[3] > 0.5) {
-    GN_TRY(blockdiag ? product_blockdiag(c, c->cg_p, c->cg_q, coef) : product_full(c, c->cg_p, c->cg_q, coef));
+    GN_TRY(blockdiag ? product_blockdiag_any(c, c->cg_p, c->cg_q, coef) : product_full(c, c->cg_p, c->cg_q, coef));
     c->launches += launch_cg_dot(c->cg_p, c->cg_q, ch, nc, c->partial, c->st);
     c->launches += launch_cg_scalars(1, c->partial, ch, nc, c->segs, n_seg, tol, out2, c->st);
     c->launches += launch_cg_update(c->cg_p, c->cg_q, d_d, c->cg_r, ch, nc, c->segs, c->partial, c->st);

@@ -10,7 +10,7 @@ namespace gn {
 //   acc[m][n] = sum_k A1(m,k) B1(k,n)  (+ sum_k A2(m,k) B2(k,n) when A2 != nullptr)
 //   t = acc + bias[n]                   (bias != nullptr)
 //   t = 1 / (1 + exp(-t))               (sigmoid)
-//   t = t * zc (1 - zc)                 (dsig != nullptr; zc = dsig[(m % dsig_rows) * ld_dsig + n])
+//   t = t * zc (1 - zc)                 (dsig != nullptr; zc = dsig[((m / dsig_div) % dsig_rows) * ld_dsig + n])
 //   t = alpha * t
 //   t = t + beta * cin[m * ld_cin + n]  (cin != nullptr)
 //   D[m * ldd + n] = t
@@ -28,7 +28,7 @@ struct GemmArgs {
   float* D = nullptr; int64_t ldd = 0;
   const float* bias = nullptr;
   bool sigmoid = false;
-  const float* dsig = nullptr; int64_t ld_dsig = 0; int dsig_rows = 1;
+  const float* dsig = nullptr; int64_t ld_dsig = 0; int dsig_rows = 1; int dsig_div = 1;
   float alpha = 1.f;
   const float* cin = nullptr; int64_t ld_cin = 0; float beta = 0.f;
 };
@@ -85,6 +85,12 @@ int launch_axpby(int64_t n, float a, const float* x, float b, const float* y, fl
 
 // Transposed copy dst[c][r] = src[r][c] (src rows x cols).
 int launch_transpose(const float* src, int rows, int cols, float* dst, cudaStream_t st);
+
+// Stored Jacobian factors (d z^L / d s^m per sample, Section 3.3.1).  D is [rows * nL][n] with row i * nL + u.
+// factor_last: D[(i, u)][t] = WL[u * n + t] * z (1 - z), z = Zprev[i * n + t]   (layer L-1 from the linear output layer)
+int launch_factor_last(const float* WL, const float* Zprev, int64_t rows, int nL, int n, float* D, cudaStream_t st);
+// factor_apply: p_u = sum_j D[(i,u)][j] U[i][j];  Q[i][j] = 2 sum_u D[(i,u)][j] p_u   (Eqs. direct-JV-cost, JTv; B = 2I)
+int launch_factor_apply(const float* D, const float* U, int64_t rows, int nL, int n, float* Q, cudaStream_t st);
 
 // ---- conjugate gradient ------------------------------------------------------------------------
 // The n coordinates are cut into chunks, each inside one segment (one segment for the full system,

@@ -166,6 +166,62 @@ __global__ void __launch_bounds__(256) axpby_kernel(long long n, float a, const 
     out[i] = fmaf(a, x[i], b * y[i]);
 }
 
+// ---------------------------------------------------------------------------------- stored Jacobian factors
+// D[(i, u)][t] = WL[u][t] * z (1 - z): one block per sample row i, threads over t (16-byte accesses when n % 4 == 0).
+__global__ void __launch_bounds__(256) factor_last_kernel(const float* __restrict__ WL, const float* __restrict__ Zprev,
+                                                          int nL, int n, float* __restrict__ D) {
+  const long long i = blockIdx.x;
+  const float* z = Zprev + i * n;
+  float* d = D + i * nL * n;
+  for (int t = threadIdx.x; t < n; t += 256) {
+    const float zz = __ldg(z + t);
+    const float ds = zz * (1.f - zz);
+    for (int u = 0; u < nL; ++u) d[(long long)u * n + t] = __ldg(WL + (long long)u * n + t) * ds;
+  }
+}
+
+// One block per sample row: pass 1 forms p_u = D_i[u][:] . U_i (block reduction per u), pass 2 re-reads D_i
+// (just read, so from cache) and writes Q_i[j] = 2 sum_u D_i[u][j] p_u.  NLMAX bounds n_L.
+template <int NLMAX>
+__global__ void __launch_bounds__(256) factor_apply_kernel(const float* __restrict__ D, const float* __restrict__ U,
+                                                           int nL, int n, float* __restrict__ Q) {
+  __shared__ float red[8][NLMAX];
+  __shared__ float pu[NLMAX];
+  const long long i = blockIdx.x;
+  const float* d = D + i * nL * n;
+  const float* u_row = U + i * n;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  float acc[NLMAX];
+#pragma unroll
+  for (int u = 0; u < NLMAX; ++u) acc[u] = 0.f;
+  for (int j = threadIdx.x; j < n; j += 256) {
+    const float uj = __ldg(u_row + j);
+#pragma unroll
+    for (int u = 0; u < NLMAX; ++u)
+      if (u < nL) acc[u] = fmaf(__ldg(d + (long long)u * n + j), uj, acc[u]);
+  }
+#pragma unroll
+  for (int u = 0; u < NLMAX; ++u) {
+    const float s = warp_sum(acc[u]);
+    if (lane == 0) red[w][u] = s;
+  }
+  __syncthreads();
+  if (threadIdx.x < NLMAX) {
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x];
+    pu[threadIdx.x] = 2.f * s;                              // B = 2I
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < n; j += 256) {
+    float q = 0.f;
+#pragma unroll
+    for (int u = 0; u < NLMAX; ++u)
+      if (u < nL) q = fmaf(__ldg(d + (long long)u * n + j), pu[u], q);
+    Q[i * n + j] = q;
+  }
+}
+
 // ---------------------------------------------------------------------------------- transpose
 __global__ void __launch_bounds__(256) transpose_kernel(const float* __restrict__ src, int rows, int cols,
                                                         float* __restrict__ dst) {
@@ -338,6 +394,80 @@ int launch_loss_delta(const float* Z, const float* Y, int64_t count, float* delt
 
 int launch_sum_partials(const double* partial, int count, double* out, bool accumulate, cudaStream_t st) {
   sum_partials_kernel<<<1, 256, 0, st>>>(partial, count, out, accumulate ? 1 : 0);
+  return 1;
+}
+
+// Register-resident form for rows of at most 1024 * STRIPS floats (n % 4 == 0): every thread keeps its
+// n_L x 4 x STRIPS slice of D_i in registers between the two passes, so D is read exactly once.
+template <int NLMAX, int STRIPS>
+__global__ void __launch_bounds__(256) factor_apply_reg_kernel(const float* __restrict__ D, const float* __restrict__ U,
+                                                               int nL, int n, float* __restrict__ Q) {
+  __shared__ float red[8][NLMAX];
+  __shared__ float pu[NLMAX];
+  const long long i = blockIdx.x;
+  const float* d = D + i * nL * n;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  float4 dv[STRIPS][NLMAX];
+  float acc[NLMAX];
+#pragma unroll
+  for (int u = 0; u < NLMAX; ++u) acc[u] = 0.f;
+#pragma unroll
+  for (int s = 0; s < STRIPS; ++s) {
+    const int j = (s * 256 + threadIdx.x) * 4;
+    const bool ok = j < n;
+#pragma unroll
+    for (int u = 0; u < NLMAX; ++u)
+      dv[s][u] = (ok && u < nL) ? __ldg(reinterpret_cast<const float4*>(d + (long long)u * n + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4 uj = ok ? __ldg(reinterpret_cast<const float4*>(U + i * n + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < NLMAX; ++u)
+      acc[u] += dv[s][u].x * uj.x + dv[s][u].y * uj.y + dv[s][u].z * uj.z + dv[s][u].w * uj.w;
+  }
+#pragma unroll
+  for (int u = 0; u < NLMAX; ++u) {
+    const float s = warp_sum(acc[u]);
+    if (lane == 0) red[w][u] = s;
+  }
+  __syncthreads();
+  if (threadIdx.x < NLMAX) {
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x];
+    pu[threadIdx.x] = 2.f * s;                              // B = 2I
+  }
+  __syncthreads();
+#pragma unroll
+  for (int s = 0; s < STRIPS; ++s) {
+    const int j = (s * 256 + threadIdx.x) * 4;
+    if (j < n) {
+      float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < NLMAX; ++u) {
+        const float pv = pu[u];
+        q.x = fmaf(dv[s][u].x, pv, q.x); q.y = fmaf(dv[s][u].y, pv, q.y);
+        q.z = fmaf(dv[s][u].z, pv, q.z); q.w = fmaf(dv[s][u].w, pv, q.w);
+      }
+      *reinterpret_cast<float4*>(Q + i * n + j) = q;
+    }
+  }
+}
+
+int launch_factor_last(const float* WL, const float* Zprev, int64_t rows, int nL, int n, float* D, cudaStream_t st) {
+  factor_last_kernel<<<(unsigned)rows, 256, 0, st>>>(WL, Zprev, nL, n, D);
+  return 1;
+}
+
+int launch_factor_apply(const float* D, const float* U, int64_t rows, int nL, int n, float* Q, cudaStream_t st) {
+  const bool vec = (n % 4 == 0) && ((reinterpret_cast<uintptr_t>(D) & 15) == 0) && ((reinterpret_cast<uintptr_t>(U) & 15) == 0) &&
+                   ((reinterpret_cast<uintptr_t>(Q) & 15) == 0);
+  if (vec && n <= 1024 && nL <= 4)  { factor_apply_reg_kernel<4, 1><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
+  if (vec && n <= 1024 && nL <= 10) { factor_apply_reg_kernel<10, 1><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
+  if (vec && n <= 2048 && nL <= 4)  { factor_apply_reg_kernel<4, 2><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
+  if (vec && n <= 2048 && nL <= 10) { factor_apply_reg_kernel<10, 2><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
+  if (vec && n <= 1024 && nL <= 16) { factor_apply_reg_kernel<16, 1><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
+  if (nL <= 4) factor_apply_kernel<4><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q);
+  else if (nL <= 10) factor_apply_kernel<10><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q);
+  else factor_apply_kernel<16><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q);
   return 1;
 }
 

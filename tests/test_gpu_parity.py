@@ -228,3 +228,76 @@ def test_a_timed_out_device_wait_is_reported_and_the_context_survives():
     g, f = ctx.grad(with_f=True)                     # a synchronising call reports no stale error
     assert np.isfinite(f)
     ctx.close()
+
+
+@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+@pytest.mark.parametrize("name", ["tiny", "ragged", "mid", "binary300"])
+def test_blockdiag_methods_agree_with_the_checker_and_each_other(name, mode):
+    import paper_1802_00130_b200 as gn
+    p = wl.make(name)
+    ctx = make_ctx(p, mode)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    ref = orc.Gv_blockdiag_stored(p["theta"], p["widths"], p["C"], XS, p["v"])
+    outs = []
+    for method in (1, 2, 0):
+        ctx.set_blockdiag_method(method)
+        outs.append(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy())
+        assert rel(outs[-1], ref) <= TOL[mode], method
+    assert rel(outs[0], outs[1]) <= 2 * TOL[mode]
+    # a new subsample invalidates the stored factors
+    ctx.set_blockdiag_method(2)
+    idx2 = np.ascontiguousarray(p["idx"][::-1][: max(1, p["nS"] // 2)])
+    ctx.set_subsample(dev(idx2))
+    ref2 = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], p["X"][idx2], p["v"])
+    assert rel(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy(), ref2) <= TOL[mode]
+    # block CG goes through the same product
+    g = orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]).astype(np.float32)
+    d2, _, _ = ctx.cg_solve(dev(g), 1.0, blockdiag=True, max_iter=5, tol=0.0)
+    ctx.set_blockdiag_method(1)
+    d1, _, _ = ctx.cg_solve(dev(g), 1.0, blockdiag=True, max_iter=5, tol=0.0)
+    assert rel(d2.cpu().numpy(), d1.cpu().numpy()) <= 20 * TOL[mode]
+    ctx.close()
+
+
+def test_stored_factors_need_a_small_output_layer():
+    import paper_1802_00130_b200 as gn
+    p = wl.make("single")                      # one layer: nothing to store
+    ctx = make_ctx(p)
+    with pytest.raises(gn.GnError) as e:
+        ctx.set_blockdiag_method(2)
+    assert e.value.status == 1
+    with pytest.raises(gn.GnError):
+        ctx.set_blockdiag_method(3)
+    ctx.close()
+
+
+def test_the_default_method_builds_factors_only_when_they_pay():
+    """Factors are not built for a few single products, are built at the eighth on one subsample, and at once by a
+    solver that may run eight or more steps."""
+    p = wl.make("mid")
+    ctx = make_ctx(p, "tf32")
+    ctx.set_subsample(dev(p["idx"]))
+    ref = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], p["X"][p["idx"]], p["v"])
+    out = ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy()          # first product: the product's own scratch
+    base = ctx.workspace_bytes
+    for k in range(6):
+        out = ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy()
+        assert ctx.workspace_bytes == base, k
+    assert rel(out, ref) <= TOL["tf32"]
+    out8 = ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy()          # eighth product: factors built and used
+    grown = ctx.workspace_bytes
+    factor_bytes = sum(p["nS"] * p["widths"][-1] * n for n in p["widths"][1:-1]) * 4
+    assert grown - base >= factor_bytes
+    assert rel(out8, ref) <= TOL["tf32"]
+    ctx.close()
+
+    ctx = make_ctx(p, "tf32")
+    ctx.set_subsample(dev(p["idx"]))
+    g = orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]).astype(np.float32)
+    ctx.cg_solve(dev(g), 1.0, blockdiag=True, max_iter=3, tol=0.0)
+    short = ctx.workspace_bytes
+    ctx.cg_solve(dev(g), 1.0, blockdiag=True, max_iter=8, tol=0.0)
+    assert ctx.workspace_bytes - short >= factor_bytes
+    ctx.cg_solve(dev(g), 1.0, blockdiag=False, max_iter=8, tol=0.0)
+    ctx.close()
