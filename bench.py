@@ -33,7 +33,7 @@ UNIT = "matvec/s"
 FP32_LANES_PER_SM, SMS = 128, 148
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant GEMM kernel, averaged over the
 # launches of one step (profiles/tf32_path_mnist2000_20_launches.md); unknown (None) for other cases
-TRAFFIC = {("tf32", "mnist2000_20"): {"bytes_per_launch": 318.5e6, "kernel": "gemm_tf32_2cta_kernel",
+TRAFFIC = {("tf32", "mnist2000_20"): {"bytes_per_launch": 290.2e6, "kernel": "gemm_tf32_2cta_kernel",
                                       "source": "profiles/tf32_path_mnist2000_20_launches.md"}}
 
 
@@ -240,22 +240,36 @@ def run_ours(args):
     out = torch.empty_like(v)
     breakdown = {}
     macs = mac_counts(p["widths"])
-    for name, fn, mac_exec, mac_alg in (("Gv", ctx.Gv, macs["full"], macs["full"]),
-                                        ("Gv_blockdiag", ctx.Gv_blockdiag, macs["block_executed"], macs["block_paper"])):
-        for _ in range(3):
-            fn(v, out=out)
-        torch.cuda.synchronize()
+    def timed(fn, reps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = args.product_reps
         a.record()
         for _ in range(reps):
             fn(v, out=out)
         b.record()
         torch.cuda.synchronize()
-        t = a.elapsed_time(b) * 1e-3 / reps
+        return a.elapsed_time(b) * 1e-3 / reps
+
+    stored_ok = len(p["widths"]) >= 3 and p["widths"][-1] <= 16
+    legs = [("Gv", ctx.Gv, 0, macs["full"], macs["full"]),
+            ("Gv_blockdiag_propagate", ctx.Gv_blockdiag, 1, macs["block_executed"], macs["block_paper"])]
+    if stored_ok:
+        legs.append(("Gv_blockdiag_stored", ctx.Gv_blockdiag, 2, macs["block_paper"], macs["block_paper"]))
+    for name, fn, method, mac_exec, mac_alg in legs:
+        ctx.set_blockdiag_method(method)
+        if method == 2:                       # the once-per-(theta, S) cost of the factors: first product - later ones
+            ctx.set_subsample(idx_dev[0])
+            torch.cuda.synchronize()
+            first = timed(fn, 1)
+        for _ in range(3):
+            fn(v, out=out)
+        torch.cuda.synchronize()
+        t = timed(fn, args.product_reps)
         breakdown[name] = {"per_s": 1.0 / t, "ms": 1e3 * t,
                            "executed_tflops": 2.0 * mac_exec * p["nS"] / t / 1e12,
                            "algorithmic_tflops": 2.0 * mac_alg * p["nS"] / t / 1e12}
+        if method == 2:
+            breakdown[name]["factor_setup_ms"] = 1e3 * max(first - t, 0.0)
+    ctx.set_blockdiag_method(0)
 
     # ---- one Newton iteration of Algorithm 3 (block-diagonal CG capped at n_cg steps), for context
     th_n, dir_n = theta.clone(), torch.zeros_like(theta)
@@ -311,7 +325,8 @@ def run_ours(args):
     achieved = kern["flop"] / (kern["ms"] * 1e-3) / 1e12 if kern["ms"] > 0 else None
     roof.update({"kernel": "gemm_tf32_2cta_kernel + gemm_tf32_kernel" if args.mode == "tf32" else "gemm_ffma_kernel",
                  "achieved": achieved, "frac": achieved / peak if achieved else None,
-                 "traffic": TRAFFIC.get((args.mode, args.workload)),
+                 "traffic": (TRAFFIC.get((args.mode, args.workload)) or {}).get("bytes_per_launch"),
+                 "traffic_note": TRAFFIC.get((args.mode, args.workload)),
                  "launches": kern["launches"], "avg_launch_us": 1e3 * kern["ms"] / max(1, kern["launches"]),
                  "share_of_step": kern["ms"] / ms if ms > 0 else None,
                  "other_contractions": {name: {"ms": prof[name]["ms"], "launches": prof[name]["launches"]}

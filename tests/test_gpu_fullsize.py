@@ -17,8 +17,10 @@ def test_mnist300_products_and_gradient_on_all_rows(mode):
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
     assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
-    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
-               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
+    ref_b = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])
+    for method in (1, 2):                  # propagate form, then the stored Jacobian factors
+        ctx.set_blockdiag_method(method)
+        assert rel(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b) <= TOL[mode], method
     g, f = ctx.grad(with_f=True)
     assert abs(f - orc.fun(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL[mode] * abs(f)
     assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL[mode]
@@ -58,8 +60,10 @@ def test_mnist2000_headline_config_at_5_percent(mode):
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
     assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
-    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
-               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
+    ref_b = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])
+    for method in (1, 2):                  # propagate form, then the stored Jacobian factors
+        ctx.set_blockdiag_method(method)
+        assert rel(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b) <= TOL[mode], method
     ctx.close()
 
 
@@ -86,17 +90,20 @@ def test_bench_configuration_at_20_percent(mode):
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
     assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
-    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
-               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
+    ref_b = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])
+    for method in (1, 2):                  # propagate form, then the stored Jacobian factors
+        ctx.set_blockdiag_method(method)
+        assert rel(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b) <= TOL[mode], method
     ctx.close()
 
 
-def properties_at_any_size(p, mode):
+def properties_at_any_size(p, mode, method=1):
     """Checks that need no oracle run: symmetry, the I/C lower bound, and the block-diagonal product agreeing with
     the full one on a direction supported on a single layer (then J_m v_m = J v)."""
     import torch
     ctx = make_ctx(p, mode)
     ctx.set_subsample(dev(p["idx"]))
+    ctx.set_blockdiag_method(method)
     rng = np.random.Generator(np.random.PCG64(123))
     n = p["n"]
     u = rng.standard_normal(n, dtype=np.float32)
@@ -125,5 +132,6 @@ def test_wide4096_full_size_properties(mode):
     properties_at_any_size(wl.make("wide4096", l=20000), mode)       # all 20000 subsample rows of the recipe
 
 
-def test_mnist2000_all_rows_properties():
-    properties_at_any_size(wl.make("mnist2000_100"), "tf32")          # |S| = l = 60000
+@pytest.mark.parametrize("method", [1, 2])
+def test_mnist2000_all_rows_properties(method):
+    properties_at_any_size(wl.make("mnist2000_100"), "tf32", method)  # |S| = l = 60000; method 2 keeps 14.4 GB of factors
