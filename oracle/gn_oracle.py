@@ -28,7 +28,15 @@ biases are part of theta and are regularised (Section 3.2.1 sums (b_j)^2 into
 the regulariser); the loss has no 1/2 so B^i = 2I (Section 3.1); f and grad f
 average over all l rows, G^S over |S|; the Jacobian's backward pass starts from
 the identity (Eq. zLindependent) while the gradient's starts from 2(z^L - y)
-(Section 3.4); the block-diagonal blocks are the layers (split 1-1-...-1).
+(Section 3.4); the block-diagonal blocks are the layers (split 1-1-...-1)
+unless a split structure is given, in which case the neurons of layer m are
+cut into split[m] contiguous groups of near-equal size (group g holds neurons
+floor(g n_m / s_m) .. floor((g+1) n_m / s_m) - 1; the paper's example and
+Table 2 give only the group counts), a partition is the weights between one
+group of layer m-1 and one group of layer m, and b^m_j goes to the partition of
+the first group of layer m-1 (Section 3.1); the CG termination rule of
+Section 4.4 counts lock-step iterations: the solve ends once CG_min steps are
+done and the stated share of partitions have met their own stop rule.
 """
 from __future__ import annotations
 
@@ -302,6 +310,129 @@ def cg_solve(theta, widths, C, XS, g, lam, blockdiag, max_iter, tol):
         return cg(lambda p: Gv_blockdiag(theta, widths, C, XS, p), g, lam, max_iter, tol,
                   segments=block_slices(widths))
     return cg(lambda p: Gv(theta, widths, C, XS, p), g, lam, max_iter, tol)
+
+
+# --------------------------------------------------------------------------- variable partition (Section 3.1)
+def group_bounds(n, s):
+    """Boundaries of the s contiguous neuron groups of a layer with n neurons."""
+    return [(g * n) // s for g in range(s + 1)]
+
+
+def partition_labels(widths, split):
+    """Partition id of every coordinate of theta for a split structure split[0..L] (Section 3.1).
+
+    Partitions are numbered layer by layer, and inside layer m by (group of layer m-1, group of layer m) with
+    the layer-m group running fastest.  w^m_{tj} belongs to (group of t, group of j); b^m_j to (first group of
+    layer m-1, group of j).  Returns (labels, P).
+    """
+    assert len(split) == len(widths) and all(1 <= s <= n for s, n in zip(split, widths))
+    labels = np.empty(num_params(widths), dtype=np.int64)
+    off, base = 0, 0
+    for m in range(1, len(widths)):
+        a, b = widths[m - 1], widths[m]
+        ga = np.searchsorted(group_bounds(a, split[m - 1]), np.arange(a), side="right") - 1   # group of neuron t
+        gb = np.searchsorted(group_bounds(b, split[m]), np.arange(b), side="right") - 1       # group of neuron j
+        lab_w = base + ga[None, :] * split[m] + gb[:, None]          # [j, t], stored with t running fastest
+        labels[off:off + a * b] = lab_w.reshape(-1)
+        off += a * b
+        labels[off:off + b] = base + gb                              # first group of layer m-1
+        off += b
+        base += split[m - 1] * split[m]
+    return labels, base
+
+
+def partition_indices(widths, split):
+    """Index arrays of the P partitions, in partition order."""
+    labels, P = partition_labels(widths, split)
+    return [np.flatnonzero(labels == p) for p in range(P)]
+
+
+def partition_diagonal_of(G, widths, split):
+    """Eq. (gausshat) for a split structure: keep the entries of a dense matrix whose row and column are in the
+    same partition, zero the rest."""
+    labels, _ = partition_labels(widths, split)
+    return np.where(labels[:, None] == labels[None, :], G, 0.0)
+
+
+def Gv_partition_definition(theta, widths, C, XS, v, split):
+    """Eq. (approx-jaco) from explicit J^i: partition p uses only its own columns J^i_p."""
+    v = np.asarray(v, dtype=np.float64)
+    parts = partition_indices(widths, split)
+    acc = np.zeros_like(v)
+    for x in XS:
+        J = jacobian(theta, widths, x)
+        for idx in parts:
+            Jp = J[:, idx]
+            acc[idx] += Jp.T @ (2.0 * (Jp @ v[idx]))
+    return v / C + acc / len(XS)
+
+
+def Gv_partition(theta, widths, C, XS, v, split):
+    """Eq. (approx-jaco) for a split structure in the order of Section 4.2, all rows at once: for the partition
+    (T_{m-1}, T_m), u_i = sum_{t in T_{m-1}} z^{m-1,i}_t mat(v_p)_{t,.} (plus c^m restricted to T_m when
+    T_{m-1} is the first group), J_p v_p = D^m_i[:, T_m] u_i (Eq. direct-JV-cost), then
+    D^m_i[:, T_m]^T (2 J_p v_p) (Eq. JTv) and the outer product with z^{m-1,i}_{T_{m-1}} (Eq. JTV-independent)."""
+    v = np.asarray(v, dtype=np.float64)
+    Z = forward(theta, widths, XS)
+    D = jacobian_factors(theta, widths, Z)
+    dirs = unpack(v, widths)
+    rows = Z[0].shape[0]
+    out = []
+    for m, (V, c) in enumerate(dirs, start=1):
+        ba, bb = group_bounds(widths[m - 1], split[m - 1]), group_bounds(widths[m], split[m])
+        GW, Gb = np.zeros_like(V), np.zeros_like(c)
+        for a in range(split[m - 1]):
+            Ta = slice(ba[a], ba[a + 1])
+            for b in range(split[m]):
+                Tb = slice(bb[b], bb[b + 1])
+                U = Z[m - 1][:, Ta] @ V[Ta, Tb]
+                if a == 0:
+                    U = U + c[Tb]
+                Dp = D[m - 1][:, :, Tb]
+                P = np.einsum("iuj,ij->iu", Dp, U)
+                Q = np.einsum("iuj,iu->ij", Dp, 2.0 * P)
+                GW[Ta, Tb] = Z[m - 1][:, Ta].T @ Q / rows
+                if a == 0:
+                    Gb[Tb] = Q.sum(axis=0) / rows
+        out.append((GW, Gb))
+    return v / C + pack(out)
+
+
+def cg_partitioned(theta, widths, C, XS, g, lam, split, max_iter, tol, cg_min=0, finished_share=1.0):
+    """The P independent systems of Eq. (p-linear) run in lock step, with the termination rule of Section 4.4:
+    every partition stops once at least `cg_min` steps are done and at least `finished_share` of the partitions
+    have met Eq. (cg-stopping-sample); a partition that met its own rule earlier stays frozen.
+    Returns (d, iterates, resnorms) like `cg`."""
+    g = np.asarray(g, dtype=np.float64)
+    parts = partition_indices(widths, split)
+    P = len(parts)
+    d = np.zeros_like(g)
+    r = -g.copy()
+    p = r.copy()
+    rho = np.array([r[s] @ r[s] for s in parts])
+    gnorm = np.sqrt(rho.copy())
+    active = np.array([tol <= 0 or np.sqrt(rho[k]) > tol * gnorm[k] for k in range(P)]) & (rho > 0)
+    iterates, resnorms = [], [np.sqrt(rho.copy())]
+    it = 0
+    while it < max_iter and active.any():
+        if it >= cg_min and (P - active.sum()) >= finished_share * P:
+            break
+        q = Gv_partition(theta, widths, C, XS, p, split) + lam * p
+        for k, s in enumerate(parts):
+            if not active[k]:
+                continue
+            alpha = rho[k] / (p[s] @ q[s])
+            d[s] += alpha * p[s]
+            r[s] -= alpha * q[s]
+            rho_new = r[s] @ r[s]
+            p[s] = r[s] + (rho_new / rho[k]) * p[s]
+            rho[k] = rho_new
+            if tol > 0 and np.sqrt(rho_new) <= tol * gnorm[k]:
+                active[k] = False
+        it += 1
+        iterates.append(d.copy())
+        resnorms.append(np.sqrt(rho.copy()))
+    return d, iterates, resnorms
 
 
 # --------------------------------------------------------------------------- Newton iteration (Algorithm 3 on one node)
