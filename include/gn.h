@@ -119,6 +119,35 @@ gn_status gn_set_batch_rows(gn_ctx* ctx, int64_t rows);
 gn_status gn_set_blockdiag_method(gn_ctx* ctx, int method);
 
 /*
+ * gn_set_split - variable partition of Section 3.1 for the block-diagonal product and its CG.
+ *   split  HOST array of L+1 counts: layer m's n_m neurons are cut into split[m] contiguous groups, group g
+ *          holding neurons floor(g n_m / split[m]) .. floor((g+1) n_m / split[m]) - 1 (the paper gives only the
+ *          counts, e.g. 3-2-3 for 150-200-30, and equal group sizes in its example).  1 <= split[m] <= n_m.
+ * A partition is the weights w^m_{tj} with t in one group of layer m-1 and j in one group of layer m; b^m_j
+ * belongs to the partition of the FIRST group of layer m-1.  Partitions are numbered layer by layer and inside
+ * layer m by a * split[m] + b (a: group below, b: group at layer m); there are sum_m split[m-1] split[m] of
+ * them (at most 1024).  gn_Gv_blockdiag then returns Eq. (approx-jaco) with one block per partition and
+ * gn_cg_solve(blockdiag = 1) runs one system per partition (Eq. p-linear).  All ones (the default) means one
+ * block per layer.  With any split[m] > 1 the product uses the stored Jacobian factors of Sections 3.3.1 and
+ * 4.2 (|S| n_L n_m floats per hidden layer, built once per (theta, subsample)); networks with two or more
+ * layers then need n_L <= 32.  Group boundaries that are multiples of 4 neurons keep the 16-byte access paths.
+ * The vectors keep the layout of theta.  Synchronises the stream.  GN_EINVAL on a bad count.
+ */
+gn_status gn_set_split(gn_ctx* ctx, const int32_t* split);
+
+/* gn_num_partitions - number of blocks of the block-diagonal system (L until gn_set_split changes it). */
+int32_t gn_num_partitions(const gn_ctx* ctx);
+
+/*
+ * gn_set_cg_termination - the rule of Section 4.4 for block-diagonal solves: every partition stops as soon as
+ * at least cg_min steps have been taken AND at least finished_share of the partitions have met their own stop
+ * rule (Eq. cg-stopping-sample); a partition that met it earlier stays frozen meanwhile.  Steps are counted in
+ * lock step (all partitions advance together on one GPU).  Defaults cg_min = 0, finished_share = 1 (every
+ * partition runs to its own stop rule); the paper's experiments use cg_min = 3.  finished_share in (0, 1].
+ */
+gn_status gn_set_cg_termination(gn_ctx* ctx, int32_t cg_min, double finished_share);
+
+/*
  * gn_set_theta - copy the model vector (Section 2.1 layout) into the context.  Activations stored
  * by an earlier gn_set_subsample become stale: products return GN_ESTATE until the subsample is
  * set again.

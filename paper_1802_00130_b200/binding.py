@@ -22,6 +22,9 @@ _SIGNATURES = {
     "gn_kernel_launches": (_i64, [_vp]),
     "gn_set_batch_rows": (_i32, [_vp, _i64]),
     "gn_set_blockdiag_method": (_i32, [_vp, _i32]),
+    "gn_set_split": (_i32, [_vp, C.POINTER(_i32)]),
+    "gn_num_partitions": (_i32, [_vp]),
+    "gn_set_cg_termination": (_i32, [_vp, _i32, _dbl]),
     "gn_set_theta": (_i32, [_vp, _vp]),
     "gn_set_theta_host": (_i32, [_vp, _vp]),
     "gn_set_subsample": (_i32, [_vp, _vp, _i64]),
@@ -196,6 +199,22 @@ class GnContext:
     def set_blockdiag_method(self, method):
         """0 choose, 1 propagate stacked streams, 2 stored Jacobian factors (Section 3.3.1)."""
         self._check(self._lib.gn_set_blockdiag_method(self._h, int(method)))
+
+    def set_split(self, split):
+        """Variable partition of Section 3.1: split[m] contiguous neuron groups in layer m (L+1 counts)."""
+        split = [int(x) for x in split]
+        if len(split) != len(self.widths):
+            raise ValueError("split needs one count per layer, input layer included")
+        arr = (C.c_int32 * len(split))(*split)
+        self._check(self._lib.gn_set_split(self._h, arr))
+
+    @property
+    def num_partitions(self):
+        return int(self._lib.gn_num_partitions(self._h))
+
+    def set_cg_termination(self, cg_min=0, finished_share=1.0):
+        """Termination rule of Section 4.4 for block-diagonal solves."""
+        self._check(self._lib.gn_set_cg_termination(self._h, int(cg_min), float(finished_share)))
 
     def set_theta(self, theta):
         import torch

@@ -40,6 +40,13 @@ struct gn_ctx {
   int bd_method = 0;        // 0 choose, 1 propagate L stacked streams, 2 stored factors
   int bd_expect = 0;        // products the running solver may still ask for (0 outside a solver)
   int bd_count = 0;         // propagate-form products since the factors were last invalidated
+  // variable partition (Section 3.1): split[m] contiguous neuron groups in layer m; all ones = one block per layer
+  std::vector<int> split;
+  bool has_split = false;
+  int P = 0;                // number of partitions = sum_m split[m-1] split[m]
+  float* SU = nullptr; float* SQ = nullptr; int64_t capSplit = 0;   // per-group right-hand sides and results
+  int cg_min = 0;           // termination rule of Section 4.4 for block-diagonal solves
+  double cg_share = 1.0;
   // row-batch workspace of f / grad
   int64_t capB = 0;
   std::vector<float*> Zb, Db;
@@ -59,7 +66,7 @@ struct gn_ctx {
   float* tmp_a = nullptr; float* tmp_b = nullptr;  // staging for *_host calls
   float* nt[4] = {nullptr, nullptr, nullptr, nullptr};  // Newton iteration: g, d, G d / G dbar, trial theta
   CgChunk* chunks[2] = {nullptr, nullptr}; int n_chunks[2] = {0, 0};
-  CgSeg* segs = nullptr;
+  CgSeg* segs = nullptr; int64_t segs_cap = 0;
 
   // optional per-GEMM timing
   struct EvPair { cudaEvent_t a, b; double flop; int kind; };
@@ -221,6 +228,9 @@ gn_status ensure_colsum(gn_ctx* c, int64_t rows, int cols) {
   c->colsum_cap = need;
   return GN_OK;
 }
+
+// First neuron of group g when a layer of n neurons is cut into `groups` contiguous groups.
+int group_lo(int n, int groups, int g) { return (int)(((long long)g * n) / groups); }
 
 const float* Wm(const gn_ctx* c, const float* vec, int m) { return vec + c->w_off[m]; }
 const float* bm(const gn_ctx* c, const float* vec, int m) { return vec + c->b_off[m]; }
@@ -397,12 +407,76 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
     run_gemm(c, g);
     const float* ds = c->RZ[m];
     if (m < L) {
-      c->launches += launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], c->DS[m], c->st);
+      c->launches += launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], 1, 1, 0, c->DS[m], c->st);
       ds = c->DS[m];
     }
     GN_TRY(weight_block(c, m, ds, c->Z[m - 1], nS, inv, v, coef, out));
   }
   return check_launch(c, "block-diagonal G v (stored factors)");
+}
+
+// Eq. (approx-jaco) for a split structure, in the order of Section 4.2.  Layer m with s_a groups below and s_b
+// groups at it: stream a holds U_a = Z_{m-1}[:, T_a] V^m[T_a, :] (+ c^m for the first group, which owns the
+// biases); one pass over the stored factors turns every (stream a, group b) slice into
+// Q_a[:, T_b] = D[:, :, T_b]^T 2 D[:, :, T_b] U_a[:, T_b]; then out_W[T_a, :] = Z_{m-1}[:, T_a]^T Q_a / |S|.
+// At the output layer D = I, so Q_a = 2 U_a.
+gn_status product_split(gn_ctx* c, const float* v, float* out, float coef) {
+  const int L = c->L, nL = c->w[L];
+  const int64_t nS = c->nS;
+  if (L >= 2) {
+    if (nL > 32) return fail(c, GN_EINVAL, "a split structure needs n_L <= 32 (stored Jacobian factors)");
+    if ((int64_t)nL * nS > 65535LL * 128) return fail(c, GN_EINVAL, "n_L * |S| exceeds 8 388 480 rows");
+    GN_TRY(ensure_factors(c));
+  }
+  int64_t need = 0;
+  for (int m = 1; m <= L; ++m) {
+    const int64_t f = (int64_t)c->split[m - 1] * nS * c->w[m];
+    if (f > need) need = f;
+  }
+  if (need > c->capSplit) {
+    GN_TRY(sync(c, "split workspace"));
+    dev_free(c, c->SU, c->capSplit); dev_free(c, c->SQ, c->capSplit);
+    c->capSplit = 0;
+    GN_TRY(dev_alloc(c, &c->SU, need));
+    GN_TRY(dev_alloc(c, &c->SQ, need));
+    c->capSplit = need;
+  }
+  const float inv = (float)(1.0 / (double)nS);
+  for (int m = 1; m <= L; ++m) {
+    const int sa = c->split[m - 1], sb = c->split[m], np = c->w[m - 1], nm = c->w[m];
+    const int64_t stride = nS * nm;
+    for (int a = 0; a < sa; ++a) {
+      const int t0 = group_lo(np, sa, a), t1 = group_lo(np, sa, a + 1);
+      GemmArgs g;
+      g.M = (int)nS; g.N = nm;
+      g.A1 = c->Z[m - 1] + t0; g.lda1 = np; g.B1 = Wm(c, v, m) + t0; g.ldb1 = np; g.K1 = t1 - t0;
+      if (a == 0) g.bias = bm(c, v, m);
+      if (m == L) g.alpha = 2.f;                          // B = 2I
+      g.D = c->SU + a * stride; g.ldd = nm;
+      run_gemm(c, g);
+    }
+    const float* Q = c->SU;
+    if (m < L) {
+      c->launches += launch_factor_apply(c->DF[m], c->SU, nS, nL, nm, sb, sa, stride, c->SQ, c->st);
+      Q = c->SQ;
+    }
+    for (int a = 0; a < sa; ++a) {
+      const int t0 = group_lo(np, sa, a), t1 = group_lo(np, sa, a + 1);
+      GemmArgs g;
+      g.mn_padded = true;                                   // both operands are context-owned
+      g.M = nm; g.N = t1 - t0;
+      g.A1 = Q + a * stride; g.lda1 = nm; g.a_kmajor = false;
+      g.B1 = c->Z[m - 1] + t0; g.ldb1 = np; g.b_kmajor = false;
+      g.K1 = (int)nS;
+      g.alpha = inv;
+      g.cin = v + c->w_off[m] + t0; g.ld_cin = np; g.beta = coef;
+      g.D = out + c->w_off[m] + t0; g.ldd = np;
+      run_gemm(c, g);
+    }
+    GN_TRY(ensure_colsum(c, nS, nm));
+    c->launches += launch_colsum(Q, nS, nm, nm, inv, v + c->b_off[m], coef, out + c->b_off[m], c->colsum_scratch, c->st);
+  }
+  return check_launch(c, "partition-wise G v");
 }
 
 // Choosing between the two forms when the caller has not: building the factors costs about as much as
@@ -412,6 +486,7 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
 constexpr int kFactorBreakEven = 8;
 
 gn_status product_blockdiag_any(gn_ctx* c, const float* v, float* out, float coef) {
+  if (c->has_split) return product_split(c, v, out, coef);
   bool stored = c->bd_method == 2;
   if (c->bd_method == 0 && stored_factors_applicable(c))
     stored = c->factors_valid || c->bd_expect >= kFactorBreakEven || c->bd_count + 1 >= kFactorBreakEven;
@@ -501,24 +576,56 @@ gn_status need_product_state(gn_ctx* c) {
   return GN_OK;
 }
 
-gn_status build_chunks(gn_ctx* c) {
-  for (int mode = 0; mode < 2; ++mode) {
-    std::vector<CgChunk> h;
-    const int n_seg = mode == 0 ? 1 : c->L;
-    for (int s = 0; s < n_seg; ++s) {
-      const int64_t a = mode == 0 ? 0 : c->w_off[s + 1];
-      const int64_t b = mode == 0 ? c->n : (s + 1 < c->L ? c->w_off[s + 2] : c->n);
-      for (int64_t k = a; k < b; k += kCgChunk) {
-        CgChunk ch;
-        ch.start = k; ch.len = (int32_t)((b - k < kCgChunk) ? b - k : kCgChunk); ch.seg = s;
-        h.push_back(ch);
+void push_range(std::vector<CgChunk>& h, int64_t a, int64_t b, int seg) {
+  for (int64_t k = a; k < b; k += kCgChunk) {
+    CgChunk ch;
+    ch.start = k; ch.len = (int32_t)((b - k < kCgChunk) ? b - k : kCgChunk); ch.seg = seg;
+    h.push_back(ch);
+  }
+}
+
+// Chunk table of the block systems.  One block per layer: the layer's run of theta.  With a split structure:
+// partition (group a of layer m-1, group b of layer m) owns, in every row j of group b of the stored
+// [n_m][n_{m-1}] matrix, the columns of group a; b^m_j goes with the first group of layer m-1.
+// Partitions are numbered layer by layer, inside a layer by a * split[m] + b.
+void block_chunks(const gn_ctx* c, std::vector<CgChunk>& h) {
+  if (!c->has_split) {
+    for (int s = 0; s < c->L; ++s) push_range(h, c->w_off[s + 1], s + 1 < c->L ? c->w_off[s + 2] : c->n, s);
+    return;
+  }
+  int base = 0;
+  for (int m = 1; m <= c->L; ++m) {
+    const int sa = c->split[m - 1], sb = c->split[m], np = c->w[m - 1], nm = c->w[m];
+    for (int b = 0; b < sb; ++b) {
+      const int j0 = group_lo(nm, sb, b), j1 = group_lo(nm, sb, b + 1);
+      if (sa == 1) {
+        push_range(h, c->w_off[m] + (int64_t)j0 * np, c->w_off[m] + (int64_t)j1 * np, base + b);
+      } else {
+        for (int a = 0; a < sa; ++a) {
+          const int t0 = group_lo(np, sa, a), t1 = group_lo(np, sa, a + 1);
+          for (int j = j0; j < j1; ++j) push_range(h, c->w_off[m] + (int64_t)j * np + t0, c->w_off[m] + (int64_t)j * np + t1, base + a * sb + b);
+        }
       }
+      push_range(h, c->b_off[m] + j0, c->b_off[m] + j1, base + b);
     }
+    base += sa * sb;
+  }
+}
+
+gn_status build_chunks(gn_ctx* c, bool block_only) {
+  for (int mode = block_only ? 1 : 0; mode < 2; ++mode) {
+    std::vector<CgChunk> h;
+    if (mode == 0) push_range(h, 0, c->n, 0);
+    else block_chunks(c, h);
+    dev_free(c, c->chunks[mode], c->n_chunks[mode]);
     c->n_chunks[mode] = (int)h.size();
     GN_TRY(dev_alloc(c, &c->chunks[mode], (int64_t)h.size()));
     GN_CUDA(c, cudaMemcpy(c->chunks[mode], h.data(), h.size() * sizeof(CgChunk), cudaMemcpyHostToDevice));
   }
-  GN_TRY(dev_alloc(c, &c->segs, (int64_t)c->L));
+  dev_free(c, c->segs, c->segs_cap);
+  c->segs_cap = 0;
+  GN_TRY(dev_alloc(c, &c->segs, (int64_t)c->P));
+  c->segs_cap = c->P;
   return GN_OK;
 }
 
@@ -556,6 +663,7 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
   c->Z.assign(L + 1, nullptr); c->RZ.assign(L + 1, nullptr); c->DS.assign(L + 1, nullptr);
   c->DF.assign(L + 1, nullptr);
   c->Zb.assign(L + 1, nullptr); c->Db.assign(L + 1, nullptr);
+  c->split.assign(L + 1, 1); c->has_split = false; c->P = L;
   gn_status s = GN_OK;
   do {
     if ((s = dev_alloc(c, &c->theta, c->n)) != GN_OK) break;
@@ -568,7 +676,7 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
     if (cudaMallocHost(&c->hscal, 16 * sizeof(double)) != cudaSuccess) { s = GN_ENOMEM; break; }
     if (cudaMallocHost(&c->h_err, 2 * sizeof(int)) != cudaSuccess) { s = GN_ENOMEM; break; }
     c->h_err[0] = c->h_err[1] = 0;
-    if ((s = build_chunks(c)) != GN_OK) break;
+    if ((s = build_chunks(c, false)) != GN_OK) break;
     if ((s = ensure_partials(c, 2 * (int64_t)c->n_chunks[1] + 64)) != GN_OK) break;
   } while (0);
   if (s != GN_OK) { gn_destroy(c); return s; }
@@ -613,6 +721,36 @@ gn_status gn_set_blockdiag_method(gn_ctx* c, int method) {
   if (method == 2 && (c->L < 2 || c->w[c->L] > 16))
     return fail(c, GN_EINVAL, "stored factors need at least two layers and n_L <= 16");
   c->bd_method = method;
+  return GN_OK;
+}
+
+gn_status gn_set_split(gn_ctx* c, const int32_t* split) {
+  if (!c) return GN_EINVAL;
+  if (!split) return fail(c, GN_EINVAL, "split is NULL");
+  int64_t P = 0;
+  bool any = false;
+  for (int m = 0; m <= c->L; ++m) {
+    if (split[m] < 1 || split[m] > c->w[m]) return fail(c, GN_EINVAL, "split[m] must lie in [1, n_m]");
+    if (split[m] > 1) any = true;
+    if (m >= 1) P += (int64_t)split[m - 1] * split[m];
+  }
+  if (P > 1024) return fail(c, GN_EINVAL, "more than 1024 partitions");
+  if (any && c->L >= 2 && c->w[c->L] > 32) return fail(c, GN_EINVAL, "a split structure needs n_L <= 32 (stored Jacobian factors)");
+  GN_TRY(sync(c, "set_split"));
+  c->split.assign(split, split + c->L + 1);
+  c->has_split = any;
+  c->P = (int)P;
+  GN_TRY(build_chunks(c, true));
+  return ensure_partials(c, 2 * (int64_t)c->n_chunks[1] + 64);
+}
+
+int32_t gn_num_partitions(const gn_ctx* c) { return c ? c->P : -1; }
+
+gn_status gn_set_cg_termination(gn_ctx* c, int32_t cg_min, double finished_share) {
+  if (!c) return GN_EINVAL;
+  if (cg_min < 0) return fail(c, GN_EINVAL, "cg_min must be >= 0");
+  if (!(finished_share > 0.0 && finished_share <= 1.0)) return fail(c, GN_EINVAL, "finished_share must lie in (0, 1]");
+  c->cg_min = cg_min; c->cg_share = finished_share;
   return GN_OK;
 }
 
@@ -741,7 +879,7 @@ gn_status gn_cg_solve(gn_ctx* c, const float* d_g, double lambda, int blockdiag,
   if (!(lambda >= 0.0)) return fail(c, GN_EINVAL, "lambda must be >= 0");
   GN_TRY(need_product_state(c));
   const int mode = blockdiag ? 1 : 0;
-  const int n_seg = blockdiag ? c->L : 1;
+  const int n_seg = blockdiag ? c->P : 1;
   const CgChunk* ch = c->chunks[mode];
   const int nc = c->n_chunks[mode];
   const float coef = (float)(1.0 / c->C + lambda);
@@ -757,6 +895,8 @@ gn_status gn_cg_solve(gn_ctx* c, const float* d_g, double lambda, int blockdiag,
   c->bd_expect = blockdiag ? max_iter : 0;
   struct Reset { int* p; ~Reset() { *p = 0; } } reset_expect{&c->bd_expect};
   while (it < max_iter && c->hscal[3] > 0.5) {
+    // Section 4.4: all partitions stop once cg_min steps are done and the stated share of them have finished
+    if (blockdiag && it >= c->cg_min && (double)n_seg - c->hscal[3] >= c->cg_share * (double)n_seg) break;
     GN_TRY(blockdiag ? product_blockdiag_any(c, c->cg_p, c->cg_q, coef) : product_full(c, c->cg_p, c->cg_q, coef));
     c->launches += launch_cg_dot(c->cg_p, c->cg_q, ch, nc, c->partial, c->st);
     c->launches += launch_cg_scalars(1, c->partial, ch, nc, c->segs, n_seg, tol, out2, c->st);

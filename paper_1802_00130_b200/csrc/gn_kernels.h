@@ -89,8 +89,12 @@ int launch_transpose(const float* src, int rows, int cols, float* dst, cudaStrea
 // Stored Jacobian factors (d z^L / d s^m per sample, Section 3.3.1).  D is [rows * nL][n] with row i * nL + u.
 // factor_last: D[(i, u)][t] = WL[u * n + t] * z (1 - z), z = Zprev[i * n + t]   (layer L-1 from the linear output layer)
 int launch_factor_last(const float* WL, const float* Zprev, int64_t rows, int nL, int n, float* D, cudaStream_t st);
-// factor_apply: p_u = sum_j D[(i,u)][j] U[i][j];  Q[i][j] = 2 sum_u D[(i,u)][j] p_u   (Eqs. direct-JV-cost, JTv; B = 2I)
-int launch_factor_apply(const float* D, const float* U, int64_t rows, int nL, int n, float* Q, cudaStream_t st);
+// factor_apply, for every neuron group T_b of the layer (groups contiguous, boundaries floor(b n / groups)) and
+// every stream a (U and Q hold `streams` matrices [rows][n], stream_stride floats apart):
+//   p_u = sum_{j in T_b} D[(i,u)][j] U_a[i][j];  Q_a[i][j] = 2 sum_u D[(i,u)][j] p_u for j in T_b
+// (Eqs. direct-JV-cost, JTv; B = 2I).  n_L <= 32.
+int launch_factor_apply(const float* D, const float* U, int64_t rows, int nL, int n, int groups, int streams,
+                        int64_t stream_stride, float* Q, cudaStream_t st);
 
 // ---- conjugate gradient ------------------------------------------------------------------------
 // The n coordinates are cut into chunks, each inside one segment (one segment for the full system,

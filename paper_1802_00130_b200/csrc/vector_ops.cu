@@ -180,45 +180,53 @@ __global__ void __launch_bounds__(256) factor_last_kernel(const float* __restric
   }
 }
 
-// One block per sample row: pass 1 forms p_u = D_i[u][:] . U_i (block reduction per u), pass 2 re-reads D_i
-// (just read, so from cache) and writes Q_i[j] = 2 sum_u D_i[u][j] p_u.  NLMAX bounds n_L.
+// One block per (sample row i, neuron group b of the layer): the group's columns [col0, col1) of D_i are the
+// factor of every partition (T_{m-1}, T_m = group b); `streams` right-hand sides (one per group of layer m-1),
+// `stream_stride` floats apart in U and Q, share them.  Pass 1 forms p_u = D_i[u][T_b] . U_i[T_b] (block
+// reduction per u), pass 2 re-reads D_i (just read, so from cache) and writes Q_i[j] = 2 sum_u D_i[u][j] p_u.
+// NLMAX bounds n_L.  With groups = 1 and streams = 1 this is the product of a whole layer block.
 template <int NLMAX>
 __global__ void __launch_bounds__(256) factor_apply_kernel(const float* __restrict__ D, const float* __restrict__ U,
-                                                           int nL, int n, float* __restrict__ Q) {
+                                                           int nL, int n, int groups, int streams, long long stream_stride,
+                                                           float* __restrict__ Q) {
   __shared__ float red[8][NLMAX];
   __shared__ float pu[NLMAX];
   const long long i = blockIdx.x;
+  const int col0 = (int)(((long long)blockIdx.y * n) / groups), col1 = (int)(((long long)(blockIdx.y + 1) * n) / groups);
   const float* d = D + i * nL * n;
-  const float* u_row = U + i * n;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  float acc[NLMAX];
+  for (int a = 0; a < streams; ++a) {
+    const float* u_row = U + a * stream_stride + i * n;
+    float* q_row = Q + a * stream_stride + i * n;
+    float acc[NLMAX];
 #pragma unroll
-  for (int u = 0; u < NLMAX; ++u) acc[u] = 0.f;
-  for (int j = threadIdx.x; j < n; j += 256) {
-    const float uj = __ldg(u_row + j);
+    for (int u = 0; u < NLMAX; ++u) acc[u] = 0.f;
+    for (int j = col0 + threadIdx.x; j < col1; j += 256) {
+      const float uj = __ldg(u_row + j);
 #pragma unroll
-    for (int u = 0; u < NLMAX; ++u)
-      if (u < nL) acc[u] = fmaf(__ldg(d + (long long)u * n + j), uj, acc[u]);
-  }
+      for (int u = 0; u < NLMAX; ++u)
+        if (u < nL) acc[u] = fmaf(__ldg(d + (long long)u * n + j), uj, acc[u]);
+    }
 #pragma unroll
-  for (int u = 0; u < NLMAX; ++u) {
-    const float s = warp_sum(acc[u]);
-    if (lane == 0) red[w][u] = s;
-  }
-  __syncthreads();
-  if (threadIdx.x < NLMAX) {
-    float s = 0.f;
+    for (int u = 0; u < NLMAX; ++u) {
+      const float s = warp_sum(acc[u]);
+      if (lane == 0) red[w][u] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x < NLMAX) {
+      float s = 0.f;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x];
-    pu[threadIdx.x] = 2.f * s;                              // B = 2I
-  }
-  __syncthreads();
-  for (int j = threadIdx.x; j < n; j += 256) {
-    float q = 0.f;
+      for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x];
+      pu[threadIdx.x] = 2.f * s;                              // B = 2I
+    }
+    __syncthreads();
+    for (int j = col0 + threadIdx.x; j < col1; j += 256) {
+      float q = 0.f;
 #pragma unroll
-    for (int u = 0; u < NLMAX; ++u)
-      if (u < nL) q = fmaf(__ldg(d + (long long)u * n + j), pu[u], q);
-    Q[i * n + j] = q;
+      for (int u = 0; u < NLMAX; ++u)
+        if (u < nL) q = fmaf(__ldg(d + (long long)u * n + j), pu[u], q);
+      q_row[j] = q;
+    }
   }
 }
 
@@ -397,57 +405,68 @@ int launch_sum_partials(const double* partial, int count, double* out, bool accu
   return 1;
 }
 
-// Register-resident form for rows of at most 1024 * STRIPS floats (n % 4 == 0): every thread keeps its
-// n_L x 4 x STRIPS slice of D_i in registers between the two passes, so D is read exactly once.
+// Register-resident form for groups of at most 1024 * STRIPS columns (n and every group boundary multiples
+// of 4): every thread keeps its n_L x 4 x STRIPS slice of D_i in registers across the passes and the streams,
+// so D is read exactly once.
 template <int NLMAX, int STRIPS>
 __global__ void __launch_bounds__(256) factor_apply_reg_kernel(const float* __restrict__ D, const float* __restrict__ U,
-                                                               int nL, int n, float* __restrict__ Q) {
+                                                               int nL, int n, int groups, int streams,
+                                                               long long stream_stride, float* __restrict__ Q) {
   __shared__ float red[8][NLMAX];
   __shared__ float pu[NLMAX];
   const long long i = blockIdx.x;
+  const int col0 = (int)(((long long)blockIdx.y * n) / groups), col1 = (int)(((long long)(blockIdx.y + 1) * n) / groups);
   const float* d = D + i * nL * n;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   float4 dv[STRIPS][NLMAX];
-  float acc[NLMAX];
-#pragma unroll
-  for (int u = 0; u < NLMAX; ++u) acc[u] = 0.f;
 #pragma unroll
   for (int s = 0; s < STRIPS; ++s) {
-    const int j = (s * 256 + threadIdx.x) * 4;
-    const bool ok = j < n;
+    const int j = col0 + (s * 256 + threadIdx.x) * 4;
+    const bool ok = j < col1;
 #pragma unroll
     for (int u = 0; u < NLMAX; ++u)
       dv[s][u] = (ok && u < nL) ? __ldg(reinterpret_cast<const float4*>(d + (long long)u * n + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    const float4 uj = ok ? __ldg(reinterpret_cast<const float4*>(U + i * n + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int u = 0; u < NLMAX; ++u)
-      acc[u] += dv[s][u].x * uj.x + dv[s][u].y * uj.y + dv[s][u].z * uj.z + dv[s][u].w * uj.w;
   }
+  for (int a = 0; a < streams; ++a) {
+    const float* u_row = U + a * stream_stride + i * n;
+    float* q_row = Q + a * stream_stride + i * n;
+    float acc[NLMAX];
 #pragma unroll
-  for (int u = 0; u < NLMAX; ++u) {
-    const float s = warp_sum(acc[u]);
-    if (lane == 0) red[w][u] = s;
-  }
-  __syncthreads();
-  if (threadIdx.x < NLMAX) {
-    float s = 0.f;
+    for (int u = 0; u < NLMAX; ++u) acc[u] = 0.f;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x];
-    pu[threadIdx.x] = 2.f * s;                              // B = 2I
-  }
-  __syncthreads();
+    for (int s = 0; s < STRIPS; ++s) {
+      const int j = col0 + (s * 256 + threadIdx.x) * 4;
+      const float4 uj = j < col1 ? __ldg(reinterpret_cast<const float4*>(u_row + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-  for (int s = 0; s < STRIPS; ++s) {
-    const int j = (s * 256 + threadIdx.x) * 4;
-    if (j < n) {
-      float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int u = 0; u < NLMAX; ++u)
+        acc[u] += dv[s][u].x * uj.x + dv[s][u].y * uj.y + dv[s][u].z * uj.z + dv[s][u].w * uj.w;
+    }
 #pragma unroll
-      for (int u = 0; u < NLMAX; ++u) {
-        const float pv = pu[u];
-        q.x = fmaf(dv[s][u].x, pv, q.x); q.y = fmaf(dv[s][u].y, pv, q.y);
-        q.z = fmaf(dv[s][u].z, pv, q.z); q.w = fmaf(dv[s][u].w, pv, q.w);
+    for (int u = 0; u < NLMAX; ++u) {
+      const float s = warp_sum(acc[u]);
+      if (lane == 0) red[w][u] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x < NLMAX) {
+      float s = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x];
+      pu[threadIdx.x] = 2.f * s;                              // B = 2I
+    }
+    __syncthreads();
+#pragma unroll
+    for (int s = 0; s < STRIPS; ++s) {
+      const int j = col0 + (s * 256 + threadIdx.x) * 4;
+      if (j < col1) {
+        float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int u = 0; u < NLMAX; ++u) {
+          const float pv = pu[u];
+          q.x = fmaf(dv[s][u].x, pv, q.x); q.y = fmaf(dv[s][u].y, pv, q.y);
+          q.z = fmaf(dv[s][u].z, pv, q.z); q.w = fmaf(dv[s][u].w, pv, q.w);
+        }
+        *reinterpret_cast<float4*>(q_row + j) = q;
       }
-      *reinterpret_cast<float4*>(Q + i * n + j) = q;
     }
   }
 }
@@ -457,17 +476,29 @@ int launch_factor_last(const float* WL, const float* Zprev, int64_t rows, int nL
   return 1;
 }
 
-int launch_factor_apply(const float* D, const float* U, int64_t rows, int nL, int n, float* Q, cudaStream_t st) {
-  const bool vec = (n % 4 == 0) && ((reinterpret_cast<uintptr_t>(D) & 15) == 0) && ((reinterpret_cast<uintptr_t>(U) & 15) == 0) &&
-                   ((reinterpret_cast<uintptr_t>(Q) & 15) == 0);
-  if (vec && n <= 1024 && nL <= 4)  { factor_apply_reg_kernel<4, 1><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
-  if (vec && n <= 1024 && nL <= 10) { factor_apply_reg_kernel<10, 1><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
-  if (vec && n <= 2048 && nL <= 4)  { factor_apply_reg_kernel<4, 2><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
-  if (vec && n <= 2048 && nL <= 10) { factor_apply_reg_kernel<10, 2><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
-  if (vec && n <= 1024 && nL <= 16) { factor_apply_reg_kernel<16, 1><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q); return 1; }
-  if (nL <= 4) factor_apply_kernel<4><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q);
-  else if (nL <= 10) factor_apply_kernel<10><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q);
-  else factor_apply_kernel<16><<<(unsigned)rows, 256, 0, st>>>(D, U, nL, n, Q);
+int launch_factor_apply(const float* D, const float* U, int64_t rows, int nL, int n, int groups, int streams,
+                        int64_t stream_stride, float* Q, cudaStream_t st) {
+  bool vec = (n % 4 == 0) && (stream_stride % 4 == 0) && ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&
+             ((reinterpret_cast<uintptr_t>(U) & 15) == 0) && ((reinterpret_cast<uintptr_t>(Q) & 15) == 0);
+  int widest = 0;
+  for (int b = 0; b < groups; ++b) {
+    const int c0 = (int)(((long long)b * n) / groups), c1 = (int)(((long long)(b + 1) * n) / groups);
+    if (c0 % 4 != 0) vec = false;
+    if (c1 - c0 > widest) widest = c1 - c0;
+  }
+  const dim3 grid((unsigned)rows, (unsigned)groups);
+  const long long ss = stream_stride;
+#define GN_FA_REG(NL, STR) { factor_apply_reg_kernel<NL, STR><<<grid, 256, 0, st>>>(D, U, nL, n, groups, streams, ss, Q); return 1; }
+  if (vec && widest <= 1024 && nL <= 4)  GN_FA_REG(4, 1)
+  if (vec && widest <= 1024 && nL <= 10) GN_FA_REG(10, 1)
+  if (vec && widest <= 2048 && nL <= 4)  GN_FA_REG(4, 2)
+  if (vec && widest <= 2048 && nL <= 10) GN_FA_REG(10, 2)
+  if (vec && widest <= 1024 && nL <= 16) GN_FA_REG(16, 1)
+#undef GN_FA_REG
+  if (nL <= 4) factor_apply_kernel<4><<<grid, 256, 0, st>>>(D, U, nL, n, groups, streams, ss, Q);
+  else if (nL <= 10) factor_apply_kernel<10><<<grid, 256, 0, st>>>(D, U, nL, n, groups, streams, ss, Q);
+  else if (nL <= 16) factor_apply_kernel<16><<<grid, 256, 0, st>>>(D, U, nL, n, groups, streams, ss, Q);
+  else factor_apply_kernel<32><<<grid, 256, 0, st>>>(D, U, nL, n, groups, streams, ss, Q);
   return 1;
 }
 
