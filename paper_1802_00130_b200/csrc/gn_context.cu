@@ -1,6 +1,7 @@
 // Host side of the C ABI (include/gn.h): context, workspaces, and the launch sequences for the
 // stored forward pass, f / gradient over row batches, the full and block-diagonal Gauss-Newton
 // products, and conjugate gradient.
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -66,7 +67,7 @@ struct gn_ctx {
   float* tmp_a = nullptr; float* tmp_b = nullptr;  // staging for *_host calls
   float* nt[4] = {nullptr, nullptr, nullptr, nullptr};  // Newton iteration: g, d, G d / G dbar, trial theta
   CgChunk* chunks[2] = {nullptr, nullptr}; int n_chunks[2] = {0, 0};
-  CgSeg* segs = nullptr; int64_t segs_cap = 0;
+  CgSeg* segs[2] = {nullptr, nullptr}; int64_t segs_cap[2] = {0, 0};   // per-segment scalars: full system, block systems
 
   // optional per-GEMM timing
   struct EvPair { cudaEvent_t a, b; double flop; int kind; };
@@ -612,20 +613,32 @@ void block_chunks(const gn_ctx* c, std::vector<CgChunk>& h) {
   }
 }
 
+// Chunk tables are kept sorted by segment, and every segment records where its chunks start, so that the
+// per-segment reductions touch only their own partial sums.
 gn_status build_chunks(gn_ctx* c, bool block_only) {
   for (int mode = block_only ? 1 : 0; mode < 2; ++mode) {
     std::vector<CgChunk> h;
     if (mode == 0) push_range(h, 0, c->n, 0);
     else block_chunks(c, h);
+    std::stable_sort(h.begin(), h.end(), [](const CgChunk& a, const CgChunk& b) { return a.seg < b.seg; });
+    const int n_seg = mode == 0 ? 1 : c->P;
+    std::vector<CgSeg> segs((size_t)n_seg);
+    for (auto& sg : segs) { std::memset(&sg, 0, sizeof(CgSeg)); }
+    for (size_t i = 0; i < h.size(); ++i) {
+      CgSeg& sg = segs[(size_t)h[i].seg];
+      if (sg.count == 0) sg.first = (int)i;
+      ++sg.count;
+    }
     dev_free(c, c->chunks[mode], c->n_chunks[mode]);
     c->n_chunks[mode] = (int)h.size();
     GN_TRY(dev_alloc(c, &c->chunks[mode], (int64_t)h.size()));
     GN_CUDA(c, cudaMemcpy(c->chunks[mode], h.data(), h.size() * sizeof(CgChunk), cudaMemcpyHostToDevice));
+    dev_free(c, c->segs[mode], c->segs_cap[mode]);
+    c->segs_cap[mode] = 0;
+    GN_TRY(dev_alloc(c, &c->segs[mode], (int64_t)n_seg));
+    c->segs_cap[mode] = n_seg;
+    GN_CUDA(c, cudaMemcpy(c->segs[mode], segs.data(), segs.size() * sizeof(CgSeg), cudaMemcpyHostToDevice));
   }
-  dev_free(c, c->segs, c->segs_cap);
-  c->segs_cap = 0;
-  GN_TRY(dev_alloc(c, &c->segs, (int64_t)c->P));
-  c->segs_cap = c->P;
   return GN_OK;
 }
 
@@ -886,7 +899,7 @@ gn_status gn_cg_solve(gn_ctx* c, const float* d_g, double lambda, int blockdiag,
   double* out2 = c->dscal + 2;
 
   c->launches += launch_cg_init(d_g, d_d, c->cg_r, c->cg_p, ch, nc, c->partial, c->st);
-  c->launches += launch_cg_scalars(0, c->partial, ch, nc, c->segs, n_seg, tol, out2, c->st);
+  c->launches += launch_cg_scalars(0, c->partial, ch, nc, c->segs[mode], n_seg, tol, out2, c->st);
   GN_CUDA(c, cudaMemcpyAsync(c->hscal + 2, out2, 2 * sizeof(double), cudaMemcpyDeviceToHost, c->st));
   GN_TRY(check_launch(c, "cg init"));
   GN_TRY(sync(c, "cg init"));
@@ -899,10 +912,10 @@ gn_status gn_cg_solve(gn_ctx* c, const float* d_g, double lambda, int blockdiag,
     if (blockdiag && it >= c->cg_min && (double)n_seg - c->hscal[3] >= c->cg_share * (double)n_seg) break;
     GN_TRY(blockdiag ? product_blockdiag_any(c, c->cg_p, c->cg_q, coef) : product_full(c, c->cg_p, c->cg_q, coef));
     c->launches += launch_cg_dot(c->cg_p, c->cg_q, ch, nc, c->partial, c->st);
-    c->launches += launch_cg_scalars(1, c->partial, ch, nc, c->segs, n_seg, tol, out2, c->st);
-    c->launches += launch_cg_update(c->cg_p, c->cg_q, d_d, c->cg_r, ch, nc, c->segs, c->partial, c->st);
-    c->launches += launch_cg_scalars(2, c->partial, ch, nc, c->segs, n_seg, tol, out2, c->st);
-    c->launches += launch_cg_direction(c->cg_r, c->cg_p, ch, nc, c->segs, c->st);
+    c->launches += launch_cg_scalars(1, c->partial, ch, nc, c->segs[mode], n_seg, tol, out2, c->st);
+    c->launches += launch_cg_update(c->cg_p, c->cg_q, d_d, c->cg_r, ch, nc, c->segs[mode], c->partial, c->st);
+    c->launches += launch_cg_scalars(2, c->partial, ch, nc, c->segs[mode], n_seg, tol, out2, c->st);
+    c->launches += launch_cg_direction(c->cg_r, c->cg_p, ch, nc, c->segs[mode], c->st);
     GN_CUDA(c, cudaMemcpyAsync(c->hscal + 2, out2, 2 * sizeof(double), cudaMemcpyDeviceToHost, c->st));
     if (d_iterates)
       GN_CUDA(c, cudaMemcpyAsync(d_iterates + (int64_t)it * c->n, d_d, c->n * sizeof(float), cudaMemcpyDeviceToDevice, c->st));

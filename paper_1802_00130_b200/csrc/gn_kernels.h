@@ -109,6 +109,7 @@ struct CgSeg {           // per-segment scalars, device resident
   double gnorm2;         // ||g||^2
   float alpha, beta;
   int active;
+  int first, count;      // this segment's chunks are entries [first, first + count) of the (segment-sorted) chunk table
   int pad;
 };
 

@@ -310,7 +310,8 @@ __global__ void __launch_bounds__(256) cg_direction_kernel(const float* __restri
   }
 }
 
-// One block; warp w handles segments w, w+8, ...  Chunks of a segment are contiguous in the table.
+// One block.  With several segments warp w handles segments w, w + 8, ..., summing that segment's own run of the
+// chunk table; with a single segment the whole block sums it.  Every sum has a fixed order.
 __global__ void __launch_bounds__(256) cg_scalars_kernel(int phase, const double* __restrict__ partial,
                                                          const CgChunk* __restrict__ chunks, int n_chunks,
                                                          CgSeg* __restrict__ seg, int n_seg, double tol,
@@ -318,32 +319,47 @@ __global__ void __launch_bounds__(256) cg_scalars_kernel(int phase, const double
   __shared__ double seg_rho[64];
   __shared__ int seg_act[64];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  (void)chunks; (void)n_chunks;
+  auto update = [&](int s, double acc) -> CgSeg {
+    CgSeg g = seg[s];
+    if (phase == 0) {
+      g.rho = acc; g.gnorm2 = acc; g.pq = 0.0; g.alpha = 0.f; g.beta = 0.f;
+      g.active = (acc > 0.0) && (tol <= 0.0 || sqrt(acc) > tol * sqrt(acc)) ? 1 : 0;
+    } else if (phase == 1) {
+      g.pq = acc;
+      g.alpha = (g.active && acc > 0.0) ? (float)(g.rho / acc) : 0.f;
+      if (!(acc > 0.0)) g.active = 0;
+    } else {
+      if (g.active) {
+        g.beta = g.rho > 0.0 ? (float)(acc / g.rho) : 0.f;
+        g.rho = acc;
+        if (!(acc > 0.0) || (tol > 0.0 && sqrt(acc) <= tol * sqrt(g.gnorm2))) g.active = 0;
+      } else {
+        g.beta = 0.f; g.alpha = 0.f;
+      }
+    }
+    seg[s] = g;
+    return g;
+  };
+  if (n_seg == 1) {
+    const int first = seg[0].first, count = seg[0].count;
+    double acc = 0.0;
+    for (int c = threadIdx.x; c < count; c += 256) acc += partial[first + c];
+    acc = block_sum_256(acc);
+    if (threadIdx.x == 0) {
+      const CgSeg g = update(0, acc);
+      host_out[0] = g.rho; host_out[1] = (double)g.active;
+    }
+    return;
+  }
   for (int s0 = 0; s0 < n_seg; s0 += 64) {
     for (int s = s0 + w; s < min(n_seg, s0 + 64); s += 8) {
-      // fixed-order sum of this segment's partials: lane-strided, then a butterfly
+      const int first = seg[s].first, count = seg[s].count;
       double acc = 0.0;
-      for (int c = lane; c < n_chunks; c += 32)
-        if (chunks[c].seg == s) acc += partial[c];
+      for (int c = lane; c < count; c += 32) acc += partial[first + c];
       acc = warp_sum(acc);
       if (lane == 0) {
-        CgSeg g = seg[s];
-        if (phase == 0) {
-          g.rho = acc; g.gnorm2 = acc; g.pq = 0.0; g.alpha = 0.f; g.beta = 0.f;
-          g.active = (acc > 0.0) && (tol <= 0.0 || sqrt(acc) > tol * sqrt(acc)) ? 1 : 0;
-        } else if (phase == 1) {
-          g.pq = acc;
-          g.alpha = (g.active && acc > 0.0) ? (float)(g.rho / acc) : 0.f;
-          if (!(acc > 0.0)) g.active = 0;
-        } else {
-          if (g.active) {
-            g.beta = g.rho > 0.0 ? (float)(acc / g.rho) : 0.f;
-            g.rho = acc;
-            if (!(acc > 0.0) || (tol > 0.0 && sqrt(acc) <= tol * sqrt(g.gnorm2))) g.active = 0;
-          } else {
-            g.beta = 0.f; g.alpha = 0.f;
-          }
-        }
-        seg[s] = g;
+        const CgSeg g = update(s, acc);
         seg_rho[s - s0] = g.rho;
         seg_act[s - s0] = g.active;
       }
