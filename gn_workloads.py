@@ -82,6 +82,22 @@ def draw_theta(rng, widths):
     return np.concatenate(parts).astype(np.float32)
 
 
+def draw_theta_sparse(rng, widths):
+    """Sparse initialisation (Section 6.2 with the count of Section 8.2): of the n_{m-1} weights into a neuron
+    of layer m, ceil(sqrt(n_{m-1})) randomly chosen ones are N(0, 1), the rest zero.  The paper does not say
+    what the biases start as; they are zero here."""
+    parts = []
+    for m in range(1, len(widths)):
+        a, b = widths[m - 1], widths[m]
+        k = int(np.ceil(np.sqrt(a)))
+        W = np.zeros((b, a), dtype=np.float32)              # row j = the weights into neuron j (theta's layout)
+        for j in range(b):
+            W[j, rng.choice(a, size=k, replace=False)] = rng.standard_normal(k, dtype=np.float32)
+        parts.append(W.reshape(-1))
+        parts.append(np.zeros(b, dtype=np.float32))
+    return np.concatenate(parts)
+
+
 def make(name, l=None, nS=None, with_v=True):
     """Build the named workload; `l` / `nS` override the row counts (same recipe)."""
     rec = dict(WORKLOADS[name])
@@ -108,15 +124,15 @@ def make(name, l=None, nS=None, with_v=True):
                 theta=theta, idx=idx, v=v, n=n)
 
 
-def make_custom(widths, l, nS, C, seed, x="uniform", n_vec=1):
-    """Free-form small problem (tests): same draw order as `make`."""
+def make_custom(widths, l, nS, C, seed, x="uniform", n_vec=1, theta="dense"):
+    """Free-form small problem (tests): same draw order as `make`; theta "dense" or "sparse" (Section 6.2)."""
     widths = list(widths)
     rng = np.random.Generator(np.random.PCG64(seed))
     X = draw_rows(rng, x, l, widths[0])
     labels = rng.integers(0, widths[-1], size=l)
     Y = np.zeros((l, widths[-1]), dtype=np.float32)
     Y[np.arange(l), labels] = 1.0
-    theta = draw_theta(rng, widths)
+    theta = draw_theta(rng, widths) if theta == "dense" else draw_theta_sparse(rng, widths)
     idx = rng.permutation(l)[:nS].astype(np.int32)
     n = num_params(widths)
     vs = [rng.standard_normal(n, dtype=np.float32) for _ in range(n_vec)]

@@ -301,3 +301,21 @@ def test_the_default_method_builds_factors_only_when_they_pay():
     assert ctx.workspace_bytes - short >= factor_bytes
     ctx.cg_solve(dev(g), 1.0, blockdiag=False, max_iter=8, tol=0.0)
     ctx.close()
+
+
+@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+def test_sparse_initialisation_of_the_paper(mode):
+    """Section 6.2: ceil(sqrt(n_{m-1})) N(0,1) weights into every neuron, the rest zero (saturating pre-activations)."""
+    p = wl.make_custom([784, 300, 300, 10], l=2000, nS=1000, C=20.0, seed=31, x="sparse80", theta="sparse")
+    w = p["widths"]
+    W1 = p["theta"][: 784 * 300].reshape(300, 784)
+    assert ((W1 != 0).sum(axis=1) == 28).all()                 # ceil(sqrt(784)) per neuron
+    ctx = make_ctx(p, mode)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    assert rel(ctx.Gv(dev(p["v"])).cpu().numpy(), orc.Gv(p["theta"], w, p["C"], XS, p["v"])) <= TOL[mode]
+    assert rel(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy(), orc.Gv_blockdiag(p["theta"], w, p["C"], XS, p["v"])) <= TOL[mode]
+    g, f = ctx.grad(with_f=True)
+    assert abs(f - orc.fun(p["theta"], w, p["C"], p["X"], p["Y"])) <= TOL[mode] * abs(f)
+    assert rel(g.cpu().numpy(), orc.grad(p["theta"], w, p["C"], p["X"], p["Y"])) <= TOL[mode]
+    ctx.close()
