@@ -49,7 +49,8 @@ struct Tf32Params {
   int tiles_n, tiles;
   int* err;
   // work list of the two-CTA kernel: pair q runs tiles q, q + P, ... for `waves` full waves of P tiles;
-  // the `rem` tiles left over are each cut along K into `slices` parts, one per pair (slices == 1: whole)
+  // the `rem` tiles left over are each cut along K into `slices` parts, one per pair, done before the
+  // pair's whole tiles (slices == 1: whole tiles, done last)
   int P, waves, rem, slices;
   float* sk_ws;          // [P][2][128][256] raw partial accumulators of the sliced tiles, slot = pair
   int* sk_flags;         // [P] arrival counters, one per sliced tile, zeroed before the launch
@@ -377,11 +378,13 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant
 //
 // Work list: with T tiles on P pairs, pair q runs tiles q, q + P, ... for the floor(T / P) full waves, so
 // that all pairs move through neighbouring tiles together (tiles of one A panel are read at the same
-// time and hit in L2).  The T mod P tiles of the last, partial wave are each cut along K into up to 8
-// slices, one per otherwise idle pair.  The pairs of a sliced tile store their raw accumulators in a
-// workspace, count themselves in on the tile's flag, wait (bounded) until all slices have arrived, and
-// then each sums one share of the tile's column chunks over all slices, in slice order, and runs the
-// epilogue on it.  The order of every sum is fixed, so results are deterministic.
+// time and hit in L2).  The T mod P tiles left over are each cut along K into up to 8 slices, one per
+// pair, and a pair does its slice before its whole tiles.  The pairs of a sliced tile store their raw
+// accumulators in a workspace, count themselves in on the tile's flag, wait (bounded) until all slices
+// have arrived, and then each sums one share of the tile's column chunks over all slices, in slice
+// order, and runs the epilogue on it - all of this on the epilogue warps while the MMA issuer is already
+// working on the pair's first whole tile in the other accumulator.  The order of every sum is fixed, so
+// results are deterministic.
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -431,20 +434,29 @@ __device__ __forceinline__ void mma2_commit_both(uint64_t* bar) {
 struct Work { int tile, kb0, kb1, sliced; };
 
 // idx-th piece of work of CTA pair `pair` (see Tf32Params); false when the pair has no more.
+// A pair that takes part in the K-sliced tiles does its slice FIRST: the store of the partial accumulator,
+// the wait for the other slices and the fix-up epilogue then run on the epilogue warps underneath the
+// MMAs of the pair's first whole tile instead of being exposed at the end of the kernel.
 __device__ __forceinline__ bool next_work(const Tf32Params& p, int pair, int total_kb, int idx, Work& w) {
-  if (idx < p.waves) { w.tile = idx * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0; return true; }
-  if (idx > p.waves || p.rem == 0) return false;
-  if (p.slices < 2) {
-    if (pair >= p.rem) return false;
-    w.tile = p.waves * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0;
+  if (p.slices >= 2) {
+    if (pair < p.rem * p.slices) {
+      if (idx == 0) {
+        const int j = pair / p.slices, sl = pair - j * p.slices;
+        w.tile = p.waves * p.P + j;
+        w.kb0 = (int)((long long)total_kb * sl / p.slices);
+        w.kb1 = (int)((long long)total_kb * (sl + 1) / p.slices);
+        w.sliced = 1;
+        return true;
+      }
+      --idx;
+    }
+    if (idx >= p.waves) return false;
+    w.tile = idx * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0;
     return true;
   }
-  if (pair >= p.rem * p.slices) return false;
-  const int j = pair / p.slices, sl = pair - j * p.slices;
-  w.tile = p.waves * p.P + j;
-  w.kb0 = (int)((long long)total_kb * sl / p.slices);
-  w.kb1 = (int)((long long)total_kb * (sl + 1) / p.slices);
-  w.sliced = 1;
+  if (idx < p.waves) { w.tile = idx * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0; return true; }
+  if (idx > p.waves || pair >= p.rem) return false;
+  w.tile = p.waves * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0;
   return true;
 }
 
