@@ -188,6 +188,8 @@ def run_ours(args):
     mode = gn.GN_TF32 if args.mode == "tf32" else gn.GN_FP32_ACCURATE
     X, Y = torch.from_numpy(p["X"]).to(dev), torch.from_numpy(p["Y"]).to(dev)
     ctx = gn.GnContext(p["widths"], p["C"], X, Y, mode)
+    if args.mode == "fp32_fma":
+        ctx.set_accurate_method(1)
     theta = torch.from_numpy(p["theta"]).to(dev)
     # a fresh subsample per step, as in the Newton iteration: rotations of one permutation
     rng = np.random.Generator(np.random.PCG64(4242 + rank))
@@ -347,13 +349,20 @@ def run_ours(args):
         peak = pk["bf16_sustained"] / 2.0
         roof = {"bound": "tensor", "unit": "TFLOP/s", "peak": peak,
                 "peak_note": f"TF32 = 1/2 of the {pk['src']} sustained bf16 cuBLAS rate ({pk['bf16_sustained']} TFLOP/s)"}
+    elif args.mode == "fp32":
+        peak = pk["bf16_sustained"] / 6.0
+        roof = {"bound": "tensor", "unit": "TFLOP/s", "peak": peak,
+                "peak_note": f"FP32-accurate on the tensor cores takes 3 TF32 products per term: 1/3 of the TF32 peak, "
+                             f"itself 1/2 of the {pk['src']} sustained bf16 cuBLAS rate ({pk['bf16_sustained']} TFLOP/s)"}
     else:
         peak = SMS * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
         roof = {"bound": "alu", "unit": "TFLOP/s", "peak": peak,
                 "peak_note": "148 SMs x 128 FP32 lanes x 2 FLOP x max SM clock"}
-    kern = prof["tensor"] if args.mode == "tf32" else prof["ffma"]
+    main = {"tf32": "tensor", "fp32": "tensor_x3", "fp32_fma": "ffma"}[args.mode]
+    kern = prof[main]
     achieved = kern["flop"] / (kern["ms"] * 1e-3) / 1e12 if kern["ms"] > 0 else None
-    roof.update({"kernel": "gemm_tf32_2cta_kernel + gemm_tf32_kernel" if args.mode == "tf32" else "gemm_ffma_kernel",
+    roof.update({"kernel": {"tensor": "gemm_tf32_2cta_kernel + gemm_tf32_kernel", "tensor_x3": "gemm_tf32x3_kernel",
+                            "ffma": "gemm_ffma_kernel"}[main],
                  "achieved": achieved, "frac": achieved / peak if achieved else None,
                  "traffic": (TRAFFIC.get((args.mode, args.workload)) or {}).get("bytes_per_launch"),
                  "traffic_note": TRAFFIC.get((args.mode, args.workload)),
@@ -363,8 +372,7 @@ def run_ours(args):
                  "frac_of_library": achieved / lib_tf32 if (achieved and lib_tf32) else None,
                  "frac_of_nominal": achieved / 1100.0 if (achieved and args.mode == "tf32") else None,
                  "other_contractions": {name: {"ms": prof[name]["ms"], "launches": prof[name]["launches"]}
-                                        for name in ("tensor", "ffma", "thin")
-                                        if name != ("tensor" if args.mode == "tf32" else "ffma")}})
+                                        for name in ("tensor", "tensor_x3", "ffma", "thin") if name != main}})
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -395,7 +403,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mnist2000_20", choices=sorted(wl.WORKLOADS))
-    ap.add_argument("--mode", default="tf32", choices=["fp32", "tf32"])
+    ap.add_argument("--mode", default="tf32", choices=["fp32", "fp32_fma", "tf32"],
+                    help="tf32: TF32 contractions; fp32: FP32-accurate mode (error-compensated tensor-core contractions "
+                         "where the shape allows); fp32_fma: FP32-accurate mode with every contraction on the FP32 FMA GEMM")
     ap.add_argument("--n-cg", dest="n_cg", type=int, default=10)
     ap.add_argument("--product-reps", type=int, default=10)
     ap.add_argument("--ref-rows", type=int, default=1024)

@@ -119,6 +119,21 @@ gn_status gn_set_batch_rows(gn_ctx* ctx, int64_t rows);
 gn_status gn_set_blockdiag_method(gn_ctx* ctx, int method);
 
 /*
+ * gn_set_accurate_method - how GN_FP32_ACCURATE contexts compute the dense contractions (the paper does not fix a
+ * floating-point width; the acceptance bound of this mode is 1e-5 relative L2 against float64).
+ *   0  choose (default): the tensor cores in error-compensated form wherever the shape suits the CTA-pair kernel
+ *      (more than 128 rows and at least 128 columns of output), the FP32 FMA GEMM elsewhere;
+ *   1  the FP32 FMA GEMM for everything;
+ *   2  same as 0.
+ * Error-compensated form: every operand X is split into X = Xhi + Xlo, both exactly representable in TF32
+ * (|X - Xhi - Xlo| <= 2^-22 |X|); the product is Alo Bhi + Ahi Blo + Ahi Bhi accumulated in FP32, with the sum over k
+ * cut into chunks of 1024 that are added in FP32 round-to-nearest outside the tensor core (its own accumulator
+ * truncates).  Splits of theta and of the stored activations are kept until set_theta / set_subsample; they
+ * double the memory those take.  No effect on GN_TF32 contexts.  GN_EINVAL for another value.
+ */
+gn_status gn_set_accurate_method(gn_ctx* ctx, int method);
+
+/*
  * gn_set_split - variable partition of Section 3.1 for the block-diagonal product and its CG.
  *   split  HOST array of L+1 counts: layer m's n_m neurons are cut into split[m] contiguous groups, group g
  *          holding neurons floor(g n_m / split[m]) .. floor((g+1) n_m / split[m]) - 1 (the paper gives only the
@@ -274,9 +289,11 @@ gn_status gn_debug_activations(gn_ctx* ctx, int m, float* d_out);
  * gn_profile - switch per-launch timing of the contraction kernels on (enable != 0) or off.  While on,
  * every GEMM launch is bracketed by a pair of CUDA events on the context's stream.
  * gn_profile_read - synchronise the stream and return, for the tensor-core kernel (index 0), the
- * FP32 FMA GEMM (index 1) and the streaming kernels for n_L-wide shapes (index 2): summed device time
- * in milliseconds, floating-point operations executed (2 M N K per launch) and number of launches;
- * then reset the counters.  Each output is an array of three entries and may be NULL.
+ * FP32 FMA GEMM (index 1), the streaming kernels for n_L-wide shapes (index 2) and the error-compensated
+ * tensor-core kernel of GN_FP32_ACCURATE contexts (index 3): summed device time in milliseconds,
+ * floating-point operations of the contractions (2 M N K per launch; for index 3 the three TF32 products
+ * per term count once) and number of launches; then reset the counters.  Each output is an array of four
+ * entries and may be NULL.
  */
 gn_status gn_profile(gn_ctx* ctx, int enable);
 gn_status gn_profile_read(gn_ctx* ctx, double* gemm_ms, double* gemm_flop, int64_t* gemm_launches);
@@ -287,7 +304,8 @@ gn_status gn_profile_read(gn_ctx* ctx, double* gemm_ms, double* gemm_flop, int64
  * a dimension <= 16, 3 = tensor-core TF32 with the promise that every [K][M] / [K][N] operand is
  * followed by at least 128 readable bytes, which lets it fetch them with one TMA box per stage;
  * 4 and 5 = as 3 with one CTA per 128-row tile, respectively a CTA pair per 256-row tile, forced;
- * 6 = as 5 but whole tiles only, i.e. without the stream-K split of tiles between CTA pairs).  a_kmajor: A is [M][K]
+ * 6 = as 5 but whole tiles only, i.e. without the stream-K split of tiles between CTA pairs;
+ * 7 = the error-compensated tensor-core form of GN_FP32_ACCURATE contexts, see gn_set_accurate_method).  a_kmajor: A is [M][K]
  * (else [K][M]); b_kmajor: B is [N][K] (else [K][N]); all row-major with the given leading
  * dimensions.  GN_EINVAL if the chosen kernel cannot take the operands (alignment, shape).
  */

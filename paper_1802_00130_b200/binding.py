@@ -22,6 +22,7 @@ _SIGNATURES = {
     "gn_kernel_launches": (_i64, [_vp]),
     "gn_set_batch_rows": (_i32, [_vp, _i64]),
     "gn_set_blockdiag_method": (_i32, [_vp, _i32]),
+    "gn_set_accurate_method": (_i32, [_vp, _i32]),
     "gn_set_split": (_i32, [_vp, C.POINTER(_i32)]),
     "gn_num_partitions": (_i32, [_vp]),
     "gn_set_cg_termination": (_i32, [_vp, _i32, _dbl]),
@@ -200,6 +201,10 @@ class GnContext:
         """0 choose, 1 propagate stacked streams, 2 stored Jacobian factors (Section 3.3.1)."""
         self._check(self._lib.gn_set_blockdiag_method(self._h, int(method)))
 
+    def set_accurate_method(self, method):
+        """0 choose, 1 FP32 FMA GEMM only, 2 error-compensated tensor-core form where the shape allows."""
+        self._check(self._lib.gn_set_accurate_method(self._h, int(method)))
+
     def set_split(self, split):
         """Variable partition of Section 3.1: split[m] contiguous neuron groups in layer m (L+1 counts)."""
         split = [int(x) for x in split]
@@ -298,11 +303,11 @@ class GnContext:
         self._check(self._lib.gn_profile(self._h, int(bool(enable))))
 
     def profile_read(self):
-        """Per-kernel GEMM timing since the last read: {"tensor": {...}, "ffma": {...}}."""
-        ms, flop, cnt = (_dbl * 3)(), (_dbl * 3)(), (_i64 * 3)()
+        """Per-kernel GEMM timing since the last read: {"tensor": {...}, "ffma": {...}, "thin": {...}, "tensor_x3": {...}}."""
+        ms, flop, cnt = (_dbl * 4)(), (_dbl * 4)(), (_i64 * 4)()
         self._check(self._lib.gn_profile_read(self._h, ms, flop, cnt))
         return {name: {"ms": ms[k], "flop": flop[k], "launches": cnt[k]}
-                for k, name in enumerate(("tensor", "ffma", "thin"))}
+                for k, name in enumerate(("tensor", "ffma", "thin", "tensor_x3"))}
 
     def debug_gemm(self, kind, A, B, a_kmajor=True, b_kmajor=True):
         """Test hook: D[M][N] from A ([M][K] or [K][M]) and B ([N][K] or [K][N]); kind 0 tensor-core, 1 FMA."""

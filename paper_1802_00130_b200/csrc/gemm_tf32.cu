@@ -717,6 +717,240 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Error-compensated variant (FP32-accurate results from the TF32 tensor cores).
+// Every operand X arrives as two matrices X = Xhi + Xlo, both exactly representable in TF32.  A logical
+// product A B is computed as Alo Bhi + Ahi Blo + Ahi Bhi (small terms first), i.e. as up to MAX_PAIRS operand
+// pairs accumulated into the same tile.  The tensor core adds into its FP32 accumulator with truncation
+// (measured: a relative bias of about 1e-9 per unit of K), so the K range is cut into chunks of
+// p.chunk_kb k-blocks; each chunk is accumulated in tensor memory on its own (the two 256-column
+// accumulators alternate per chunk) and the epilogue warps add the chunks into a running sum held in
+// registers, in FP32 with round-to-nearest.  That needs 128 registers per epilogue thread for the sums
+// alone, so the block has three warpgroups and moves registers between them:
+//   warps 0..3   (56 registers)   0 = TMA producer, 1 = MMA issuer, 2 = tensor-memory allocation, 3 idle
+//   warps 4..11  (224 registers)  epilogue, two warps per 32-lane quadrant of tensor memory
+// Whole tiles only, in wave order (no K slices).  Same pair protocol as the kernel above.
+constexpr int MAX_PAIRS = 6;
+constexpr int X3_THREADS = 384;
+constexpr int X3_REGS_LOW = 56, X3_REGS_HIGH = 224;   // 128 * 56 + 256 * 224 = 384 * 168
+
+struct MapSet { CUtensorMap a[MAX_PAIRS], b[MAX_PAIRS]; };
+
+struct X3Params {
+  int n_pairs;
+  int kblocks[MAX_PAIRS];
+  int chunk_kb;
+};
+
+template <int STAGES>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(X3_THREADS, 1)
+gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, const X3Params xp) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE2_BYTES);
+  uint64_t* empty = full + STAGES;
+  uint64_t* acc_full = empty + STAGES;   // [2]
+  uint64_t* acc_empty = acc_full + 2;    // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1;
+  int total_kb = 0;
+  for (int i = 0; i < xp.n_pairs; ++i) total_kb += xp.kblocks[i];
+  const int n_chunks_k = (total_kb + xp.chunk_kb - 1) / xp.chunk_kb;
+  const int bn = p.bn, hb = p.bn >> 1;
+  const uint32_t pair_tx = 2u * (A_STAGE_BYTES + (uint32_t)hb * BK * 4);
+  // tiles of this pair: pair, pair + P, ... (whole waves), then one of the `rem` left over
+  const int my_tiles = p.waves + (pair < p.rem ? 1 : 0);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 16); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(X3_REGS_LOW));
+    if (warp == 0) {
+      // ---------------------------------------------------------------- producer (both CTAs)
+      int it = 0;
+      bool ok = true;
+      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+        const int t = ti * p.P + pair;
+        const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM;
+        const int n0 = (t % p.tiles_n) * bn + (int)rank * hb;
+        int pr = 0, kk = 0;                       // operand pair and k-block inside it
+        for (int kb = 0; kb < total_kb; ++kb, ++it, ++kk) {
+          while (kk >= xp.kblocks[pr]) { kk = 0; ++pr; }
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          int good = 1;
+          if (lane == 0) good = wait_or_abort(&empty[s], ph ^ 1, abort_flag, p.err, 1) ? 1 : 0;
+          good = __shfl_sync(0xffffffffu, good, 0);
+          if (!good) { ok = false; break; }
+          if (rank == 0 && lane == 0) mbar_expect_tx(&full[s], pair_tx);
+          __syncwarp();
+          const uint32_t full_leader = map_to_cta(smem_u32(&full[s]), 0);
+          const int k0 = kk * BK;
+          const CUtensorMap* ma = &maps.a[pr];
+          const CUtensorMap* mb = &maps.b[pr];
+          uint8_t* sa = smem + s * STAGE2_BYTES;
+          uint8_t* sb = sa + A_STAGE_BYTES;
+          if (!p.a_mn) {
+            if (lane == 0) tma2_load_2d(sa, ma, k0, m0, full_leader);
+          } else {
+            if (lane == 0) tma2_load_3d(sa, ma, 0, k0, m0 / 32, full_leader);
+          }
+          if (!p.b_mn) {
+            if (lane == 8) tma2_load_2d(sb, mb, k0, n0, full_leader);
+          } else {
+            if (lane == 8) tma2_load_3d(sb, mb, 0, k0, n0 / 32, full_leader);
+          }
+        }
+      }
+    } else if (warp == 1 && rank == 0 && lane == 0) {
+      // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+      const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(p.a_mn ? 1 : 0) << 15) |
+                             ((uint32_t)(p.b_mn ? 1 : 0) << 16) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+      const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
+      const uint32_t a_step = p.a_mn ? 1024 : 32, b_step = p.b_mn ? 1024 : 32;
+      const uint32_t a_sbo = p.a_mn ? 512 : 1024, b_sbo = p.b_mn ? 512 : 1024;
+      const uint32_t a_lay = p.a_mn ? 1 : 2, b_lay = p.b_mn ? 1 : 2;
+      int it = 0, ci = 0;                          // ring position, running chunk count (accumulator phase)
+      bool ok = true;
+      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+        for (int ch = 0; ch < n_chunks_k && ok; ++ch, ++ci) {
+          const int kb0 = ch * xp.chunk_kb, kb1 = min(total_kb, kb0 + xp.chunk_kb);
+          const int buf = ci & 1;
+          const uint32_t aph = (ci >> 1) & 1;
+          ok = wait_or_abort(&acc_empty[buf], aph ^ 1, abort_flag, p.err, 4);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN_MAX);
+          for (int kb = kb0; kb < kb1; ++kb, ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (it / STAGES) & 1;
+            ok = wait_or_abort(&full[s], ph, abort_flag, p.err, 2);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t sa = smem_u32(smem + s * STAGE2_BYTES);
+            const uint32_t sb = sa + A_STAGE_BYTES;
+#pragma unroll
+            for (int k = 0; k < BK / 8; ++k) {
+              const uint64_t ad = make_desc(sa + k * a_step, a_lbo, a_sbo, a_lay);
+              const uint64_t bd = make_desc(sb + k * b_step, b_lbo, b_sbo, b_lay);
+              mma2_tf32(tmem_d, ad, bd, idesc, (kb > kb0 || k != 0) ? 1u : 0u);
+            }
+            mma2_commit_both(&empty[s]);
+          }
+          if (ok) mma2_commit_both(&acc_full[buf]);
+        }
+      }
+    }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(X3_REGS_HIGH));
+    // ------------------------------------------------------------------ epilogue (warps 4..11, both CTAs)
+    const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;
+    const int row = quad * 32 + lane;
+    int ci = 0;
+    bool alive = true;
+    for (int ti = 0; ti < my_tiles && alive; ++ti) {
+      const int t = ti * p.P + pair;
+      const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM, n0 = (t % p.tiles_n) * bn;
+      const int n_cc = min(bn / 32, (p.N - n0 + 31) / 32);       // column chunks of this tile that exist
+      float run[4][32];                                          // this warp's chunks: half, half + 2, half + 4, half + 6
+      for (int ch = 0; ch < n_chunks_k; ++ch, ++ci) {
+        const int buf = ci & 1;
+        const uint32_t aph = (ci >> 1) & 1;
+        int good = 1;
+        if (lane == 0) good = wait_or_abort(&acc_full[buf], aph, abort_flag, p.err, 3) ? 1 : 0;
+        good = __shfl_sync(0xffffffffu, good, 0);
+        if (!good) { alive = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int c = half + 2 * j;
+          if (c < n_cc) {                                        // warp-uniform
+            float v[32];
+            tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
+            // (a select, not a branch: two code paths over the 128 sums would double their registers)
+#pragma unroll
+            for (int i = 0; i < 32; ++i) run[j][i] = (ch == 0 ? 0.f : run[j][i]) + v[i];
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
+      }
+      if (!alive) break;
+      const int m = m0 + row;
+      if (m >= p.M) continue;
+      const float* zrow = p.dsig ? p.dsig + (long long)((m / p.dsig_div) % p.dsig_rows) * p.ld_dsig : nullptr;
+      const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
+      float* drow = p.D + (long long)m * p.ldd;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int c = half + 2 * j;
+        if (c >= n_cc) continue;
+        const int nb = n0 + c * 32;
+        if (p.vec_epi && nb + 32 <= p.N) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            float4 bz = make_float4(0.f, 0.f, 0.f, 0.f), zc = bz, cc = bz;
+            if (p.bias) bz = __ldg(reinterpret_cast<const float4*>(p.bias + nb) + q);
+            if (zrow) zc = __ldg(reinterpret_cast<const float4*>(zrow + nb) + q);
+            if (crow) cc = __ldg(reinterpret_cast<const float4*>(crow + nb) + q);
+            float x[4] = {run[j][4 * q] + bz.x, run[j][4 * q + 1] + bz.y, run[j][4 * q + 2] + bz.z, run[j][4 * q + 3] + bz.w};
+            const float z[4] = {zc.x, zc.y, zc.z, zc.w};
+            const float cv[4] = {cc.x, cc.y, cc.z, cc.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              if (p.sigmoid) x[e] = 1.f / (1.f + expf(-x[e]));
+              if (zrow) x[e] *= z[e] * (1.f - z[e]);
+              x[e] *= p.alpha;
+              if (crow) x[e] = fmaf(p.beta, cv[e], x[e]);
+            }
+            reinterpret_cast<float4*>(drow + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
+            // the running sums leave few registers: keep the loads of at most two steps in flight
+            if (q & 1) asm volatile("" ::: "memory");
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int n = nb + i;
+            if (n < p.N) {
+              float x = run[j][i] + (p.bias ? __ldg(p.bias + n) : 0.f);
+              if (p.sigmoid) x = 1.f / (1.f + expf(-x));
+              if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
+              x *= p.alpha;
+              if (crow) x = fmaf(p.beta, __ldg(crow + n), x);
+              drow[n] = x;
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  cluster_sync_all();
+  if (warp == 2) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
 // One CTA waits on an mbarrier that nothing ever arrives on, with the same bounded-wait code the GEMM
 // roles use but a caller-chosen limit; it must record its code and return.  Exercises the path from a
 // timed-out device wait to GN_ETIMEOUT on the host without hanging anything.
@@ -934,6 +1168,82 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
     const int grid = p.tiles < num_sms() ? p.tiles : num_sms();
     gemm_tf32_kernel<kStages><<<grid, 320, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
   }
+  return 1;
+}
+
+// ---- error-compensated form ---------------------------------------------------------------------
+// 8 k-blocks = 256 products per accumulation in tensor memory: the truncation bias of one chunk stays near 5e-7
+// relative (measured), and the running sums outside are round-to-nearest.
+constexpr int kChunkKb = 8;
+
+bool gemm_tf32x3_eligible(const GemmArgs& g) {
+  // the operands' own alignment does not matter: the kernel reads their hi / lo copies
+  return g.M > BM && g.N >= 128 && encode_fn() != nullptr;
+}
+
+int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st) {
+  static int usable = -1;
+  if (usable < 0) {
+    // the register split of the kernel (128 x 56 + 256 x 224) must not exceed what the block is launched with
+    cudaFuncAttributes fa;
+    usable = cudaFuncGetAttributes(&fa, gemm_tf32x3_kernel<kStages2>) == cudaSuccess &&
+             fa.numRegs * X3_THREADS >= 128 * X3_REGS_LOW + 256 * X3_REGS_HIGH &&
+             cudaFuncSetAttribute(gemm_tf32x3_kernel<kStages2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2) == cudaSuccess;
+    cudaGetLastError();
+  }
+  if (!usable || !g.A1lo || !g.B1lo || (g.A2 && (!g.A2lo || !g.B2lo))) return -1;
+  struct PairList {
+    const float* A[MAX_PAIRS]; const float* B[MAX_PAIRS]; int K[MAX_PAIRS]; long long lda[MAX_PAIRS], ldb[MAX_PAIRS]; int n = 0;
+    void add(const float* a, long long la, const float* b, long long lb, int k) { A[n] = a; lda[n] = la; B[n] = b; ldb[n] = lb; K[n] = k; ++n; }
+  } pl;
+  // small terms first
+  pl.add(g.A1lo, g.lda1, g.B1, g.ldb1, g.K1);
+  pl.add(g.A1, g.lda1, g.B1lo, g.ldb1, g.K1);
+  if (g.A2) {
+    pl.add(g.A2lo, g.lda2, g.B2, g.ldb2, g.K2);
+    pl.add(g.A2, g.lda2, g.B2lo, g.ldb2, g.K2);
+  }
+  pl.add(g.A1, g.lda1, g.B1, g.ldb1, g.K1);
+  if (g.A2) pl.add(g.A2, g.lda2, g.B2, g.ldb2, g.K2);
+  const int bn = choose_bn2(g.M, g.N, false);
+  const int b_rows = bn / 2;
+  MapSet maps;
+  const CUtensorMapSwizzle kmaj = CU_TENSOR_MAP_SWIZZLE_128B;
+  for (int s = 0; s < MAX_PAIRS; ++s) {
+    if (s >= pl.n) { maps.a[s] = maps.a[0]; maps.b[s] = maps.b[0]; continue; }   // never dereferenced
+    bool ok;
+    if (g.a_kmajor) ok = make_map(&maps.a[s], pl.A[s], g.M, pl.K[s], pl.lda[s], BK, BM, kmaj);
+    else            ok = make_map_mn3d(&maps.a[s], pl.A[s], pl.K[s], g.M, pl.lda[s], BM / 32);
+    if (g.b_kmajor) ok = ok && make_map(&maps.b[s], pl.B[s], g.N, pl.K[s], pl.ldb[s], BK, b_rows, kmaj);
+    else            ok = ok && make_map_mn3d(&maps.b[s], pl.B[s], pl.K[s], g.N, pl.ldb[s], b_rows / 32);
+    if (!ok) return -1;
+  }
+  Tf32Params p{};
+  X3Params xp{};
+  p.M = g.M; p.N = g.N;
+  xp.n_pairs = pl.n;
+  for (int s = 0; s < pl.n; ++s) xp.kblocks[s] = (pl.K[s] + BK - 1) / BK;
+  xp.chunk_kb = kChunkKb;
+  p.a_mn = g.a_kmajor ? 0 : 1; p.b_mn = g.b_kmajor ? 0 : 1;
+  p.a_3d = p.a_mn; p.b_3d = p.b_mn;
+  p.D = g.D; p.ldd = g.ldd;
+  p.bias = g.bias; p.sigmoid = g.sigmoid;
+  p.dsig = g.dsig; p.ld_dsig = g.ld_dsig; p.dsig_rows = g.dsig_rows > 0 ? g.dsig_rows : 1; p.dsig_div = g.dsig_div > 0 ? g.dsig_div : 1;
+  p.alpha = g.alpha;
+  p.cin = g.cin; p.ld_cin = g.ld_cin; p.beta = g.beta;
+  p.vec_epi = aligned16(g.D) && (g.ldd % 4 == 0) && (!g.bias || aligned16(g.bias)) &&
+              (!g.dsig || (aligned16(g.dsig) && g.ld_dsig % 4 == 0)) &&
+              (!g.cin || (aligned16(g.cin) && g.ld_cin % 4 == 0));
+  p.bn = bn;
+  p.tiles_n = (g.N + bn - 1) / bn;
+  p.err = err_flag;
+  p.tiles = ((g.M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;
+  const int pairs = num_sms() / 2;
+  p.P = p.tiles < pairs ? p.tiles : pairs;
+  p.waves = p.tiles / p.P;
+  p.rem = p.tiles - p.waves * p.P;
+  p.slices = 1;
+  gemm_tf32x3_kernel<kStages2><<<2 * p.P, X3_THREADS, kSmemBytes2, st>>>(maps, p, xp);
   return 1;
 }
 

@@ -56,6 +56,19 @@ struct gn_ctx {
   float* thin_scratch = nullptr; int64_t thin_cap = 0;
   float* sk_ws = nullptr; int* sk_flags = nullptr;   // stream-K workspace of the tensor-core kernel
   bool sk_enabled = true;
+  // FP32-accurate mode on the tensor cores (3 x TF32): hi / lo parts of the operands
+  int acc_method = 0;        // 0 choose (tensor cores where the shape allows), 1 FP32 FMA only, 2 as 0
+  bool x3_usable = true;     // cleared if the error-compensated kernel could not be launched
+  uint64_t theta_epoch = 1, sub_epoch = 1;   // bumped whenever theta / the stored activations are rewritten
+  struct SplitBuf { float* hi = nullptr; float* lo = nullptr; int64_t cap = 0; };
+  struct SplitEntry {        // split of a matrix that lives in theta or in the stored Z_m, kept until those change
+    const float* src; int64_t rows; int cols; int64_t ld; int kind; uint64_t epoch; SplitBuf buf;
+  };
+  std::vector<SplitEntry> split_cache;
+  struct SplitSlot {         // split of any other operand: one slot per operand role, overwritten by the next use
+    const float* src = nullptr; int64_t rows = 0; int cols = 0; int64_t ld = 0; SplitBuf buf;
+  };
+  SplitSlot split_slot[4];
   double* partial = nullptr; int64_t partial_cap = 0;
   double* dscal = nullptr;   // device: [0] loss, [1] theta^T theta, [2] cg sum rho, [3] cg active
   double* hscal = nullptr;   // pinned mirror
@@ -154,6 +167,8 @@ gn_status sync(gn_ctx* c, const char* where) {
   return GN_OK;
 }
 
+gn_status ensure_sk_workspace(gn_ctx* c);
+
 void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
   gn_ctx::EvPair* e = nullptr;
   if (c->profiling) {
@@ -169,17 +184,16 @@ void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
     }
   }
   if (kind == 0) {
-    if (!c->sk_ws && c->sk_enabled) {   // first tensor-core launch of this context: stream-K workspace
-      if (dev_alloc(c, &c->sk_ws, gemm_tf32_workspace_floats()) != GN_OK ||
-          dev_alloc(c, &c->sk_flags, (int64_t)gemm_tf32_workspace_flags()) != GN_OK) {
-        c->sk_ws = nullptr; c->sk_flags = nullptr; c->sk_enabled = false;
-      }
-    }
+    ensure_sk_workspace(c);   // first tensor-core launch of this context: stream-K workspace
     const bool sk = c->sk_enabled && g.two_cta != 2;
     GemmArgs g2 = g;
     if (g2.two_cta == 2) g2.two_cta = 1;
     const int r = launch_gemm_tf32(g2, c->err_flag + 1, sk ? c->sk_ws : nullptr, sk ? c->sk_flags : nullptr, c->st);
     if (r < 0) { c->sticky = GN_ECUDA; c->err = "cuTensorMapEncodeTiled failed"; }
+    else c->launches += r;
+  } else if (kind == 3) {
+    const int r = launch_gemm_tf32x3(g, c->err_flag + 1, c->st);
+    if (r < 0) { c->sticky = GN_ECUDA; c->err = "the error-compensated tensor-core kernel could not be launched"; c->x3_usable = false; }
     else c->launches += r;
   } else if (kind == 2) {
     c->launches += launch_gemm_thin(g, c->thin_scratch, c->st);
@@ -189,8 +203,104 @@ void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
   if (e) cudaEventRecord(e->b, c->st);
 }
 
+gn_status ensure_sk_workspace(gn_ctx* c) {
+  if (!c->sk_ws && c->sk_enabled) {
+    if (dev_alloc(c, &c->sk_ws, gemm_tf32_workspace_floats()) != GN_OK ||
+        dev_alloc(c, &c->sk_flags, (int64_t)gemm_tf32_workspace_flags()) != GN_OK) {
+      c->sk_ws = nullptr; c->sk_flags = nullptr; c->sk_enabled = false;
+    }
+  }
+  return c->sk_ws ? GN_OK : GN_ENOMEM;
+}
+
+inline int64_t round4(int64_t x) { return (x + 3) & ~(int64_t)3; }
+
+bool split_buf_reserve(gn_ctx* c, gn_ctx::SplitBuf& b, int64_t need) {
+  if (need <= b.cap) return true;
+  cudaStreamSynchronize(c->st);   // an earlier contraction may still be reading the old buffers
+  dev_free(c, b.hi, b.cap); dev_free(c, b.lo, b.cap);
+  b.cap = 0;
+  if (dev_alloc(c, &b.hi, need) != GN_OK) return false;
+  if (dev_alloc(c, &b.lo, need) != GN_OK) { dev_free(c, b.hi, need); return false; }
+  b.cap = need;
+  return true;
+}
+
+// hi / lo parts of the stored matrix [rows][cols] (leading dimension ld) that serves as an operand.  Matrices
+// inside theta or inside the stored activations Z_m are split once per set_theta / set_subsample; anything
+// else goes through the slot of its operand role (0 = A1, 1 = B1, 2 = A2, 3 = B2) and is split again on every
+// use unless the caller vouches (reuse) that the slot still holds this very operand, unchanged.
+constexpr int64_t kMaxTransientSplitFloats = 1500LL * 1000 * 1000;   // 6 GB per part
+
+bool split_operand(gn_ctx* c, const float* src, int64_t rows, int cols, int64_t ld, int role, bool reuse,
+                   const float** hi, const float** lo, int64_t* ld_out) {
+  const int64_t ldo = round4(cols);
+  *ld_out = ldo;
+  int kind = 0;
+  uint64_t epoch = 0;
+  if (src >= c->theta && src < c->theta + c->n) { kind = 1; epoch = c->theta_epoch; }
+  else {
+    for (int m = 0; m <= c->L && kind == 0; ++m)
+      if (c->Z[m] && src >= c->Z[m] && src < c->Z[m] + c->capS * c->w[m]) { kind = 2; epoch = c->sub_epoch; }
+  }
+  if (kind != 0) {
+    gn_ctx::SplitEntry* e = nullptr;
+    for (auto& x : c->split_cache)
+      if (x.src == src && x.rows == rows && x.cols == cols && x.ld == ld && x.kind == kind) { e = &x; break; }
+    if (!e) {
+      if (c->split_cache.size() >= 4096) return false;
+      gn_ctx::SplitEntry x{};
+      x.src = src; x.rows = rows; x.cols = cols; x.ld = ld; x.kind = kind; x.epoch = 0;
+      c->split_cache.push_back(x);
+      e = &c->split_cache.back();
+    }
+    if (e->epoch != epoch) {
+      if (!split_buf_reserve(c, e->buf, rows * ldo)) return false;
+      c->launches += launch_split_tf32(src, rows, cols, ld, e->buf.hi, e->buf.lo, ldo, c->st);
+      e->epoch = epoch;
+    }
+    *hi = e->buf.hi; *lo = e->buf.lo;
+    return true;
+  }
+  if (rows * ldo > kMaxTransientSplitFloats) return false;
+  gn_ctx::SplitSlot& sl = c->split_slot[role];
+  const bool same = reuse && sl.src == src && sl.rows == rows && sl.cols == cols && sl.ld == ld && sl.buf.hi;
+  if (!same) {
+    sl.src = nullptr;
+    if (!split_buf_reserve(c, sl.buf, rows * ldo)) return false;
+    c->launches += launch_split_tf32(src, rows, cols, ld, sl.buf.hi, sl.buf.lo, ldo, c->st);
+    sl.src = src; sl.rows = rows; sl.cols = cols; sl.ld = ld;
+  }
+  *hi = sl.buf.hi; *lo = sl.buf.lo;
+  return true;
+}
+
+// FP32-accurate contraction on the tensor cores: every operand as hi + lo TF32 parts, three products per
+// operand pair, accumulation in chunks (gemm_tf32.cu).  False if the problem has to go to the FP32 FMA GEMM.
+bool run_gemm_x3(gn_ctx* c, const GemmArgs& g) {
+  if (!c->x3_usable || !gemm_tf32x3_eligible(g)) return false;
+  GemmArgs h = g;
+  const float *hi = nullptr, *lo = nullptr;
+  int64_t ldo = 0;
+  // stored matrices: A is [M][K] (K-major) or [K][M]; B is [N][K] (K-major) or [K][N]
+  if (!split_operand(c, g.A1, g.a_kmajor ? g.M : g.K1, g.a_kmajor ? g.K1 : g.M, g.lda1, 0, g.a1_split_fresh, &hi, &lo, &ldo)) return false;
+  h.A1 = hi; h.A1lo = lo; h.lda1 = ldo;
+  if (!split_operand(c, g.B1, g.b_kmajor ? g.N : g.K1, g.b_kmajor ? g.K1 : g.N, g.ldb1, 1, false, &hi, &lo, &ldo)) return false;
+  h.B1 = hi; h.B1lo = lo; h.ldb1 = ldo;
+  if (g.A2) {
+    if (!split_operand(c, g.A2, g.a_kmajor ? g.M : g.K2, g.a_kmajor ? g.K2 : g.M, g.lda2, 2, false, &hi, &lo, &ldo)) return false;
+    h.A2 = hi; h.A2lo = lo; h.lda2 = ldo;
+    if (!split_operand(c, g.B2, g.b_kmajor ? g.N : g.K2, g.b_kmajor ? g.K2 : g.N, g.ldb2, 3, false, &hi, &lo, &ldo)) return false;
+    h.B2 = hi; h.B2lo = lo; h.ldb2 = ldo;
+  }
+  h.mn_padded = true;     // the parts live in context allocations, which carry slack after their last row
+  run_gemm_kind(c, h, 3);
+  return true;
+}
+
 // Kernel choice: streaming kernels for the n_L-wide shapes (both precisions: they are exact FP32),
-// the tensor-core kernel in TF32 mode when TMA can address the operands, else the FP32 FMA GEMM.
+// the tensor-core kernel in TF32 mode when TMA can address the operands and, in its error-compensated
+// form, in FP32-accurate mode when the shape suits the CTA-pair kernel; else the FP32 FMA GEMM.
 void run_gemm(gn_ctx* c, const GemmArgs& g) {
   const ThinKind thin = gemm_thin_kind(g);
   // In TF32 mode the n_L-wide forward products go to the tensor-core kernel as one 32- or 64-column
@@ -208,6 +318,7 @@ void run_gemm(gn_ctx* c, const GemmArgs& g) {
     run_gemm_kind(c, g, 2);
     return;
   }
+  if (c->prec == GN_FP32_ACCURATE && c->acc_method != 1 && run_gemm_x3(c, g)) return;
   run_gemm_kind(c, g, (c->prec == GN_TF32 && gemm_tf32_eligible(g)) ? 0 : 1);
 }
 
@@ -273,8 +384,10 @@ gn_status weight_block(gn_ctx* c, int m, const float* ds, const float* Zprev, in
 
 // Activation-space half (Eq. communi-g / communi-jaco followed by Eq. ztox-g):
 // dst = (ds W^mT) * sigma'(z^{m-1}), rows stacked modulo z_rows.
-void backward_data(gn_ctx* c, int m, const float* ds, int64_t rows, const float* Zprev, int64_t z_rows, float* dst) {
+void backward_data(gn_ctx* c, int m, const float* ds, int64_t rows, const float* Zprev, int64_t z_rows, float* dst,
+                   bool ds_just_used = false) {
   GemmArgs g;
+  g.a1_split_fresh = ds_just_used;   // the weight block of the same layer has just read these very rows of ds
   g.M = (int)rows; g.N = c->w[m - 1];
   g.A1 = ds; g.lda1 = c->w[m]; g.a_kmajor = true;
   g.B1 = Wm(c, c->theta, m); g.ldb1 = c->w[m - 1]; g.b_kmajor = false;
@@ -309,7 +422,7 @@ gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
   for (int m = L; m >= 1; --m) {
     GN_TRY(weight_block(c, m, ds, c->Z[m - 1], nS, inv, v, coef, out));
     if (m > 1) {
-      backward_data(c, m, ds, nS, c->Z[m - 1], nS, c->DS[m - 1]);
+      backward_data(c, m, ds, nS, c->Z[m - 1], nS, c->DS[m - 1], true);
       ds = c->DS[m - 1];
     }
   }
@@ -546,7 +659,7 @@ gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
         } else {
           GN_TRY(weight_block(c, m, c->Db[m], Zprev, rows, inv_l, cin0, beta0, d_grad, !(m == 1 && r0 + rows == c->l)));
         }
-        if (m > 1) backward_data(c, m, c->Db[m], rows, c->Zb[m - 1], rows, c->Db[m - 1]);
+        if (m > 1) backward_data(c, m, c->Db[m], rows, c->Zb[m - 1], rows, c->Db[m - 1], true);
       }
     }
   }
@@ -737,6 +850,13 @@ gn_status gn_set_blockdiag_method(gn_ctx* c, int method) {
   return GN_OK;
 }
 
+gn_status gn_set_accurate_method(gn_ctx* c, int method) {
+  if (!c) return GN_EINVAL;
+  if (method < 0 || method > 2) return fail(c, GN_EINVAL, "method must be 0 (choose), 1 (FP32 FMA) or 2 (3 x TF32 where the shape allows)");
+  c->acc_method = method;
+  return GN_OK;
+}
+
 gn_status gn_set_split(gn_ctx* c, const int32_t* split) {
   if (!c) return GN_EINVAL;
   if (!split) return fail(c, GN_EINVAL, "split is NULL");
@@ -771,6 +891,7 @@ gn_status gn_set_theta(gn_ctx* c, const float* d_theta) {
   if (!c) return GN_EINVAL;
   if (!d_theta) return fail(c, GN_EINVAL, "theta is NULL");
   GN_CUDA(c, cudaMemcpyAsync(c->theta, d_theta, c->n * sizeof(float), cudaMemcpyDeviceToDevice, c->st));
+  ++c->theta_epoch;
   c->have_theta = true;
   c->have_sub = false;
   return GN_OK;
@@ -780,6 +901,7 @@ gn_status gn_set_theta_host(gn_ctx* c, const float* h_theta) {
   if (!c) return GN_EINVAL;
   if (!h_theta) return fail(c, GN_EINVAL, "theta is NULL");
   GN_CUDA(c, cudaMemcpyAsync(c->theta, h_theta, c->n * sizeof(float), cudaMemcpyHostToDevice, c->st));
+  ++c->theta_epoch;
   GN_TRY(sync(c, "set_theta_host"));
   c->have_theta = true;
   c->have_sub = false;
@@ -795,6 +917,7 @@ static gn_status set_subsample_impl(gn_ctx* c, const int32_t* idx, int64_t nS, c
   c->have_sub = false;
   c->factors_valid = false;
   c->bd_count = 0;
+  ++c->sub_epoch;             // the stored activations are about to be rewritten
   if (nS > c->capS) {
     GN_TRY(sync(c, "set_subsample"));
     dev_free(c, c->idx, c->capS);
@@ -949,16 +1072,16 @@ gn_status gn_profile(gn_ctx* c, int enable) {
 gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t* gemm_launches) {
   if (!c) return GN_EINVAL;
   GN_TRY(sync(c, "profile_read"));
-  double ms[3] = {0.0, 0.0, 0.0}, flop[3] = {0.0, 0.0, 0.0};
-  int64_t cnt[3] = {0, 0, 0};
+  double ms[4] = {0.0, 0.0, 0.0, 0.0}, flop[4] = {0.0, 0.0, 0.0, 0.0};
+  int64_t cnt[4] = {0, 0, 0, 0};
   for (size_t i = 0; i < c->ev_used; ++i) {
     float t = 0.f;
-    const int k = c->ev[i].kind < 0 || c->ev[i].kind > 2 ? 1 : c->ev[i].kind;
+    const int k = c->ev[i].kind < 0 || c->ev[i].kind > 3 ? 1 : c->ev[i].kind;
     if (cudaEventElapsedTime(&t, c->ev[i].a, c->ev[i].b) == cudaSuccess) ms[k] += t;
     flop[k] += c->ev[i].flop;
     cnt[k] += 1;
   }
-  for (int k = 0; k < 3; ++k) {
+  for (int k = 0; k < 4; ++k) {
     if (gemm_ms) gemm_ms[k] = ms[k];
     if (gemm_flop) gemm_flop[k] = flop[k];
     if (gemm_launches) gemm_launches[k] = cnt[k];
@@ -971,7 +1094,7 @@ gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t
 gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* dA, int64_t lda, int a_kmajor,
                         const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd) {
   if (!c) return GN_EINVAL;
-  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 6) return fail(c, GN_EINVAL, "bad GEMM arguments");
+  if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 7) return fail(c, GN_EINVAL, "bad GEMM arguments");
   GemmArgs g;
   g.M = M; g.N = N; g.K1 = K;
   g.A1 = dA; g.lda1 = lda; g.a_kmajor = a_kmajor != 0;
@@ -980,6 +1103,11 @@ gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* d
   // kinds 3..6 are the tensor-core kernel with options: 3 = MN-major operands declared padded,
   // 4 = one CTA per tile forced, 5 = CTA pair per tile forced, 6 = as 5 without splitting tiles
   // between pairs (all with padded operands)
+  if (kind == 7) {          // error-compensated tensor-core form (3 x TF32, chunked accumulation)
+    if (!run_gemm_x3(c, g)) return fail(c, GN_EINVAL, "the error-compensated tensor-core form does not take this problem");
+    GN_TRY(check_launch(c, "debug_gemm"));
+    return sync(c, "debug_gemm");
+  }
   g.mn_padded = (kind >= 3);
   if (kind == 4) g.two_cta = 0;
   if (kind == 5) g.two_cta = 1;

@@ -22,6 +22,11 @@ struct GemmArgs {
   int M = 0, N = 0;
   const float* A1 = nullptr; const float* B1 = nullptr; int K1 = 0; int64_t lda1 = 0, ldb1 = 0;
   const float* A2 = nullptr; const float* B2 = nullptr; int K2 = 0; int64_t lda2 = 0, ldb2 = 0;
+  // Error-compensated form of the tensor-core kernel (3 x TF32): when A1lo is set, every operand X is given as
+  // X = Xhi + Xlo with both parts exactly representable in TF32 (A1, B1, A2, B2 hold the hi parts; same
+  // layouts and leading dimensions for the lo parts), and acc = sum Alo Bhi + Ahi Blo + Ahi Bhi.
+  const float* A1lo = nullptr; const float* B1lo = nullptr; const float* A2lo = nullptr; const float* B2lo = nullptr;
+  bool a1_split_fresh = false;   // caller's word that A1 is, unchanged, the A1 of the previous contraction
   bool a_kmajor = true, b_kmajor = true;
   bool mn_padded = false;  // every MN-major operand is followed by >= 128 readable bytes
   int two_cta = -1;        // tensor-core kernel: -1 choose, 0 one CTA per tile, 1 CTA pair per 256-row tile
@@ -44,6 +49,11 @@ int launch_gemm_ffma(const GemmArgs& g, cudaStream_t st);
 // gemm_tf32_workspace_flags() ints that lets the two-CTA kernel cut the tiles of its last, partial
 // wave along K over the idle CTA pairs; pass nullptr to keep whole tiles.
 bool gemm_tf32_eligible(const GemmArgs& g);
+// Error-compensated form (GemmArgs::A1lo ...): whether it takes a problem (the shape must suit the CTA-pair
+// kernel; the hi / lo parts must be 16-byte aligned with leading dimensions that are multiples of 4 and be
+// followed by >= 128 readable bytes), and its launch.  Returns launches made, or -1 if it cannot run.
+bool gemm_tf32x3_eligible(const GemmArgs& g);
+int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st);
 int64_t gemm_tf32_workspace_floats();
 int gemm_tf32_workspace_flags();
 int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st);
@@ -82,6 +92,11 @@ int launch_sum_partials(const double* partial, int count, double* out, bool accu
 
 // out[i] = a x[i] + b y[i]; out may be x or y.
 int launch_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out, cudaStream_t st);
+
+// Two-term TF32 split of a [rows][cols] matrix with leading dimension ld into hi and lo (leading dimension
+// ld_out): hi = x rounded to TF32, lo = (x - hi) rounded to TF32, so x = hi + lo up to 2^-22 |x|.
+int launch_split_tf32(const float* src, int64_t rows, int cols, int64_t ld, float* hi, float* lo, int64_t ld_out,
+                      cudaStream_t st);
 
 // Transposed copy dst[c][r] = src[r][c] (src rows x cols).
 int launch_transpose(const float* src, int rows, int cols, float* dst, cudaStream_t st);

@@ -375,6 +375,41 @@ __global__ void __launch_bounds__(256) cg_scalars_kernel(int phase, const double
   }
 }
 
+// ---- two-term TF32 split -----------------------------------------------------------------------
+__device__ __forceinline__ float round_tf32(float x) {
+  uint32_t u;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+  return __uint_as_float(u);
+}
+
+// hi = tf32(x), lo = tf32(x - hi).  x - hi is exact in FP32 (at most 13 significant bits), so the only
+// loss is the rounding of lo: |x - hi - lo| <= 2^-22 |x|.
+template <bool VEC>
+__global__ void split_tf32_kernel(const float* __restrict__ src, int64_t rows, int cols, int64_t ld,
+                                  float* __restrict__ hi, float* __restrict__ lo, int64_t ld_out) {
+  const int per_row = VEC ? cols / 4 : cols;
+  const int64_t total = rows * per_row;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / per_row;
+    const int cidx = (int)(i - r * per_row);
+    if (VEC) {
+      const float4 x = __ldg(reinterpret_cast<const float4*>(src + r * ld) + cidx);
+      float4 h, l;
+      h.x = round_tf32(x.x); l.x = round_tf32(x.x - h.x);
+      h.y = round_tf32(x.y); l.y = round_tf32(x.y - h.y);
+      h.z = round_tf32(x.z); l.z = round_tf32(x.z - h.z);
+      h.w = round_tf32(x.w); l.w = round_tf32(x.w - h.w);
+      reinterpret_cast<float4*>(hi + r * ld_out)[cidx] = h;
+      reinterpret_cast<float4*>(lo + r * ld_out)[cidx] = l;
+    } else {
+      const float x = __ldg(src + r * ld + cidx);
+      const float h = round_tf32(x);
+      hi[r * ld_out + cidx] = h;
+      lo[r * ld_out + cidx] = round_tf32(x - h);
+    }
+  }
+}
+
 }  // namespace
 
 int launch_gather_rows(const float* src, int64_t src_rows, int cols, const int32_t* idx, int64_t n_idx,
@@ -522,6 +557,19 @@ int launch_axpby(int64_t n, float a, const float* x, float b, const float* y, fl
   long long blocks = (n + 255) / 256;
   if (blocks > 148LL * 16) blocks = 148LL * 16;
   axpby_kernel<<<(unsigned)blocks, 256, 0, st>>>(n, a, x, b, y, out);
+  return 1;
+}
+
+int launch_split_tf32(const float* src, int64_t rows, int cols, int64_t ld, float* hi, float* lo, int64_t ld_out,
+                      cudaStream_t st) {
+  if (rows < 1 || cols < 1) return 0;
+  const bool vec = cols % 4 == 0 && ld % 4 == 0 && ld_out % 4 == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0 &&
+                   (reinterpret_cast<uintptr_t>(hi) & 15) == 0 && (reinterpret_cast<uintptr_t>(lo) & 15) == 0;
+  const int64_t total = rows * (vec ? cols / 4 : cols);
+  int64_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (vec) split_tf32_kernel<true><<<(int)blocks, 256, 0, st>>>(src, rows, cols, ld, hi, lo, ld_out);
+  else     split_tf32_kernel<false><<<(int)blocks, 256, 0, st>>>(src, rows, cols, ld, hi, lo, ld_out);
   return 1;
 }
 

@@ -9,7 +9,7 @@ from test_gpu_parity import TOL, dev, make_ctx, rel
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+@pytest.mark.parametrize("mode", ["fp32", "fma", "tf32"])
 def test_mnist300_products_and_gradient_on_all_rows(mode):
     p = wl.make("mnist300")
     ctx = make_ctx(p, mode)
@@ -52,7 +52,7 @@ def test_svhn1000_products_and_cg():
     ctx.close()
 
 
-@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+@pytest.mark.parametrize("mode", ["fp32", "fma", "tf32"])
 def test_mnist2000_headline_config_at_5_percent(mode):
     p = wl.make("mnist2000_5")
     ctx = make_ctx(p, mode)

@@ -34,13 +34,13 @@ def operands(M, N, K, a_k, b_k, seed):
 
 @pytest.mark.parametrize("a_k,b_k", [(True, True), (True, False), (False, True), (False, False)])
 @pytest.mark.parametrize("shape", SHAPES)
-@pytest.mark.parametrize("kind,tol", [(1, 2e-6), (0, 1e-3), (3, 1e-3), (4, 1e-3), (5, 1e-3), (6, 1e-3)])
+@pytest.mark.parametrize("kind,tol", [(1, 2e-6), (0, 1e-3), (3, 1e-3), (4, 1e-3), (5, 1e-3), (6, 1e-3), (7, 2e-6)])
 def test_gemm_layouts(ctx, kind, tol, shape, a_k, b_k):
     import torch
     import paper_1802_00130_b200 as gn
     M, N, K = shape
     A, B, ref = operands(M, N, K, a_k, b_k, seed=M + 7 * N + 13 * K)
-    if kind >= 3:      # operands with readable slack after their last row, as the library's own workspaces have
+    if 3 <= kind <= 6:      # operands with readable slack after their last row, as the library's own workspaces have
         bufA = torch.zeros(A.size + 64, dtype=torch.float32, device="cuda")
         bufB = torch.zeros(B.size + 64, dtype=torch.float32, device="cuda")
         dA = bufA[: A.size].view(A.shape).copy_(torch.from_numpy(A))
@@ -50,6 +50,9 @@ def test_gemm_layouts(ctx, kind, tol, shape, a_k, b_k):
     try:
         D = ctx.debug_gemm(kind, dA, dB, a_kmajor=a_k, b_kmajor=b_k)
     except gn.GnError as e:
+        if kind == 7:   # the error-compensated form serves the shapes of the CTA-pair kernel only (any alignment)
+            assert e.status == 1 and (M <= 128 or N < 128)
+            return
         # the tensor-core kernel refuses operands TMA cannot address (leading dimension not a multiple of 4)
         assert kind in (0, 3, 4, 5, 6) and e.status == 1
         lda, ldb = A.shape[1], B.shape[1]

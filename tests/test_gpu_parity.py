@@ -7,7 +7,9 @@ from oracle import gn_oracle as orc
 
 pytestmark = pytest.mark.gpu
 
-TOL = {"fp32": 1e-5, "tf32": 2e-3}       # relative L2, FP32-accurate / TF32 contractions
+# relative L2.  "fp32": FP32-accurate mode as it comes (error-compensated tensor-core contractions where the shape
+# allows, FP32 FMA elsewhere); "fma": the same mode with every contraction on the FP32 FMA GEMM; "tf32": TF32 mode.
+TOL = {"fp32": 1e-5, "fma": 1e-5, "tf32": 2e-3}
 
 
 def rel(a, b):
@@ -22,7 +24,9 @@ def make_ctx(p, mode="fp32"):
     dev = torch.device("cuda:0")
     X = torch.from_numpy(p["X"]).to(dev)
     Y = torch.from_numpy(p["Y"]).to(dev)
-    ctx = gn.GnContext(p["widths"], p["C"], X, Y, gn.GN_FP32_ACCURATE if mode == "fp32" else gn.GN_TF32)
+    ctx = gn.GnContext(p["widths"], p["C"], X, Y, gn.GN_TF32 if mode == "tf32" else gn.GN_FP32_ACCURATE)
+    if mode == "fma":
+        ctx.set_accurate_method(1)
     ctx.set_theta(torch.from_numpy(p["theta"]).to(dev))
     return ctx
 
@@ -35,7 +39,7 @@ def dev(a):
 SMALL = ["tiny", "ragged", "single", "mid", "binary300"]
 
 
-@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+@pytest.mark.parametrize("mode", ["fp32", "fma", "tf32"])
 @pytest.mark.parametrize("name", SMALL)
 def test_small_workloads_all_quantities(name, mode):
     p = wl.make(name)
@@ -269,6 +273,9 @@ def test_stored_factors_need_a_small_output_layer():
     assert e.value.status == 1
     with pytest.raises(gn.GnError):
         ctx.set_blockdiag_method(3)
+    with pytest.raises(gn.GnError) as e:
+        ctx.set_accurate_method(3)
+    assert e.value.status == 1
     ctx.close()
 
 
@@ -319,3 +326,32 @@ def test_sparse_initialisation_of_the_paper(mode):
     assert abs(f - orc.fun(p["theta"], w, p["C"], p["X"], p["Y"])) <= TOL[mode] * abs(f)
     assert rel(g.cpu().numpy(), orc.grad(p["theta"], w, p["C"], p["X"], p["Y"])) <= TOL[mode]
     ctx.close()
+
+
+def test_accurate_mode_methods_agree():
+    """FP32-accurate mode on the tensor cores (hi/lo TF32 parts, chunked accumulation) against the FP32 FMA GEMM:
+    both within the bound of the mode, and within twice that of each other; a new theta and a new subsample
+    refresh the cached parts."""
+    p = wl.make("mid")
+    w, C = p["widths"], p["C"]
+    outs = {}
+    for mode in ("fp32", "fma"):
+        ctx = make_ctx(p, mode)
+        ctx.set_subsample(dev(p["idx"]))
+        XS = p["X"][p["idx"]]
+        a = ctx.Gv(dev(p["v"])).cpu().numpy()
+        assert rel(a, orc.Gv(p["theta"], w, C, XS, p["v"])) <= TOL[mode]
+        # second theta, second subsample on the same context
+        rng = np.random.Generator(np.random.PCG64(7))
+        th2 = (p["theta"] * (1.0 + 0.1 * rng.standard_normal(p["n"]))).astype(np.float32)
+        ctx.set_theta(dev(th2))
+        idx2 = np.ascontiguousarray(p["idx"][::-1][: p["nS"] - 3])
+        ctx.set_subsample(dev(idx2))
+        b = ctx.Gv(dev(p["v"])).cpu().numpy()
+        assert rel(b, orc.Gv(th2, w, C, p["X"][idx2], p["v"])) <= TOL[mode]
+        g = ctx.grad().cpu().numpy()
+        assert rel(g, orc.grad(th2, w, C, p["X"], p["Y"])) <= TOL[mode]
+        outs[mode] = (a, b, g)
+        ctx.close()
+    for x, y in zip(outs["fp32"], outs["fma"]):
+        assert rel(x, y) <= 2e-5
