@@ -244,20 +244,23 @@ bool split_operand(gn_ctx* c, const float* src, int64_t rows, int cols, int64_t 
       if (c->Z[m] && src >= c->Z[m] && src < c->Z[m] + c->capS * c->w[m]) { kind = 2; epoch = c->sub_epoch; }
   }
   if (kind != 0) {
+    // one entry per start address: a matrix that comes back with another shape (a subsample of another
+    // size in the same buffers) replaces the old parts instead of adding to them
     gn_ctx::SplitEntry* e = nullptr;
     for (auto& x : c->split_cache)
-      if (x.src == src && x.rows == rows && x.cols == cols && x.ld == ld && x.kind == kind) { e = &x; break; }
+      if (x.src == src && x.kind == kind) { e = &x; break; }
     if (!e) {
       if (c->split_cache.size() >= 4096) return false;
       gn_ctx::SplitEntry x{};
-      x.src = src; x.rows = rows; x.cols = cols; x.ld = ld; x.kind = kind; x.epoch = 0;
+      x.src = src; x.kind = kind; x.epoch = 0;
       c->split_cache.push_back(x);
       e = &c->split_cache.back();
     }
-    if (e->epoch != epoch) {
+    if (e->epoch != epoch || e->rows != rows || e->cols != cols || e->ld != ld) {
+      e->epoch = 0;
       if (!split_buf_reserve(c, e->buf, rows * ldo)) return false;
       c->launches += launch_split_tf32(src, rows, cols, ld, e->buf.hi, e->buf.lo, ldo, c->st);
-      e->epoch = epoch;
+      e->rows = rows; e->cols = cols; e->ld = ld; e->epoch = epoch;
     }
     *hi = e->buf.hi; *lo = e->buf.lo;
     return true;
