@@ -53,7 +53,7 @@ struct Tf32Params {
   // pair's whole tiles (slices == 1: whole tiles, done last)
   int P, waves, rem, slices;
   float* sk_ws;          // [P][2][128][256] raw partial accumulators of the sliced tiles, slot = pair
-  int* sk_flags;         // [P] arrival counters, one per sliced tile, zeroed before the launch
+  int* sk_flags;         // [P] arrival counters, one per sliced tile; zero between launches (the kernel resets them)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -378,7 +378,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant
 //
 // Work list: with T tiles on P pairs, pair q runs tiles q, q + P, ... for the floor(T / P) full waves, so
 // that all pairs move through neighbouring tiles together (tiles of one A panel are read at the same
-// time and hit in L2).  The T mod P tiles left over are each cut along K into up to 8 slices, one per
+// time and hit in L2).  The T mod P tiles left over are each cut along K into up to 16 slices, one per
 // pair, and a pair does its slice before its whole tiles.  The pairs of a sliced tile store their raw
 // accumulators in a workspace, count themselves in on the tile's flag, wait (bounded) until all slices
 // have arrived, and then each sums one share of the tile's column chunks over all slices, in slice
@@ -618,15 +618,20 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
         __syncwarp();
         if (lane == 0) {
           mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
-          atomicAdd(p.sk_flags + pair / p.slices, 1);
+          int* flag_w = p.sk_flags + pair / p.slices;
+          atomicAdd(flag_w, 1);
           // 2. wait until the 16 warps of every slice of this tile have stored theirs
-          const volatile int* flag = p.sk_flags + pair / p.slices;
+          const volatile int* flag = flag_w;
           const int want = 16 * p.slices;
           const unsigned long long t0 = globaltimer();
           while (*flag < want) {
             if (*abort_flag || globaltimer() - t0 > WAIT_LIMIT_NS) { atomicCAS(p.err, 0, 5); *abort_flag = 1; good = 0; break; }
           }
           __threadfence();
+          // 3. count out again: the last of the tile's warps to have seen the full count puts the flag back to
+          // zero for the next launch (no memset between launches; the count only grows until then, so nobody
+          // still waiting can miss it)
+          if (good && atomicAdd(flag_w, 1) == 2 * want - 1) *reinterpret_cast<volatile int*>(flag_w) = 0;
         }
         good = __shfl_sync(0xffffffffu, good, 0);
         if (!good) break;
@@ -1068,6 +1073,7 @@ bool gemm_tf32_eligible(const GemmArgs& g) {
 }
 
 constexpr int kStages2 = 6;
+constexpr int kMaxSlices = 16;   // K slices per left-over tile
 constexpr int kSmemBytes2 = kStages2 * STAGE2_BYTES + 1024 + 256;
 
 // Two-CTA tile width (a multiple of 64 so that each CTA's half is whole 32-column chunks).  With the
@@ -1155,13 +1161,12 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
     }
     if (stream_k && p.rem > 0) {
       int sl = pairs / p.rem;
-      if (sl > 8) sl = 8;
+      if (sl > kMaxSlices) sl = kMaxSlices;
       if (sl > total_kb) sl = total_kb;
       // a slice costs a store and a re-read of the tile on top of its MMAs: not worth it for short K
       if (sl >= 2 && total_kb / sl >= 4) p.slices = sl;
     }
     if (p.waves == 0) launch_pairs = p.rem * p.slices;
-    if (p.slices >= 2) cudaMemsetAsync(sk_flags, 0, sizeof(int) * pairs, st);
     gemm_tf32_2cta_kernel<kStages2><<<2 * launch_pairs, 320, kSmemBytes2, st>>>(maps[0], maps[1], maps[2], maps[3], p);
   } else {
     p.tiles = ((g.M + BM - 1) / BM) * p.tiles_n;

@@ -161,6 +161,8 @@ gn_status sync(gn_ctx* c, const char* where) {
   if (c->h_err[1] != 0) {
     const int code = c->h_err[1];
     cudaMemsetAsync(c->err_flag + 1, 0, sizeof(int), c->st);
+    // a launch that gave up may have left arrival counts of its K-sliced tiles behind
+    if (c->sk_flags) cudaMemsetAsync(c->sk_flags, 0, sizeof(int) * gemm_tf32_workspace_flags(), c->st);
     return fail(c, GN_ETIMEOUT, std::string(where) + ": a bounded wait in the tensor-core pipeline ran out (role " +
                                     std::to_string(code) + "); results are invalid");
   }
@@ -206,7 +208,8 @@ void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
 gn_status ensure_sk_workspace(gn_ctx* c) {
   if (!c->sk_ws && c->sk_enabled) {
     if (dev_alloc(c, &c->sk_ws, gemm_tf32_workspace_floats()) != GN_OK ||
-        dev_alloc(c, &c->sk_flags, (int64_t)gemm_tf32_workspace_flags()) != GN_OK) {
+        dev_alloc(c, &c->sk_flags, (int64_t)gemm_tf32_workspace_flags()) != GN_OK ||
+        cudaMemsetAsync(c->sk_flags, 0, sizeof(int) * gemm_tf32_workspace_flags(), c->st) != cudaSuccess) {
       c->sk_ws = nullptr; c->sk_flags = nullptr; c->sk_enabled = false;
     }
   }

@@ -46,8 +46,10 @@ int launch_gemm_ffma(const GemmArgs& g, cudaStream_t st);
 // *err_flag receives a non-zero code if a bounded device-side wait ran out.  Returns launches made,
 // or -1 if a tensor map could not be encoded.
 // sk_ws / sk_flags: optional workspace of gemm_tf32_workspace_floats() floats and
-// gemm_tf32_workspace_flags() ints that lets the two-CTA kernel cut the tiles of its last, partial
-// wave along K over the idle CTA pairs; pass nullptr to keep whole tiles.
+// gemm_tf32_workspace_flags() ints that lets the two-CTA kernel cut the tiles left over after its whole
+// waves along K over the CTA pairs; pass nullptr to keep whole tiles.  The flags must be zero before the
+// first launch; every launch that completes leaves them zero again (after a launch that gave up on a
+// bounded wait they must be cleared by the caller).
 bool gemm_tf32_eligible(const GemmArgs& g);
 // Error-compensated form (GemmArgs::A1lo ...): whether it takes a problem (the shape must suit the CTA-pair
 // kernel; the hi / lo parts must be 16-byte aligned with leading dimensions that are multiples of 4 and be
