@@ -725,21 +725,24 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
 // ------------------------------------------------------------------------------------------------
 // Error-compensated variant (FP32-accurate results from the TF32 tensor cores).
 // Every operand X arrives as two matrices X = Xhi + Xlo, both exactly representable in TF32.  A logical
-// product A B is computed as Alo Bhi + Ahi Blo + Ahi Bhi (small terms first), i.e. as up to MAX_PAIRS operand
-// pairs accumulated into the same tile.  The tensor core adds into its FP32 accumulator with truncation
-// (measured: a relative bias of about 1e-9 per unit of K), so the K range is cut into chunks of
-// p.chunk_kb k-blocks; each chunk is accumulated in tensor memory on its own (the two 256-column
-// accumulators alternate per chunk) and the epilogue warps add the chunks into a running sum held in
-// registers, in FP32 with round-to-nearest.  That needs 128 registers per epilogue thread for the sums
+// product A B is computed as Alo Bhi + Ahi Blo + Ahi Bhi: a ring slot holds the hi and lo tiles of both
+// operands for one k-block (64 KB per CTA) and every K = 8 step issues the three products, small terms
+// first, so each operand byte is fetched once for three MMAs.  The tensor core adds into its FP32
+// accumulator with truncation (measured: a relative bias of about 1e-9 per unit of K in a plain TF32
+// accumulation), so the K range is cut into chunks of xp.chunk_kb k-blocks; each chunk is accumulated in
+// tensor memory on its own (the two 256-column accumulators alternate per chunk) and the epilogue warps add
+// the chunks into a running sum held in registers, in FP32 with round-to-nearest.  That needs 128 registers per epilogue thread for the sums
 // alone, so the block has three warpgroups and moves registers between them:
 //   warps 0..3   (56 registers)   0 = TMA producer, 1 = MMA issuer, 2 = tensor-memory allocation, 3 idle
 //   warps 4..11  (224 registers)  epilogue, two warps per 32-lane quadrant of tensor memory
 // Whole tiles only, in wave order (no K slices).  Same pair protocol as the kernel above.
-constexpr int MAX_PAIRS = 6;
+constexpr int MAX_PAIRS = 2;                          // logical operand pairs accumulated into one tile
 constexpr int X3_THREADS = 384;
+constexpr int X3_STAGES = 3;
+constexpr int X3_STAGE_BYTES = 2 * STAGE2_BYTES;      // 64 KB: A hi, A lo, B-half hi, B-half lo
 constexpr int X3_REGS_LOW = 56, X3_REGS_HIGH = 224;   // 128 * 56 + 256 * 224 = 384 * 168
 
-struct MapSet { CUtensorMap a[MAX_PAIRS], b[MAX_PAIRS]; };
+struct MapSet { CUtensorMap a_hi[MAX_PAIRS], a_lo[MAX_PAIRS], b_hi[MAX_PAIRS], b_lo[MAX_PAIRS]; };
 
 struct X3Params {
   int n_pairs;
@@ -752,7 +755,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(X3_THREADS, 1)
 gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, const X3Params xp) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE2_BYTES);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * X3_STAGE_BYTES);
   uint64_t* empty = full + STAGES;
   uint64_t* acc_full = empty + STAGES;   // [2]
   uint64_t* acc_empty = acc_full + 2;    // [2]
@@ -766,7 +769,7 @@ gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, cons
   for (int i = 0; i < xp.n_pairs; ++i) total_kb += xp.kblocks[i];
   const int n_chunks_k = (total_kb + xp.chunk_kb - 1) / xp.chunk_kb;
   const int bn = p.bn, hb = p.bn >> 1;
-  const uint32_t pair_tx = 2u * (A_STAGE_BYTES + (uint32_t)hb * BK * 4);
+  const uint32_t pair_tx = 4u * (A_STAGE_BYTES + (uint32_t)hb * BK * 4);   // two CTAs x (hi + lo) x (A + B half)
   // tiles of this pair: pair, pair + P, ... (whole waves), then one of the `rem` left over
   const int my_tiles = p.waves + (pair < p.rem ? 1 : 0);
 
@@ -808,19 +811,21 @@ gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, cons
           __syncwarp();
           const uint32_t full_leader = map_to_cta(smem_u32(&full[s]), 0);
           const int k0 = kk * BK;
-          const CUtensorMap* ma = &maps.a[pr];
-          const CUtensorMap* mb = &maps.b[pr];
-          uint8_t* sa = smem + s * STAGE2_BYTES;
-          uint8_t* sb = sa + A_STAGE_BYTES;
+          uint8_t* sa = smem + s * X3_STAGE_BYTES;            // A hi | A lo | B hi | B lo
+          uint8_t* sb = sa + 2 * A_STAGE_BYTES;
           if (!p.a_mn) {
-            if (lane == 0) tma2_load_2d(sa, ma, k0, m0, full_leader);
+            if (lane == 0) tma2_load_2d(sa, &maps.a_hi[pr], k0, m0, full_leader);
+            if (lane == 1) tma2_load_2d(sa + A_STAGE_BYTES, &maps.a_lo[pr], k0, m0, full_leader);
           } else {
-            if (lane == 0) tma2_load_3d(sa, ma, 0, k0, m0 / 32, full_leader);
+            if (lane == 0) tma2_load_3d(sa, &maps.a_hi[pr], 0, k0, m0 / 32, full_leader);
+            if (lane == 1) tma2_load_3d(sa + A_STAGE_BYTES, &maps.a_lo[pr], 0, k0, m0 / 32, full_leader);
           }
           if (!p.b_mn) {
-            if (lane == 8) tma2_load_2d(sb, mb, k0, n0, full_leader);
+            if (lane == 8) tma2_load_2d(sb, &maps.b_hi[pr], k0, n0, full_leader);
+            if (lane == 9) tma2_load_2d(sb + B2_STAGE_MAX, &maps.b_lo[pr], k0, n0, full_leader);
           } else {
-            if (lane == 8) tma2_load_3d(sb, mb, 0, k0, n0 / 32, full_leader);
+            if (lane == 8) tma2_load_3d(sb, &maps.b_hi[pr], 0, k0, n0 / 32, full_leader);
+            if (lane == 9) tma2_load_3d(sb + B2_STAGE_MAX, &maps.b_lo[pr], 0, k0, n0 / 32, full_leader);
           }
         }
       }
@@ -849,13 +854,17 @@ gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, cons
             ok = wait_or_abort(&full[s], ph, abort_flag, p.err, 2);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t sa = smem_u32(smem + s * STAGE2_BYTES);
-            const uint32_t sb = sa + A_STAGE_BYTES;
+            const uint32_t sa = smem_u32(smem + s * X3_STAGE_BYTES);
+            const uint32_t sb = sa + 2 * A_STAGE_BYTES;
 #pragma unroll
             for (int k = 0; k < BK / 8; ++k) {
-              const uint64_t ad = make_desc(sa + k * a_step, a_lbo, a_sbo, a_lay);
-              const uint64_t bd = make_desc(sb + k * b_step, b_lbo, b_sbo, b_lay);
-              mma2_tf32(tmem_d, ad, bd, idesc, (kb > kb0 || k != 0) ? 1u : 0u);
+              const uint64_t ah = make_desc(sa + k * a_step, a_lbo, a_sbo, a_lay);
+              const uint64_t al = make_desc(sa + A_STAGE_BYTES + k * a_step, a_lbo, a_sbo, a_lay);
+              const uint64_t bh = make_desc(sb + k * b_step, b_lbo, b_sbo, b_lay);
+              const uint64_t bl = make_desc(sb + B2_STAGE_MAX + k * b_step, b_lbo, b_sbo, b_lay);
+              mma2_tf32(tmem_d, al, bh, idesc, (kb > kb0 || k != 0) ? 1u : 0u);   // small terms first
+              mma2_tf32(tmem_d, ah, bl, idesc, 1u);
+              mma2_tf32(tmem_d, ah, bh, idesc, 1u);
             }
             mma2_commit_both(&empty[s]);
           }
@@ -1177,9 +1186,10 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
 }
 
 // ---- error-compensated form ---------------------------------------------------------------------
-// 8 k-blocks = 256 products per accumulation in tensor memory: the truncation bias of one chunk stays near 5e-7
-// relative (measured), and the running sums outside are round-to-nearest.
-constexpr int kChunkKb = 8;
+// 4 k-blocks = 128 terms (384 products) per accumulation in tensor memory: the truncation bias of one chunk stays
+// below 1e-6 relative (measured), and the running sums outside are round-to-nearest.
+constexpr int kChunkKb = 4;
+constexpr int kSmemBytes3 = X3_STAGES * X3_STAGE_BYTES + 1024 + 256;
 
 bool gemm_tf32x3_eligible(const GemmArgs& g) {
   // the operands' own alignment does not matter: the kernel reads their hi / lo copies
@@ -1191,43 +1201,38 @@ int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   if (usable < 0) {
     // the register split of the kernel (128 x 56 + 256 x 224) must not exceed what the block is launched with
     cudaFuncAttributes fa;
-    usable = cudaFuncGetAttributes(&fa, gemm_tf32x3_kernel<kStages2>) == cudaSuccess &&
+    usable = cudaFuncGetAttributes(&fa, gemm_tf32x3_kernel<X3_STAGES>) == cudaSuccess &&
              fa.numRegs * X3_THREADS >= 128 * X3_REGS_LOW + 256 * X3_REGS_HIGH &&
-             cudaFuncSetAttribute(gemm_tf32x3_kernel<kStages2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2) == cudaSuccess;
+             cudaFuncSetAttribute(gemm_tf32x3_kernel<X3_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes3) == cudaSuccess;
     cudaGetLastError();
   }
   if (!usable || !g.A1lo || !g.B1lo || (g.A2 && (!g.A2lo || !g.B2lo))) return -1;
-  struct PairList {
-    const float* A[MAX_PAIRS]; const float* B[MAX_PAIRS]; int K[MAX_PAIRS]; long long lda[MAX_PAIRS], ldb[MAX_PAIRS]; int n = 0;
-    void add(const float* a, long long la, const float* b, long long lb, int k) { A[n] = a; lda[n] = la; B[n] = b; ldb[n] = lb; K[n] = k; ++n; }
-  } pl;
-  // small terms first
-  pl.add(g.A1lo, g.lda1, g.B1, g.ldb1, g.K1);
-  pl.add(g.A1, g.lda1, g.B1lo, g.ldb1, g.K1);
-  if (g.A2) {
-    pl.add(g.A2lo, g.lda2, g.B2, g.ldb2, g.K2);
-    pl.add(g.A2, g.lda2, g.B2lo, g.ldb2, g.K2);
-  }
-  pl.add(g.A1, g.lda1, g.B1, g.ldb1, g.K1);
-  if (g.A2) pl.add(g.A2, g.lda2, g.B2, g.ldb2, g.K2);
   const int bn = choose_bn2(g.M, g.N, false);
   const int b_rows = bn / 2;
+  const float* Ah[2] = {g.A1, g.A2}; const float* Al[2] = {g.A1lo, g.A2lo};
+  const float* Bh[2] = {g.B1, g.B2}; const float* Bl[2] = {g.B1lo, g.B2lo};
+  const int Ks[2] = {g.K1, g.A2 ? g.K2 : 0};
+  const long long lda[2] = {g.lda1, g.lda2}, ldb[2] = {g.ldb1, g.ldb2};
   MapSet maps;
   const CUtensorMapSwizzle kmaj = CU_TENSOR_MAP_SWIZZLE_128B;
   for (int s = 0; s < MAX_PAIRS; ++s) {
-    if (s >= pl.n) { maps.a[s] = maps.a[0]; maps.b[s] = maps.b[0]; continue; }   // never dereferenced
-    bool ok;
-    if (g.a_kmajor) ok = make_map(&maps.a[s], pl.A[s], g.M, pl.K[s], pl.lda[s], BK, BM, kmaj);
-    else            ok = make_map_mn3d(&maps.a[s], pl.A[s], pl.K[s], g.M, pl.lda[s], BM / 32);
-    if (g.b_kmajor) ok = ok && make_map(&maps.b[s], pl.B[s], g.N, pl.K[s], pl.ldb[s], BK, b_rows, kmaj);
-    else            ok = ok && make_map_mn3d(&maps.b[s], pl.B[s], pl.K[s], g.N, pl.ldb[s], b_rows / 32);
+    const int src = Ah[s] ? s : 0;      // unused second pair: repeat the first (never dereferenced)
+    bool ok = true;
+    const float* as[2] = {Ah[src], Al[src]}; CUtensorMap* am[2] = {&maps.a_hi[s], &maps.a_lo[s]};
+    const float* bs[2] = {Bh[src], Bl[src]}; CUtensorMap* bm[2] = {&maps.b_hi[s], &maps.b_lo[s]};
+    for (int h = 0; h < 2 && ok; ++h) {
+      if (g.a_kmajor) ok = make_map(am[h], as[h], g.M, Ks[src], lda[src], BK, BM, kmaj);
+      else            ok = make_map_mn3d(am[h], as[h], Ks[src], g.M, lda[src], BM / 32);
+      if (g.b_kmajor) ok = ok && make_map(bm[h], bs[h], g.N, Ks[src], ldb[src], BK, b_rows, kmaj);
+      else            ok = ok && make_map_mn3d(bm[h], bs[h], Ks[src], g.N, ldb[src], b_rows / 32);
+    }
     if (!ok) return -1;
   }
   Tf32Params p{};
   X3Params xp{};
   p.M = g.M; p.N = g.N;
-  xp.n_pairs = pl.n;
-  for (int s = 0; s < pl.n; ++s) xp.kblocks[s] = (pl.K[s] + BK - 1) / BK;
+  xp.n_pairs = g.A2 ? 2 : 1;
+  for (int s = 0; s < xp.n_pairs; ++s) xp.kblocks[s] = (Ks[s] + BK - 1) / BK;
   xp.chunk_kb = kChunkKb;
   p.a_mn = g.a_kmajor ? 0 : 1; p.b_mn = g.b_kmajor ? 0 : 1;
   p.a_3d = p.a_mn; p.b_3d = p.b_mn;
@@ -1248,7 +1253,7 @@ int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   p.waves = p.tiles / p.P;
   p.rem = p.tiles - p.waves * p.P;
   p.slices = 1;
-  gemm_tf32x3_kernel<kStages2><<<2 * p.P, X3_THREADS, kSmemBytes2, st>>>(maps, p, xp);
+  gemm_tf32x3_kernel<X3_STAGES><<<2 * p.P, X3_THREADS, kSmemBytes3, st>>>(maps, p, xp);
   return 1;
 }
 
