@@ -127,9 +127,11 @@ gn_status gn_set_blockdiag_method(gn_ctx* ctx, int method);
  *   2  same as 0.
  * Error-compensated form: every operand X is split into X = Xhi + Xlo, both exactly representable in TF32
  * (|X - Xhi - Xlo| <= 2^-22 |X|); the product is Alo Bhi + Ahi Blo + Ahi Bhi accumulated in FP32, with the sum over k
- * cut into chunks of 1024 that are added in FP32 round-to-nearest outside the tensor core (its own accumulator
+ * cut into chunks of 128 terms that are added in FP32 round-to-nearest outside the tensor core (its own accumulator
  * truncates).  Splits of theta and of the stored activations are kept until set_theta / set_subsample; they
- * double the memory those take.  No effect on GN_TF32 contexts.  GN_EINVAL for another value.
+ * double the memory those take.  If the kernel cannot be launched on this device or a split buffer cannot be
+ * allocated, the contraction runs on the FP32 FMA GEMM instead.  No effect on GN_TF32 contexts.  GN_EINVAL for
+ * another value.
  */
 gn_status gn_set_accurate_method(gn_ctx* ctx, int method);
 

@@ -626,6 +626,7 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
           const unsigned long long t0 = globaltimer();
           while (*flag < want) {
             if (*abort_flag || globaltimer() - t0 > WAIT_LIMIT_NS) { atomicCAS(p.err, 0, 5); *abort_flag = 1; good = 0; break; }
+            __nanosleep(200);   // sixteen warps per pair poll the same word: keep them off the L2 while the pair's MMAs run
           }
           __threadfence();
           // 3. count out again: the last of the tile's warps to have seen the full count puts the flag back to
@@ -1191,21 +1192,28 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
 constexpr int kChunkKb = 4;
 constexpr int kSmemBytes3 = X3_STAGES * X3_STAGE_BYTES + 1024 + 256;
 
-bool gemm_tf32x3_eligible(const GemmArgs& g) {
-  // the operands' own alignment does not matter: the kernel reads their hi / lo copies
-  return g.M > BM && g.N >= 128 && encode_fn() != nullptr;
-}
-
-int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st) {
+// The register split of the kernel (128 x 56 + 256 x 224) must not exceed what the block is launched with, and
+// the kernel needs its dynamic shared memory granted: checked once.
+bool gemm_tf32x3_usable() {
   static int usable = -1;
   if (usable < 0) {
-    // the register split of the kernel (128 x 56 + 256 x 224) must not exceed what the block is launched with
     cudaFuncAttributes fa;
-    usable = cudaFuncGetAttributes(&fa, gemm_tf32x3_kernel<X3_STAGES>) == cudaSuccess &&
+    usable = encode_fn() != nullptr &&
+             cudaFuncGetAttributes(&fa, gemm_tf32x3_kernel<X3_STAGES>) == cudaSuccess &&
              fa.numRegs * X3_THREADS >= 128 * X3_REGS_LOW + 256 * X3_REGS_HIGH &&
              cudaFuncSetAttribute(gemm_tf32x3_kernel<X3_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes3) == cudaSuccess;
     cudaGetLastError();
   }
+  return usable != 0;
+}
+
+bool gemm_tf32x3_eligible(const GemmArgs& g) {
+  // the operands' own alignment does not matter: the kernel reads their hi / lo copies
+  return g.M > BM && g.N >= 128 && gemm_tf32x3_usable();
+}
+
+int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st) {
+  const bool usable = gemm_tf32x3_usable();
   if (!usable || !g.A1lo || !g.B1lo || (g.A2 && (!g.A2lo || !g.B2lo))) return -1;
   const int bn = choose_bn2(g.M, g.N, false);
   const int b_rows = bn / 2;
