@@ -182,14 +182,26 @@ __global__ void __launch_bounds__(256) gemm_thin_m_partial_kernel(const ThinMPar
   }
 }
 
+// One block per 32 consecutive elements of the [M][N] result (lane = element); warp w adds chunks w, w + 8, ...
+// and the eight warp sums are added in warp order: a fixed order, and eight short chains instead of one long one.
 __global__ void __launch_bounds__(256) gemm_thin_m_final_kernel(const float* __restrict__ scratch, int chunks, int M, int N,
                                                                 const Epi e) {
-  const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (i >= (long long)M * N) return;
-  const int m = (int)(i / N), n = (int)(i % N);
+  __shared__ float sh[8][33];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const long long total = (long long)M * N;
+  const long long i = (long long)blockIdx.x * 32 + lane;
   float s = 0.f;
-  for (int c = 0; c < chunks; ++c) s += scratch[((long long)c * M + m) * N + n];
-  e.D[(long long)m * e.ldd + n] = apply_epi(e, s, m, n);
+  if (i < total)
+    for (int c = w; c < chunks; c += 8) s += __ldg(scratch + (long long)c * total + i);
+  sh[w][lane] = s;
+  __syncthreads();
+  if (w == 0 && i < total) {
+    float t = sh[0][lane];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) t += sh[k][lane];
+    const int m = (int)(i / N), n = (int)(i % N);
+    e.D[(long long)m * e.ldd + n] = apply_epi(e, t, m, n);
+  }
 }
 
 // ------------------------------------------------------------------------------------ thin-K
@@ -334,7 +346,7 @@ int launch_gemm_thin(const GemmArgs& g, float* scratch, cudaStream_t st) {
     else if (g.M <= 12) gemm_thin_m_partial_kernel<12><<<grid, 256, 0, st>>>(p);
     else gemm_thin_m_partial_kernel<16><<<grid, 256, 0, st>>>(p);
     const long long total = (long long)g.M * g.N;
-    gemm_thin_m_final_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(scratch, used, g.M, g.N, make_epi(g));
+    gemm_thin_m_final_kernel<<<(unsigned)((total + 31) / 32), 256, 0, st>>>(scratch, used, g.M, g.N, make_epi(g));
     return 2;
   }
   if (kind == THIN_K) {

@@ -117,16 +117,27 @@ __global__ void __launch_bounds__(256) colsum_partial_vec_kernel(const float* __
   }
 }
 
+// One block per 32 columns (lane = column); warp w adds parts w, w + 8, ... and the eight warp sums are added
+// in warp order.  Double precision, fixed order; eight short chains instead of one long one per column.
 __global__ void __launch_bounds__(256) colsum_final_kernel(const float* __restrict__ scratch, int n_parts, int cols,
                                                            float alpha, const float* __restrict__ cin, float beta,
                                                            float* __restrict__ out) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= cols) return;
+  __shared__ double sh[8][33];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + lane;
   double s = 0.0;
-  for (int k = 0; k < n_parts; ++k) s += (double)scratch[(long long)k * cols + c];
-  float v = alpha * (float)s;
-  if (cin) v = fmaf(beta, cin[c], v);
-  out[c] = v;
+  if (c < cols)
+    for (int k = w; k < n_parts; k += 8) s += (double)__ldg(scratch + (long long)k * cols + c);
+  sh[w][lane] = s;
+  __syncthreads();
+  if (w == 0 && c < cols) {
+    double t = sh[0][lane];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) t += sh[k][lane];
+    float v = alpha * (float)t;
+    if (cin) v = fmaf(beta, cin[c], v);
+    out[c] = v;
+  }
 }
 
 // ---------------------------------------------------------------------------------- loss
@@ -439,7 +450,7 @@ int launch_colsum(const float* A, int64_t rows, int cols, int64_t lda, float alp
     dim3 grid((cols + 31) / 32, parts);
     colsum_partial_kernel<<<grid, 256, 0, st>>>(A, rows, cols, lda, scratch);
   }
-  colsum_final_kernel<<<(cols + 255) / 256, 256, 0, st>>>(scratch, parts, cols, alpha, cin, beta, out);
+  colsum_final_kernel<<<(cols + 31) / 32, 256, 0, st>>>(scratch, parts, cols, alpha, cin, beta, out);
   return 2;
 }
 
