@@ -33,9 +33,9 @@ UNIT = "matvec/s"
 FP32_LANES_PER_SM, SMS = 128, 148
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant GEMM kernel, averaged over the
 # launches of one step (profiles/tf32_path_mnist2000_20_launches.md); unknown (None) for other cases
-TRAFFIC = {("tf32", "mnist2000_20"): {"bytes_per_launch": 292.7e6, "kernel": "gemm_tf32_2cta_kernel",
+TRAFFIC = {("tf32", "mnist2000_20"): {"bytes_per_launch": 299.2e6, "kernel": "gemm_tf32_2cta_kernel",
                                       "source": "profiles/tf32_path_mnist2000_20_launches.md"},
-           ("fp32", "mnist2000_20"): {"bytes_per_launch": 561.9e6, "kernel": "gemm_tf32x3_kernel",
+           ("fp32", "mnist2000_20"): {"bytes_per_launch": 561.7e6, "kernel": "gemm_tf32x3_kernel",
                                       "source": "profiles/fp32_path_mnist2000_20_launches.md"}}
 
 

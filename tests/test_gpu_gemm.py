@@ -79,3 +79,18 @@ def test_streaming_kernels_for_thin_shapes(ctx, M, N, K, a_k, b_k):
     err = np.linalg.norm(D.cpu().numpy() - ref) / np.linalg.norm(ref)
     assert err <= 2e-6, err
     assert np.max(np.abs(D.cpu().numpy() - ref)) <= 1e-4 * np.sqrt(K)
+
+
+def test_error_compensated_form_at_long_k_with_one_signed_terms(ctx):
+    """All products positive and K = 40000: the worst case for an accumulator that truncates.  The chunked
+    accumulation must keep the result within 2e-6 of float64 with no drift towards zero worth speaking of."""
+    import torch
+    rng = np.random.Generator(np.random.PCG64(77))
+    M, N, K = 256, 256, 40000
+    A = rng.uniform(0.05, 1.0, (K, M)).astype(np.float32)          # [K][M] and [K][N]: the weight-block layout
+    B = rng.uniform(0.05, 1.0, (K, N)).astype(np.float32)
+    ref = A.astype(np.float64).T @ B.astype(np.float64)
+    D = ctx.debug_gemm(7, torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), a_kmajor=False, b_kmajor=False)
+    D = D.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(D - ref) / np.linalg.norm(ref) <= 2e-6
+    assert abs(np.mean(D - ref)) / np.mean(ref) <= 1.5e-6
