@@ -926,6 +926,16 @@ static gn_status set_subsample_impl(gn_ctx* c, const int32_t* idx, int64_t nS, c
   ++c->sub_epoch;             // the stored activations are about to be rewritten
   if (nS > c->capS) {
     GN_TRY(sync(c, "set_subsample"));
+    // the stored activations move: the hi / lo parts kept for matrices inside the old buffers go with them
+    for (size_t i = 0; i < c->split_cache.size();) {
+      if (c->split_cache[i].kind == 2) {
+        dev_free(c, c->split_cache[i].buf.hi, c->split_cache[i].buf.cap);
+        dev_free(c, c->split_cache[i].buf.lo, c->split_cache[i].buf.cap);
+        c->split_cache.erase(c->split_cache.begin() + (long)i);
+      } else {
+        ++i;
+      }
+    }
     dev_free(c, c->idx, c->capS);
     for (int m = 0; m <= c->L; ++m) dev_free(c, c->Z[m], c->capS * c->w[m]);
     for (int m = 1; m <= c->L; ++m) { dev_free(c, c->RZ[m], m * c->capS * c->w[m]); dev_free(c, c->DS[m], m * c->capS * c->w[m]); }

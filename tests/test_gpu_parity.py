@@ -355,3 +355,25 @@ def test_accurate_mode_methods_agree():
         ctx.close()
     for x, y in zip(outs["fp32"], outs["fma"]):
         assert rel(x, y) <= 2e-5
+
+
+def test_accurate_mode_regrows_its_operand_parts_with_the_subsample():
+    """A larger subsample after a smaller one moves the stored activations; the hi/lo parts cached for the old
+    buffers must be dropped (no stale parts, no memory left behind)."""
+    p = wl.make("mid")
+    w, C = p["widths"], p["C"]
+    v = dev(p["v"])
+    small = np.ascontiguousarray(p["idx"][: p["nS"] // 2])
+    ctx = make_ctx(p, "fp32")
+    ctx.set_subsample(dev(small))
+    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], w, C, p["X"][small], p["v"])) <= TOL["fp32"]
+    ctx.set_subsample(dev(p["idx"]))
+    ref = orc.Gv(p["theta"], w, C, p["X"][p["idx"]], p["v"])
+    assert rel(ctx.Gv(v).cpu().numpy(), ref) <= TOL["fp32"]
+    grown = ctx.workspace_bytes
+    ctx.close()
+    fresh = make_ctx(p, "fp32")
+    fresh.set_subsample(dev(p["idx"]))
+    assert rel(fresh.Gv(v).cpu().numpy(), ref) <= TOL["fp32"]
+    assert grown <= fresh.workspace_bytes
+    fresh.close()
