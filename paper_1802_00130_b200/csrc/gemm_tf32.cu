@@ -1089,7 +1089,7 @@ constexpr int kSmemBytes2 = kStages2 * STAGE2_BYTES + 1024 + 256;
 // Two-CTA tile width (a multiple of 64 so that each CTA's half is whole 32-column chunks).  With the
 // work split evenly over the pairs (stream-K) only the padding of N to whole tiles costs anything;
 // without it the number of waves decides as well.
-int choose_bn2(int M, int N, bool stream_k) {
+int choose_bn2(int M, int N, bool stream_k, int fixed_cost = 320) {
   const long long tiles_m = (M + 2 * BM - 1) / (2 * BM);
   const int pairs = num_sms() / 2;
   int best = 256;
@@ -1097,7 +1097,7 @@ int choose_bn2(int M, int N, bool stream_k) {
   for (int bn = 256; bn >= 128; bn -= 64) {
     const long long tiles_n = (N + bn - 1) / bn;
     const long long tiles = tiles_m * tiles_n;
-    const long long cost = (stream_k ? tiles_n : (tiles + pairs - 1) / pairs) * (320 + bn);
+    const long long cost = (stream_k ? tiles_n : (tiles + pairs - 1) / pairs) * (fixed_cost + bn);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
   }
   return best;
@@ -1215,7 +1215,9 @@ bool gemm_tf32x3_eligible(const GemmArgs& g) {
 int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   const bool usable = gemm_tf32x3_usable();
   if (!usable || !g.A1lo || !g.B1lo || (g.A2 && (!g.A2lo || !g.B2lo))) return -1;
-  const int bn = choose_bn2(g.M, g.N, false);
+  // this kernel is bound by its MMAs, not by the operand feed: a tile's time is nearly proportional to its width
+  // (measured: 96 + bn units against the TF32 kernel's 320 + bn), so narrower tiles win more often
+  const int bn = choose_bn2(g.M, g.N, false, 96);
   const int b_rows = bn / 2;
   const float* Ah[2] = {g.A1, g.A2}; const float* Al[2] = {g.A1lo, g.A2lo};
   const float* Bh[2] = {g.B1, g.B2}; const float* Bl[2] = {g.B1lo, g.B2lo};
