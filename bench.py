@@ -35,7 +35,7 @@ FP32_LANES_PER_SM, SMS = 128, 148
 # launches of one step (profiles/tf32_path_mnist2000_20_launches.md); unknown (None) for other cases
 TRAFFIC = {("tf32", "mnist2000_20"): {"bytes_per_launch": 299.2e6, "kernel": "gemm_tf32_2cta_kernel",
                                       "source": "profiles/tf32_path_mnist2000_20_launches.md"},
-           ("fp32", "mnist2000_20"): {"bytes_per_launch": 561.7e6, "kernel": "gemm_tf32x3_kernel",
+           ("fp32", "mnist2000_20"): {"bytes_per_launch": 580.5e6, "kernel": "gemm_tf32x3_kernel",
                                       "source": "profiles/fp32_path_mnist2000_20_launches.md"}}
 
 
