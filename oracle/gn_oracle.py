@@ -263,14 +263,15 @@ def Gv_blockdiag(theta, widths, C, XS, v):
 
 
 # --------------------------------------------------------------------------- CG
-def cg(matvec, g, lam, max_iter, tol, segments=None):
+def cg(matvec, g, lam, max_iter, tol, segments=None, keep_iterates=True):
     """Conjugate gradient on (A + lam I) d = -g, d_0 = 0, no preconditioner.
 
     Stop rule of Eq. (CG-stopping-cond): ||(A + lam I) d + g|| <= tol ||g|| (the left side
     is the CG residual norm) or `max_iter` steps.  `segments` (list of slices) runs the
     independent systems of Eq. (p-linear) side by side: every scalar is per segment and a
     segment that met its stop rule is frozen.  Returns (d, iterates, resnorms) where
-    resnorms[k][s] is segment s's residual norm after k steps.
+    resnorms[k][s] is segment s's residual norm after k steps (iterates stays empty when
+    `keep_iterates` is False: at the largest networks fifty copies of d do not fit).
     """
     g = np.asarray(g, dtype=np.float64)
     if segments is None:
@@ -299,7 +300,8 @@ def cg(matvec, g, lam, max_iter, tol, segments=None):
             if tol > 0 and np.sqrt(rho_new) <= tol * gnorm[k]:
                 active[k] = False
         it += 1
-        iterates.append(d.copy())
+        if keep_iterates:
+            iterates.append(d.copy())
         resnorms.append(np.sqrt(rho.copy()))
     return d, iterates, resnorms
 
@@ -430,7 +432,8 @@ def cg_partitioned(theta, widths, C, XS, g, lam, split, max_iter, tol, cg_min=0,
             if tol > 0 and np.sqrt(rho_new) <= tol * gnorm[k]:
                 active[k] = False
         it += 1
-        iterates.append(d.copy())
+        if keep_iterates:
+            iterates.append(d.copy())
         resnorms.append(np.sqrt(rho.copy()))
     return d, iterates, resnorms
 

@@ -67,8 +67,10 @@ struct gn_ctx {
   std::vector<SplitEntry> split_cache;
   struct SplitSlot {         // split of any other operand: one slot per operand role, overwritten by the next use
     const float* src = nullptr; int64_t rows = 0; int cols = 0; int64_t ld = 0; SplitBuf buf;
+    uint64_t seq = 0;        // contraction (gemm_seq) that wrote these parts
   };
   SplitSlot split_slot[4];
+  uint64_t gemm_seq = 0;     // counts contractions (run_gemm calls)
   double* partial = nullptr; int64_t partial_cap = 0;
   double* dscal = nullptr;   // device: [0] loss, [1] theta^T theta, [2] cg sum rho, [3] cg active
   double* hscal = nullptr;   // pinned mirror
@@ -232,7 +234,9 @@ bool split_buf_reserve(gn_ctx* c, gn_ctx::SplitBuf& b, int64_t need) {
 // hi / lo parts of the stored matrix [rows][cols] (leading dimension ld) that serves as an operand.  Matrices
 // inside theta or inside the stored activations Z_m are split once per set_theta / set_subsample; anything
 // else goes through the slot of its operand role (0 = A1, 1 = B1, 2 = A2, 3 = B2) and is split again on every
-// use unless the caller vouches (reuse) that the slot still holds this very operand, unchanged.
+// use unless the caller vouches (reuse) that the contraction just before this one read this very operand,
+// unchanged.  The caller's word is checked: the parts are taken over only if that previous contraction is
+// the one that wrote the slot (it may have gone to another kernel and left the slot alone).
 constexpr int64_t kMaxTransientSplitFloats = 1500LL * 1000 * 1000;   // 6 GB per part
 
 bool split_operand(gn_ctx* c, const float* src, int64_t rows, int cols, int64_t ld, int role, bool reuse,
@@ -270,13 +274,15 @@ bool split_operand(gn_ctx* c, const float* src, int64_t rows, int cols, int64_t 
   }
   if (rows * ldo > kMaxTransientSplitFloats) return false;
   gn_ctx::SplitSlot& sl = c->split_slot[role];
-  const bool same = reuse && sl.src == src && sl.rows == rows && sl.cols == cols && sl.ld == ld && sl.buf.hi;
+  const bool same = reuse && sl.seq != 0 && sl.seq + 1 == c->gemm_seq && sl.src == src && sl.rows == rows &&
+                    sl.cols == cols && sl.ld == ld && sl.buf.hi;
   if (!same) {
-    sl.src = nullptr;
+    sl.src = nullptr; sl.seq = 0;
     if (!split_buf_reserve(c, sl.buf, rows * ldo)) return false;
     c->launches += launch_split_tf32(src, rows, cols, ld, sl.buf.hi, sl.buf.lo, ldo, c->st);
     sl.src = src; sl.rows = rows; sl.cols = cols; sl.ld = ld;
   }
+  sl.seq = c->gemm_seq;
   *hi = sl.buf.hi; *lo = sl.buf.lo;
   return true;
 }
@@ -308,6 +314,7 @@ bool run_gemm_x3(gn_ctx* c, const GemmArgs& g) {
 // the tensor-core kernel in TF32 mode when TMA can address the operands and, in its error-compensated
 // form, in FP32-accurate mode when the shape suits the CTA-pair kernel; else the FP32 FMA GEMM.
 void run_gemm(gn_ctx* c, const GemmArgs& g) {
+  ++c->gemm_seq;
   const ThinKind thin = gemm_thin_kind(g);
   // In TF32 mode the n_L-wide forward products go to the tensor-core kernel as one 32- or 64-column
   // tile: TMA streams A about 2.5x faster than the SIMT streaming kernel does (measured).
@@ -1120,6 +1127,7 @@ gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* d
   // 4 = one CTA per tile forced, 5 = CTA pair per tile forced, 6 = as 5 without splitting tiles
   // between pairs (all with padded operands)
   if (kind == 7) {          // error-compensated tensor-core form (3 x TF32, chunked accumulation)
+    ++c->gemm_seq;
     if (!run_gemm_x3(c, g)) return fail(c, GN_EINVAL, "the error-compensated tensor-core form does not take this problem");
     GN_TRY(check_launch(c, "debug_gemm"));
     return sync(c, "debug_gemm");

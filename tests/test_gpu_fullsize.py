@@ -4,7 +4,7 @@ import pytest
 
 import gn_workloads as wl
 from oracle import gn_oracle as orc
-from test_gpu_parity import TOL, dev, make_ctx, rel
+from test_gpu_parity import TOL, dev, make_ctx, rel, relb
 
 pytestmark = pytest.mark.gpu
 
@@ -16,39 +16,65 @@ def test_mnist300_products_and_gradient_on_all_rows(mode):
     ctx.set_subsample(dev(p["idx"]))
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
+    assert relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"]), p["widths"]) <= TOL[mode]
     ref_b = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])
     for method in (1, 2):                  # propagate form, then the stored Jacobian factors
         ctx.set_blockdiag_method(method)
-        assert rel(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b) <= TOL[mode], method
+        assert relb(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b, p["widths"]) <= TOL[mode], method
     g, f = ctx.grad(with_f=True)
     assert abs(f - orc.fun(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL[mode] * abs(f)
-    assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL[mode]
+    assert relb(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]), p["widths"]) <= TOL[mode]
     ctx.close()
 
 
 def test_svhn1000_products_and_cg():
+    from test_oracle_cg_sensitivity import AMPLIFICATION_BOUND
     p = wl.make("svhn1000", l=5000)          # all 2500 subsample rows, fewer rows for f / grad
     ctx = make_ctx(p)
     ctx.set_subsample(dev(p["idx"]))
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
-    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
-               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
+    product_error = relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"]), p["widths"])
+    assert product_error <= 1.5e-6           # far inside the 1e-5 of the mode; the CG bound below builds on it
+    assert relb(ctx.Gv_blockdiag(v).cpu().numpy(),
+               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"]), p["widths"]) <= TOL["fp32"]
     g = ctx.grad()
     g_ref = orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])
-    assert rel(g.cpu().numpy(), g_ref) <= TOL["fp32"]
-    # 20 CG steps on the full system: compare the first 10 iterates
+    assert relb(g.cpu().numpy(), g_ref, p["widths"]) <= TOL["fp32"]
+    # 20 CG steps on the full system (Eq. sample-gaussnewton): iterates 1..10 and the residual history.
+    # On this system a product error eps moves the iterates by up to AMPLIFICATION_BOUND * eps from the third step
+    # on (tests/test_oracle_cg_sensitivity.py shows it with the checker alone), so the 1e-4 that holds on the small
+    # configurations is out of reach of any FP32 product here; the bound is that factor times the error asserted above.
+    bound = AMPLIFICATION_BOUND * 1.5e-6
     g32 = g_ref.astype(np.float32)
-    _, its_ref, _ = orc.cg_solve(p["theta"], p["widths"], p["C"], XS, g32, 1.0, False, 10, 0.0)
+    _, its_ref, res_ref = orc.cg_solve(p["theta"], p["widths"], p["C"], XS, g32, 1.0, False, 20, 0.0)
     d, its, res, iterates = ctx.cg_solve(dev(g32), 1.0, blockdiag=False, max_iter=20, tol=0.0, keep_iterates=True)
-    assert its == 20
-    # FP32 products perturb the CG scalars; on this system (condition number ~1e3 at lambda = 1) the
-    # iterates follow the float64 ones to ~3e-4, the tiny configuration (test_gpu_parity) to 1e-4
+    assert its == 20 == len(its_ref)
     for k in range(10):
-        assert rel(iterates[k].cpu().numpy(), its_ref[k]) <= 1e-3
-    assert res[-1] < 1e-4 * res[0]          # residual norms are not monotone in CG, but it has converged
+        assert rel(iterates[k].cpu().numpy(), its_ref[k]) <= (1e-4 if k < 2 else bound), k
+    # r_k = -g - A d_k: an iterate that is off by `bound` relative moves the residual by at most about bound * ||g||
+    tot = [float(r[0]) for r in res_ref]
+    for k in range(21):
+        assert abs(res[k] - tot[k]) <= 1e-3 * tot[k] + bound * tot[0], k
+    assert res[20] < 1e-4 * res[0]
+    ctx.close()
+
+
+@pytest.mark.parametrize("mode", ["tf32"])
+def test_svhn1000_tf32_products_and_gradient(mode):
+    p = wl.make("svhn1000", l=5000)
+    ctx = make_ctx(p, mode)
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    v = dev(p["v"])
+    assert relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"]), p["widths"]) <= TOL[mode]
+    ref_b = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])
+    for method in (1, 2):
+        ctx.set_blockdiag_method(method)
+        assert relb(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b, p["widths"]) <= TOL[mode], method
+    g, f = ctx.grad(with_f=True)
+    assert abs(f - orc.fun(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL[mode] * abs(f)
+    assert relb(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]), p["widths"]) <= TOL[mode]
     ctx.close()
 
 
@@ -59,25 +85,63 @@ def test_mnist2000_headline_config_at_5_percent(mode):
     ctx.set_subsample(dev(p["idx"]))
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
+    assert relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"]), p["widths"]) <= TOL[mode]
     ref_b = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])
     for method in (1, 2):                  # propagate form, then the stored Jacobian factors
         ctx.set_blockdiag_method(method)
-        assert rel(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b) <= TOL[mode], method
+        assert relb(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b, p["widths"]) <= TOL[mode], method
     ctx.close()
 
 
-def test_wide4096_reduced_rows_and_properties_at_full_size():
-    import torch
-    # element-wise parity on the first 1500 subsample rows of the same recipe ...
+@pytest.fixture(scope="module")
+def wide4096_reduced():
+    """1024-4096-4096-4096-4096-100 on the first rows of its recipe (l = 4000, |S| = 1500): the checker's f, gradient,
+    full and block-diagonal products, computed once for both precision modes."""
     p = wl.make("wide4096", l=4000, nS=1500)
-    ctx = make_ctx(p)
-    ctx.set_subsample(dev(p["idx"]))
     XS = p["X"][p["idx"]]
+    th, w, C = p["theta"], p["widths"], p["C"]
+    ref = dict(f=orc.fun(th, w, C, p["X"], p["Y"]), grad=orc.grad(th, w, C, p["X"], p["Y"]),
+               Gv=orc.Gv(th, w, C, XS, p["v"]), Gvb=orc.Gv_blockdiag(th, w, C, XS, p["v"]))
+    return p, ref
+
+
+@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+def test_wide4096_reduced_rows_all_quantities(wide4096_reduced, mode):
+    p, ref = wide4096_reduced
+    ctx = make_ctx(p, mode)
+    ctx.set_subsample(dev(p["idx"]))
     v = dev(p["v"])
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL["fp32"]
-    g = ctx.grad()
-    assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= TOL["fp32"]
+    assert relb(ctx.Gv(v).cpu().numpy(), ref["Gv"], p["widths"]) <= TOL[mode]
+    # n_L = 100 rules out the stored Jacobian factors: the block-diagonal product propagates its L streams
+    assert relb(ctx.Gv_blockdiag(v).cpu().numpy(), ref["Gvb"], p["widths"]) <= TOL[mode]
+    g, f = ctx.grad(with_f=True)
+    assert abs(f - ref["f"]) <= TOL[mode] * abs(f)
+    assert relb(g.cpu().numpy(), ref["grad"], p["widths"]) <= TOL[mode]
+    ctx.close()
+
+
+def test_wide4096_fifty_cg_steps(wide4096_reduced):
+    """Eq. sample-gaussnewton with the stop rule of Eq. CG-stopping-cond switched off: 50 steps on the full system of
+    the 1024-4096-4096-4096-4096-100 network over 256 subsample rows; iterates 1..10 and all 51 residual norms."""
+    p, ref = wide4096_reduced
+    idx = np.ascontiguousarray(p["idx"][:256])
+    XS = p["X"][idx]
+    ctx = make_ctx(p)
+    ctx.set_subsample(dev(idx))
+    g32 = ref["grad"].astype(np.float32)
+    matvec = lambda x: orc.Gv(p["theta"], p["widths"], p["C"], XS, x)
+    _, its_ref, _ = orc.cg(matvec, g32, 1.0, 10, 0.0)
+    _, _, res_ref = orc.cg(matvec, g32, 1.0, 50, 0.0, keep_iterates=False)
+    _, its, _, iterates = ctx.cg_solve(dev(g32), 1.0, blockdiag=False, max_iter=10, tol=0.0, keep_iterates=True)
+    assert its == 10
+    for k in range(10):
+        assert rel(iterates[k].cpu().numpy(), its_ref[k]) <= 1e-4, k
+    del iterates
+    d, its, res = ctx.cg_solve(dev(g32), 1.0, blockdiag=False, max_iter=50, tol=0.0)
+    assert its == 50
+    tot = [float(r[0]) for r in res_ref]
+    for k in range(51):
+        assert abs(res[k] - tot[k]) <= 1e-3 * tot[k] + 1e-4 * tot[0], k
     ctx.close()
 
 
@@ -89,11 +153,11 @@ def test_bench_configuration_at_20_percent(mode):
     ctx.set_subsample(dev(p["idx"]))
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])) <= TOL[mode]
+    assert relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"]), p["widths"]) <= TOL[mode]
     ref_b = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])
     for method in (1, 2):                  # propagate form, then the stored Jacobian factors
         ctx.set_blockdiag_method(method)
-        assert rel(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b) <= TOL[mode], method
+        assert relb(ctx.Gv_blockdiag(v).cpu().numpy(), ref_b, p["widths"]) <= TOL[mode], method
     ctx.close()
 
 

@@ -18,6 +18,19 @@ def rel(a, b):
     return np.linalg.norm(a - b) / np.linalg.norm(b)
 
 
+def relb(a, b, widths):
+    """Largest relative L2 error over the whole vector and over every W^m run and every b^m run of the Section 2.1
+    layout taken apart: the bias blocks and the n_L-wide output layer come from other kernels than the large weight
+    blocks and are a fraction of a percent of the vector, so one norm over all n coordinates would hide them."""
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    worst = rel(a, b)
+    for w_off, b_off, end in wl.layer_offsets(widths):
+        for lo, hi in ((w_off, b_off), (b_off, end)):
+            worst = max(worst, rel(a[lo:hi], b[lo:hi]))
+    return worst
+
+
 def make_ctx(p, mode="fp32"):
     import torch
     import paper_1802_00130_b200 as gn
@@ -56,12 +69,12 @@ def test_small_workloads_all_quantities(name, mode):
     assert abs(f - orc.fun(th, w, C, p["X"], p["Y"])) <= TOL[mode] * abs(f)
     g, f2 = ctx.grad(with_f=True)
     assert abs(f2 - f) <= 1e-12 * abs(f)
-    assert rel(g.cpu().numpy(), orc.grad(th, w, C, p["X"], p["Y"])) <= TOL[mode]
+    assert relb(g.cpu().numpy(), orc.grad(th, w, C, p["X"], p["Y"]), p["widths"]) <= TOL[mode]
     # products
     out = ctx.Gv(dev(p["v"])).cpu().numpy()
-    assert rel(out, orc.Gv(th, w, C, XS, p["v"])) <= TOL[mode]
+    assert relb(out, orc.Gv(th, w, C, XS, p["v"]), p["widths"]) <= TOL[mode]
     outb = ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy()
-    assert rel(outb, orc.Gv_blockdiag(th, w, C, XS, p["v"])) <= TOL[mode]
+    assert relb(outb, orc.Gv_blockdiag(th, w, C, XS, p["v"]), p["widths"]) <= TOL[mode]
     ctx.close()
 
 
@@ -72,8 +85,8 @@ def test_tiny_against_explicit_jacobians():
     XS = p["X"][p["idx"]]
     a = orc.Gv_definition(p["theta"], p["widths"], p["C"], XS, p["v"])
     b = orc.Gv_blockdiag_definition(p["theta"], p["widths"], p["C"], XS, p["v"])
-    assert rel(ctx.Gv(dev(p["v"])).cpu().numpy(), a) <= 1e-5
-    assert rel(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy(), b) <= 1e-5
+    assert relb(ctx.Gv(dev(p["v"])).cpu().numpy(), a, p["widths"]) <= 1e-5
+    assert relb(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy(), b, p["widths"]) <= 1e-5
     ctx.close()
 
 
@@ -84,7 +97,7 @@ def test_row_batches_give_the_same_f_and_gradient(rows):
     ctx.set_batch_rows(rows)
     g, f = ctx.grad(with_f=True)
     assert abs(f - orc.fun(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= 1e-5 * abs(f)
-    assert rel(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"])) <= 1e-5
+    assert relb(g.cpu().numpy(), orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]), p["widths"]) <= 1e-5
     assert abs(ctx.fun() - f) <= 1e-12 * abs(f)
     ctx.close()
 
@@ -140,17 +153,17 @@ def test_degenerate_subsamples():
     # a single row
     one = np.array([5], dtype=np.int32)
     ctx.set_subsample(dev(one))
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], p["X"][one], p["v"])) <= 1e-5
+    assert relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], p["X"][one], p["v"]), p["widths"]) <= 1e-5
     # repeated rows count once per occurrence
     dup = np.array([1, 1, 4, 7, 7, 7], dtype=np.int32)
     ctx.set_subsample(dev(dup))
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], p["X"][dup], p["v"])) <= 1e-5
-    assert rel(ctx.Gv_blockdiag(v).cpu().numpy(),
-               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], p["X"][dup], p["v"])) <= 1e-5
+    assert relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], p["X"][dup], p["v"]), p["widths"]) <= 1e-5
+    assert relb(ctx.Gv_blockdiag(v).cpu().numpy(),
+               orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], p["X"][dup], p["v"]), p["widths"]) <= 1e-5
     # S = all rows, and a larger set after a smaller one (workspace regrowth)
     allrows = np.arange(p["l"], dtype=np.int32)
     ctx.set_subsample(dev(allrows))
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], p["X"], p["v"])) <= 1e-5
+    assert relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], p["X"], p["v"]), p["widths"]) <= 1e-5
     # the host-buffer entry points give the same bits as the device ones
     a = ctx.Gv(v).cpu().numpy()
     b = ctx.Gv_host(p["v"])
@@ -247,14 +260,14 @@ def test_blockdiag_methods_agree_with_the_checker_and_each_other(name, mode):
     for method in (1, 2, 0):
         ctx.set_blockdiag_method(method)
         outs.append(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy())
-        assert rel(outs[-1], ref) <= TOL[mode], method
+        assert relb(outs[-1], ref, p["widths"]) <= TOL[mode], method
     assert rel(outs[0], outs[1]) <= 2 * TOL[mode]
     # a new subsample invalidates the stored factors
     ctx.set_blockdiag_method(2)
     idx2 = np.ascontiguousarray(p["idx"][::-1][: max(1, p["nS"] // 2)])
     ctx.set_subsample(dev(idx2))
     ref2 = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], p["X"][idx2], p["v"])
-    assert rel(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy(), ref2) <= TOL[mode]
+    assert relb(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy(), ref2, p["widths"]) <= TOL[mode]
     # block CG goes through the same product
     g = orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]).astype(np.float32)
     d2, _, _ = ctx.cg_solve(dev(g), 1.0, blockdiag=True, max_iter=5, tol=0.0)
@@ -291,12 +304,12 @@ def test_the_default_method_builds_factors_only_when_they_pay():
     for k in range(6):
         out = ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy()
         assert ctx.workspace_bytes == base, k
-    assert rel(out, ref) <= TOL["tf32"]
+    assert relb(out, ref, p["widths"]) <= TOL["tf32"]
     out8 = ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy()          # eighth product: factors built and used
     grown = ctx.workspace_bytes
     factor_bytes = sum(p["nS"] * p["widths"][-1] * n for n in p["widths"][1:-1]) * 4
     assert grown - base >= factor_bytes
-    assert rel(out8, ref) <= TOL["tf32"]
+    assert relb(out8, ref, p["widths"]) <= TOL["tf32"]
     ctx.close()
 
     ctx = make_ctx(p, "tf32")
@@ -320,11 +333,11 @@ def test_sparse_initialisation_of_the_paper(mode):
     ctx = make_ctx(p, mode)
     ctx.set_subsample(dev(p["idx"]))
     XS = p["X"][p["idx"]]
-    assert rel(ctx.Gv(dev(p["v"])).cpu().numpy(), orc.Gv(p["theta"], w, p["C"], XS, p["v"])) <= TOL[mode]
-    assert rel(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy(), orc.Gv_blockdiag(p["theta"], w, p["C"], XS, p["v"])) <= TOL[mode]
+    assert relb(ctx.Gv(dev(p["v"])).cpu().numpy(), orc.Gv(p["theta"], w, p["C"], XS, p["v"]), p["widths"]) <= TOL[mode]
+    assert relb(ctx.Gv_blockdiag(dev(p["v"])).cpu().numpy(), orc.Gv_blockdiag(p["theta"], w, p["C"], XS, p["v"]), p["widths"]) <= TOL[mode]
     g, f = ctx.grad(with_f=True)
     assert abs(f - orc.fun(p["theta"], w, p["C"], p["X"], p["Y"])) <= TOL[mode] * abs(f)
-    assert rel(g.cpu().numpy(), orc.grad(p["theta"], w, p["C"], p["X"], p["Y"])) <= TOL[mode]
+    assert relb(g.cpu().numpy(), orc.grad(p["theta"], w, p["C"], p["X"], p["Y"]), p["widths"]) <= TOL[mode]
     ctx.close()
 
 
@@ -340,7 +353,7 @@ def test_accurate_mode_methods_agree():
         ctx.set_subsample(dev(p["idx"]))
         XS = p["X"][p["idx"]]
         a = ctx.Gv(dev(p["v"])).cpu().numpy()
-        assert rel(a, orc.Gv(p["theta"], w, C, XS, p["v"])) <= TOL[mode]
+        assert relb(a, orc.Gv(p["theta"], w, C, XS, p["v"]), p["widths"]) <= TOL[mode]
         # second theta, second subsample on the same context
         rng = np.random.Generator(np.random.PCG64(7))
         th2 = (p["theta"] * (1.0 + 0.1 * rng.standard_normal(p["n"]))).astype(np.float32)
@@ -348,9 +361,9 @@ def test_accurate_mode_methods_agree():
         idx2 = np.ascontiguousarray(p["idx"][::-1][: p["nS"] - 3])
         ctx.set_subsample(dev(idx2))
         b = ctx.Gv(dev(p["v"])).cpu().numpy()
-        assert rel(b, orc.Gv(th2, w, C, p["X"][idx2], p["v"])) <= TOL[mode]
+        assert relb(b, orc.Gv(th2, w, C, p["X"][idx2], p["v"]), p["widths"]) <= TOL[mode]
         g = ctx.grad().cpu().numpy()
-        assert rel(g, orc.grad(th2, w, C, p["X"], p["Y"])) <= TOL[mode]
+        assert relb(g, orc.grad(th2, w, C, p["X"], p["Y"]), p["widths"]) <= TOL[mode]
         outs[mode] = (a, b, g)
         ctx.close()
     for x, y in zip(outs["fp32"], outs["fma"]):
@@ -366,14 +379,37 @@ def test_accurate_mode_regrows_its_operand_parts_with_the_subsample():
     small = np.ascontiguousarray(p["idx"][: p["nS"] // 2])
     ctx = make_ctx(p, "fp32")
     ctx.set_subsample(dev(small))
-    assert rel(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], w, C, p["X"][small], p["v"])) <= TOL["fp32"]
+    assert relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], w, C, p["X"][small], p["v"]), p["widths"]) <= TOL["fp32"]
     ctx.set_subsample(dev(p["idx"]))
     ref = orc.Gv(p["theta"], w, C, p["X"][p["idx"]], p["v"])
-    assert rel(ctx.Gv(v).cpu().numpy(), ref) <= TOL["fp32"]
+    assert relb(ctx.Gv(v).cpu().numpy(), ref, p["widths"]) <= TOL["fp32"]
     grown = ctx.workspace_bytes
     ctx.close()
     fresh = make_ctx(p, "fp32")
     fresh.set_subsample(dev(p["idx"]))
-    assert rel(fresh.Gv(v).cpu().numpy(), ref) <= TOL["fp32"]
+    assert relb(fresh.Gv(v).cpu().numpy(), ref, p["widths"]) <= TOL["fp32"]
     assert grown <= fresh.workspace_bytes
     fresh.close()
+
+
+@pytest.mark.parametrize("widths", [[20, 256, 64, 4], [784, 128, 64, 10], [100, 300, 100, 3]])
+def test_accurate_mode_splits_every_operand_it_contracts(widths):
+    """Networks whose weight block of a layer goes to another kernel than its activation gradient (17 <= n_m <= 128
+    under a layer of >= 128 neurons): the hi / lo parts of delta s^m that the error-compensated kernel contracts must
+    be those of this product, not the ones a previous product left behind.  Two products with different directions,
+    then ten CG steps (every step after the first would reuse stale parts)."""
+    p = wl.make_custom(widths, l=900, nS=400, C=9.0, seed=77, x="uniform", n_vec=2)
+    ctx = make_ctx(p, "fp32")
+    ctx.set_subsample(dev(p["idx"]))
+    XS = p["X"][p["idx"]]
+    th, w, C = p["theta"], p["widths"], p["C"]
+    for v in (p["vs"][0], p["vs"][1], p["vs"][0]):
+        assert relb(ctx.Gv(dev(v)).cpu().numpy(), orc.Gv(th, w, C, XS, v), w) <= 1e-5
+    g = orc.grad(th, w, C, p["X"], p["Y"]).astype(np.float32)
+    assert relb(ctx.grad().cpu().numpy(), g, w) <= 1e-5
+    _, its_ref, _ = orc.cg_solve(th, w, C, XS, g, 1.0, False, 10, 0.0)
+    _, its, _, iterates = ctx.cg_solve(dev(g), 1.0, blockdiag=False, max_iter=10, tol=0.0, keep_iterates=True)
+    assert its == 10
+    for k in range(10):
+        assert rel(iterates[k].cpu().numpy(), its_ref[k]) <= 1e-4, k
+    ctx.close()
