@@ -8,7 +8,8 @@ One step = one pass of the whole path at the 784-2000-2000-2000-10 network:
 The metric is Gauss-Newton matrix-vector products per second over whole steps (2 n_cg products per
 step); the breakdown gives the product-only rates and FLOP/s.
 
-    python bench.py --gpus N --steps K --warmup W            (N > 1: launched with torch.distributed.run)
+    python bench.py --gpus N --steps K --warmup W            (N > 1: starts N ranks under torch.distributed.run
+                                                              itself unless it already runs under one)
     python bench.py --impl reference ...                      (the float64 CPU checker on a bounded sample)
 """
 from __future__ import annotations
@@ -117,7 +118,15 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle arm
-def oracle_sample_rates(p, sample_rows, n_cg, threads_note=True):
+def step_config(args, p, world):
+    """The `config` object of the JSON line; both arms print the same keys."""
+    return {"workload": args.workload, "widths": p["widths"], "l": p["l"], "S": p["nS"], "C": p["C"], "n_cg": args.n_cg,
+            "step": "set_subsample + grad(all rows) + n_cg CG steps full + n_cg CG steps block-diagonal",
+            "l2": "per-step working set (activations of S and of the row batches) exceeds the 126 MB L2",
+            "parallelism": "replicas only" if world > 1 else "single GPU"}
+
+
+def oracle_sample_rates(p, sample_rows, n_cg):
     """Times the float64 checker on `sample_rows` rows and scales to the step's row counts."""
     from oracle import gn_oracle as orc
     rows = min(sample_rows, p["nS"])
@@ -132,6 +141,17 @@ def oracle_sample_rates(p, sample_rows, n_cg, threads_note=True):
                 Gv_per_s=rows / (t_full * p["nS"]), cpu_s=t_full + t_blk + t_grad + t_fwd)
 
 
+def oracle_one_core(p, n_cg, rows=128):
+    """The same sample with the BLAS pool held to one thread (fewer rows: one core is slow)."""
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        return None
+    with threadpool_limits(limits=1):
+        r = oracle_sample_rates(p, rows, n_cg)
+    return {"value": r["value"], "Gv_per_s": r["Gv_per_s"], "rows": r["rows"], "cores": 1}
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -144,32 +164,75 @@ def blas_threads():
 
 
 def run_reference(args):
+    """The float64 checker as it stands on the host cores: each step times one bounded row sample of the workload;
+    `value` is that rate scaled by row count to the workload's |S| and l, `ms_per_step` is the time actually spent
+    per sampled step, and `full_step_ms_extrapolated` is what a whole step would take at that rate."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     p = wl.make(args.workload)
     for _ in range(min(args.warmup, 1)):
         oracle_sample_rates(p, max(64, args.ref_rows // 8), args.n_cg)
-    vals = []
-    t0 = time.perf_counter()
+    vals, walls = [], []
     for _ in range(args.steps):
+        t0 = time.perf_counter()
         vals.append(oracle_sample_rates(p, args.ref_rows, args.n_cg))
-    dt = time.perf_counter() - t0
+        walls.append(time.perf_counter() - t0)
     v = float(np.median([x["value"] for x in vals]))
     cores = blas_threads()
-    sample = (f"{vals[0]['rows']} rows per product and per gradient pass, scaled by row count to "
-              f"|S|={p['nS']}, l={p['l']}; numpy float64")
+    sample = (f"{vals[0]['rows']} of |S|={p['nS']} rows per product and {vals[0]['rows']} of l={p['l']} rows per gradient "
+              f"pass, one of each per step; rates scaled by row count; numpy float64")
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": 1e3 * float(np.median([x["step_s"] for x in vals])),
+            "warmup": args.warmup, "ms_per_step": 1e3 * float(np.median(walls)),
+            "full_step_ms_extrapolated": 1e3 * float(np.median([x["step_s"] for x in vals])),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "widths": p["widths"], "l": p["l"], "S": p["nS"], "n_cg": args.n_cg},
-            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
-            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-            "wall_s": dt}
+            "config": step_config(args, p, 1),
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                             "one_core": oracle_one_core(p, args.n_cg)},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------------------------ GPU arm
+def free_port():
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def relaunch_with_ranks(args):
+    """`--gpus N` given to a plain `python bench.py`: start N ranks (one per GPU) under torch.distributed.run
+    with the same arguments and hand back its exit code; rank 0 of that job prints the line."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def run_dry(args):
+    """Launch / aggregation rehearsal without a GPU (`--dry-run`): the ranks join a gloo group, each pretends its
+    timed region took 10 ms x (rank + 1), and rank 0 prints what the aggregation makes of it under `dry_run`.
+    No kernel runs and no metric value is reported (`value` is null)."""
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    group = None
+    if world > 1:
+        dist.init_process_group("gloo")
+        group = dist
+        dist.barrier()
+    ms = max_over_ranks(10.0 * (rank + 1), group, torch.device("cpu"))
+    rate = whole_job_rate(2 * args.n_cg * args.steps, world, ms)
+    if group:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                          "warmup": args.warmup, "scaling": "weak", "data": "none (dry run: no kernel was launched)",
+                          "dry_run": {"ms": ms, "rate_from_pretended_times": rate, "backend": "gloo"}}))
+
+
 def run_ours(args):
     import torch
     import paper_1802_00130_b200 as gn
@@ -221,7 +284,6 @@ def run_ours(args):
     barrier()
     sampler = ClockSampler(local) if rank == 0 else None
     launches0 = ctx.kernel_launches
-    ctx.profile(True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_wall0 = time.time()
     e0.record()
@@ -231,11 +293,20 @@ def run_ours(args):
     barrier()
     t_wall1 = time.time()
     ms = e0.elapsed_time(e1)
-    prof = ctx.profile_read()
-    ctx.profile(False)
     launches = ctx.kernel_launches - launches0
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     ms = max_over_ranks(ms, dist, dev)
+    # second pass over the same K steps with a CUDA-event pair around every contraction launch (on the context's
+    # stream): per-kernel FLOP/s for the roofline.  The headline above is timed without these events.
+    ctx.profile(True)
+    e0.record()
+    for k in range(args.steps):
+        step(args.warmup + k)
+    e1.record()
+    barrier()
+    ms_profiled = e0.elapsed_time(e1)
+    prof = ctx.profile_read()
+    ctx.profile(False)
     matvecs = 2 * n_cg * args.steps * world
     value = whole_job_rate(2 * n_cg * args.steps, world, ms)
 
@@ -369,7 +440,10 @@ def run_ours(args):
                  "traffic": (TRAFFIC.get((args.mode, args.workload)) or {}).get("bytes_per_launch"),
                  "traffic_note": TRAFFIC.get((args.mode, args.workload)),
                  "launches": kern["launches"], "avg_launch_us": 1e3 * kern["ms"] / max(1, kern["launches"]),
-                 "share_of_step": kern["ms"] / ms if ms > 0 else None,
+                 "share_of_step": kern["ms"] / ms_profiled if ms_profiled > 0 else None,
+                 "timing": "CUDA events around every launch of the kernel, on its stream, in a second pass over the same "
+                           "K steps (the headline pass carries no per-launch events)",
+                 "ms_per_step_with_events": ms_profiled / args.steps,
                  "library_tf32_8192_tflops": lib_tf32,
                  "frac_of_library": achieved / lib_tf32 if (achieved and lib_tf32) else None,
                  "frac_of_nominal": achieved / 1100.0 if (achieved and args.mode == "tf32") else None,
@@ -382,15 +456,12 @@ def run_ours(args):
         cpu = {"value": r["value"], "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                "sample": f"{r['rows']} rows per product and per gradient pass ({r['cpu_s']:.1f} s of CPU work), "
                          f"scaled by row count to |S|={p['nS']}, l={p['l']}",
-               "Gv_per_s": r["Gv_per_s"]}
+               "Gv_per_s": r["Gv_per_s"], "one_core": oracle_one_core(p, n_cg)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "tf32" if args.mode == "tf32" else "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "widths": p["widths"], "l": p["l"], "S": p["nS"], "C": p["C"],
-                       "n_cg": n_cg, "step": "set_subsample + grad(all rows) + n_cg CG steps full + n_cg CG steps block-diagonal",
-                       "l2": "per-step working set (activations of S and of the row batches) exceeds the 126 MB L2",
-                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "config": step_config(args, p, world),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof, "cpu_baseline": cpu,
             "breakdown": breakdown}
     print(json.dumps(line))
@@ -412,11 +483,17 @@ def main():
     ap.add_argument("--product-reps", type=int, default=10)
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="rehearse the launch of the ranks and the aggregation over them on CPU (gloo); no kernels, no value")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(relaunch_with_ranks(args))
+    elif args.dry_run:
+        run_dry(args)
     else:
         run_ours(args)
 
