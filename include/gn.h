@@ -315,6 +315,15 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
                         int a_kmajor, const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd);
 
 /*
+ * gn_debug_option - test and measurement hook: switch a launch strategy of the context for A/B runs.
+ * option 0: independent contractions of a layer issued as one launch of the CTA-pair kernel (value 0 =
+ * one launch per contraction); option 1: cutting left-over tiles along K between CTA pairs (value 0 = whole
+ * tiles only; cannot be switched back on).  Results do not depend on option 0 beyond rounding order inside a tile
+ * (none: tiles are computed identically); GN_EINVAL for an unknown option.
+ */
+gn_status gn_debug_option(gn_ctx* ctx, int option, int value);
+
+/*
  * gn_thin_m_gemm_noalloc - D[M][N] = sum_r A[r][m] B[r][n] for M <= 16 (the shape of the output layer's
  * weight block, rows = |S| or a row batch) without a context and without allocating anything.
  * The paper has no counterpart to this call; it exists for callers that must not allocate device memory

@@ -56,6 +56,19 @@ struct Tf32Params {
   int* sk_flags;         // [P] arrival counters, one per sliced tile; zero between launches (the kernel resets them)
 };
 
+// Up to MAX_GROUP independent problems in one launch of the two-CTA kernel.  Pair q runs, problem after problem,
+// its tiles of the problem's whole waves (q, q + P, ...) and then tiles rstart[g][q] .. rstart[g][q + 1] - 1 of the
+// tiles left over after those waves; the host deals the left-over tiles so that the pairs' total loads come out even
+// (longest tiles first), which lets the short tiles of one problem fill the partial last wave of another.
+constexpr int MAX_GROUP = 3;
+constexpr int MAX_PAIRS_LAUNCH = 80;        // >= SMs / 2
+struct GroupParams {
+  int n_prob;
+  Tf32Params pr[MAX_GROUP];
+  unsigned short rstart[MAX_GROUP][MAX_PAIRS_LAUNCH + 1];
+};
+struct GroupMaps { CUtensorMap m[MAX_GROUP][4]; };   // per problem: A0, B0, A1, B1
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ unsigned long long globaltimer() {
@@ -431,14 +444,17 @@ __device__ __forceinline__ void mma2_commit_both(uint64_t* bar) {
                ::"r"(smem_u32(bar)), "h"(mask) : "memory");
 }
 
-struct Work { int tile, kb0, kb1, sliced; };
+struct Work { int prob, tile, kb0, kb1, sliced; };
 
-// idx-th piece of work of CTA pair `pair` (see Tf32Params); false when the pair has no more.
-// A pair that takes part in the K-sliced tiles does its slice FIRST: the store of the partial accumulator,
-// the wait for the other slices and the fix-up epilogue then run on the epilogue warps underneath the
+// idx-th piece of work of CTA pair `pair` (see Tf32Params and GroupParams); false when the pair has no more.
+// A single problem whose left-over tiles are cut along K: the pair does its slice FIRST; the store of the partial
+// accumulator, the wait for the other slices and the fix-up epilogue then run on the epilogue warps underneath the
 // MMAs of the pair's first whole tile instead of being exposed at the end of the kernel.
-__device__ __forceinline__ bool next_work(const Tf32Params& p, int pair, int total_kb, int idx, Work& w) {
-  if (p.slices >= 2) {
+__device__ __forceinline__ bool next_work(const GroupParams& gp, int pair, int idx, Work& w) {
+  if (gp.pr[0].slices >= 2) {                  // (only ever set for a launch with one problem)
+    const Tf32Params& p = gp.pr[0];
+    const int total_kb = p.kblocks[0] + p.kblocks[1];
+    w.prob = 0;
     if (pair < p.rem * p.slices) {
       if (idx == 0) {
         const int j = pair / p.slices, sl = pair - j * p.slices;
@@ -454,10 +470,17 @@ __device__ __forceinline__ bool next_work(const Tf32Params& p, int pair, int tot
     w.tile = idx * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0;
     return true;
   }
-  if (idx < p.waves) { w.tile = idx * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0; return true; }
-  if (idx > p.waves || pair >= p.rem) return false;
-  w.tile = p.waves * p.P + pair; w.kb0 = 0; w.kb1 = total_kb; w.sliced = 0;
-  return true;
+  for (int g = 0; g < gp.n_prob; ++g) {
+    const Tf32Params& p = gp.pr[g];
+    const int r0 = gp.rstart[g][pair], n_rem = gp.rstart[g][pair + 1] - r0;
+    if (idx < p.waves + n_rem) {
+      w.prob = g; w.kb0 = 0; w.kb1 = p.kblocks[0] + p.kblocks[1]; w.sliced = 0;
+      w.tile = idx < p.waves ? idx * p.P + pair : p.waves * p.P + r0 + (idx - p.waves);
+      return true;
+    }
+    idx -= p.waves + n_rem;
+  }
+  return false;
 }
 
 constexpr int B2_STAGE_MAX = (BN_MAX / 2) * BK * 4;          // 16 KB: this CTA's half of the B tile
@@ -465,9 +488,7 @@ constexpr int STAGE2_BYTES = A_STAGE_BYTES + B2_STAGE_MAX;   // 32 KB
 
 template <int STAGES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(320, 1)
-gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
-                      const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
-                      const Tf32Params p) {
+gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constant__ GroupParams gp) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE2_BYTES);
@@ -479,11 +500,8 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
-  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int total_kb = p.kblocks[0] + p.kblocks[1];
-  const int bn = p.bn, hb = p.bn >> 1;                       // hb: B rows staged by each CTA
-  const uint32_t pair_tx = 2u * (A_STAGE_BYTES + (uint32_t)hb * BK * 4);
-  (void)n_pairs;
+  const int pair = blockIdx.x >> 1;
+  int* const err = gp.pr[0].err;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -505,7 +523,10 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
     int it = 0;
     bool ok = true;
     Work w;
-    for (int wi = 0; ok && next_work(p, pair, total_kb, wi, w); ++wi) {
+    for (int wi = 0; ok && next_work(gp, pair, wi, w); ++wi) {
+      const Tf32Params& p = gp.pr[w.prob];
+      const int bn = p.bn, hb = p.bn >> 1;                     // hb: B rows staged by each CTA
+      const uint32_t pair_tx = 2u * (A_STAGE_BYTES + (uint32_t)hb * BK * 4);
       const int t = w.tile, kb0 = w.kb0, kb1 = w.kb1;
       const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM;
       const int n0 = (t % p.tiles_n) * bn + (int)rank * hb;
@@ -513,7 +534,7 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1;
         int good = 1;
-        if (lane == 0) good = wait_or_abort(&empty[s], ph ^ 1, abort_flag, p.err, 1) ? 1 : 0;
+        if (lane == 0) good = wait_or_abort(&empty[s], ph ^ 1, abort_flag, err, 1) ? 1 : 0;
         good = __shfl_sync(0xffffffffu, good, 0);
         if (!good) { ok = false; break; }
         if (rank == 0 && lane == 0) mbar_expect_tx(&full[s], pair_tx);
@@ -521,8 +542,8 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
         const uint32_t full_leader = map_to_cta(smem_u32(&full[s]), 0);
         const int pr = kb < p.kblocks[0] ? 0 : 1;
         const int k0 = (pr == 0 ? kb : kb - p.kblocks[0]) * BK;
-        const CUtensorMap* ma = pr == 0 ? &tmA0 : &tmA1;
-        const CUtensorMap* mb = pr == 0 ? &tmB0 : &tmB1;
+        const CUtensorMap* ma = &gm.m[w.prob][2 * pr];
+        const CUtensorMap* mb = &gm.m[w.prob][2 * pr + 1];
         uint8_t* sa = smem + s * STAGE2_BYTES;
         uint8_t* sb = sa + A_STAGE_BYTES;
         if (!p.a_mn) {
@@ -545,27 +566,28 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
   } else if (warp == 1) {
     if (rank == 0 && lane == 0) {
       // ---------------------------------------------------------------- MMA issuer (leader CTA only)
-      const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(p.a_mn ? 1 : 0) << 15) |
-                             ((uint32_t)(p.b_mn ? 1 : 0) << 16) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
-      const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
-      const uint32_t a_step = p.a_mn ? 1024 : 32, b_step = p.b_mn ? 1024 : 32;
-      const uint32_t a_sbo = p.a_mn ? 512 : 1024, b_sbo = p.b_mn ? 512 : 1024;
-      const uint32_t a_lay = p.a_mn ? 1 : 2, b_lay = p.b_mn ? 1 : 2;
       int it = 0, ti = 0;
       bool ok = true;
       Work w;
-      for (int wi = 0; ok && next_work(p, pair, total_kb, wi, w); ++wi, ++ti) {
+      for (int wi = 0; ok && next_work(gp, pair, wi, w); ++wi, ++ti) {
+        const Tf32Params& p = gp.pr[w.prob];
+        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(p.a_mn ? 1 : 0) << 15) |
+                               ((uint32_t)(p.b_mn ? 1 : 0) << 16) | ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+        const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
+        const uint32_t a_step = p.a_mn ? 1024 : 32, b_step = p.b_mn ? 1024 : 32;
+        const uint32_t a_sbo = p.a_mn ? 512 : 1024, b_sbo = p.b_mn ? 512 : 1024;
+        const uint32_t a_lay = p.a_mn ? 1 : 2, b_lay = p.b_mn ? 1 : 2;
         const int kb0 = w.kb0, kb1 = w.kb1;
         const int buf = ti & 1;
         const uint32_t aph = (ti >> 1) & 1;
-        ok = wait_or_abort(&acc_empty[buf], aph ^ 1, abort_flag, p.err, 4);
+        ok = wait_or_abort(&acc_empty[buf], aph ^ 1, abort_flag, err, 4);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN_MAX);
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
-          ok = wait_or_abort(&full[s], ph, abort_flag, p.err, 2);
+          ok = wait_or_abort(&full[s], ph, abort_flag, err, 2);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + s * STAGE2_BYTES);
@@ -588,13 +610,15 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
     const int row = quad * 32 + lane;                          // row of this CTA's 128-row block
     int ti = 0;
     Work w;
-    for (int wi = 0; next_work(p, pair, total_kb, wi, w); ++wi, ++ti) {
+    for (int wi = 0; next_work(gp, pair, wi, w); ++wi, ++ti) {
+      const Tf32Params& p = gp.pr[w.prob];
+      const int bn = p.bn;
       const int t = w.tile;
       const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM, n0 = (t % p.tiles_n) * bn;
       const int buf = ti & 1;
       const uint32_t aph = (ti >> 1) & 1;
       int good = 1;
-      if (lane == 0) good = wait_or_abort(&acc_full[buf], aph, abort_flag, p.err, 3) ? 1 : 0;
+      if (lane == 0) good = wait_or_abort(&acc_full[buf], aph, abort_flag, err, 3) ? 1 : 0;
       good = __shfl_sync(0xffffffffu, good, 0);
       if (!good) break;
       tc_fence_after();
@@ -625,7 +649,7 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
           const int want = 16 * p.slices;
           const unsigned long long t0 = globaltimer();
           while (*flag < want) {
-            if (*abort_flag || globaltimer() - t0 > WAIT_LIMIT_NS) { atomicCAS(p.err, 0, 5); *abort_flag = 1; good = 0; break; }
+            if (*abort_flag || globaltimer() - t0 > WAIT_LIMIT_NS) { atomicCAS(err, 0, 5); *abort_flag = 1; good = 0; break; }
             __nanosleep(200);   // sixteen warps per pair poll the same word: keep them off the L2 while the pair's MMAs run
           }
           __threadfence();
@@ -643,13 +667,16 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
         const float* zrow = p.dsig ? p.dsig + (long long)((m / p.dsig_div) % p.dsig_rows) * p.ld_dsig : nullptr;
         const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
         float* drow = p.D + (long long)m * p.ldd;
+        const float* const bias = p.bias;
+        const float alpha = p.alpha, beta = p.beta;
+        const int N = p.N, sigm = p.sigmoid, vec_epi = p.vec_epi;
         // whole tile: this warp's chunks are half, half + 2, ...; sliced tile: the pair's share of the
         // chunks is sl, sl + slices, ..., dealt alternately to the two warps of a quadrant
         const int c_first = w.sliced ? sl + half * p.slices : half;
         const int c_step = w.sliced ? 2 * p.slices : 2;
         for (int c = c_first; c < n_chunks; c += c_step) {
           const int nb = n0 + c * 32;
-          const bool fullc = p.vec_epi && nb + 32 <= p.N;
+          const bool fullc = vec_epi && nb + 32 <= N;
           float4 zc[8], ci[8];
           if (fullc && m_ok) {
 #pragma unroll
@@ -679,16 +706,16 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
               float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (p.bias) bz = __ldg(reinterpret_cast<const float4*>(p.bias + nb) + q);
+              if (bias) bz = __ldg(reinterpret_cast<const float4*>(bias + nb) + q);
               float x[4] = {v[4 * q] + bz.x, v[4 * q + 1] + bz.y, v[4 * q + 2] + bz.z, v[4 * q + 3] + bz.w};
               const float z[4] = {zc[q].x, zc[q].y, zc[q].z, zc[q].w};
               const float cc[4] = {ci[q].x, ci[q].y, ci[q].z, ci[q].w};
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                if (p.sigmoid) x[j] = 1.f / (1.f + __expf(-x[j]));
+                if (sigm) x[j] = 1.f / (1.f + __expf(-x[j]));
                 if (zrow) x[j] *= z[j] * (1.f - z[j]);
-                x[j] *= p.alpha;
-                if (crow) x[j] = fmaf(p.beta, cc[j], x[j]);
+                x[j] *= alpha;
+                if (crow) x[j] = fmaf(beta, cc[j], x[j]);
               }
               reinterpret_cast<float4*>(drow + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
             }
@@ -696,12 +723,12 @@ gemm_tf32_2cta_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_con
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               const int n = nb + j;
-              if (n < p.N) {
-                float x = v[j] + (p.bias ? __ldg(p.bias + n) : 0.f);
-                if (p.sigmoid) x = 1.f / (1.f + __expf(-x));
+              if (n < N) {
+                float x = v[j] + (bias ? __ldg(bias + n) : 0.f);
+                if (sigm) x = 1.f / (1.f + __expf(-x));
                 if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
-                x *= p.alpha;
-                if (crow) x = fmaf(p.beta, __ldg(crow + n), x);
+                x *= alpha;
+                if (crow) x = fmaf(beta, __ldg(crow + n), x);
                 drow[n] = x;
               }
             }
@@ -1106,22 +1133,11 @@ int choose_bn2(int M, int N, bool stream_k, int fixed_cost = 320) {
 int64_t gemm_tf32_workspace_floats() { return (int64_t)(num_sms() / 2) * 2 * BM * BN_MAX; }
 int gemm_tf32_workspace_flags() { return num_sms() / 2; }
 
-int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(gemm_tf32_kernel<kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    attr_set = true;
-  }
-  static bool attr2_set = false;
-  if (!attr2_set) {
-    cudaFuncSetAttribute(gemm_tf32_2cta_kernel<kStages2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
-    attr2_set = true;
-  }
-  const bool two_cta = g.two_cta >= 0 ? g.two_cta != 0 : (g.M > BM && g.N >= 128);
-  const bool stream_k = two_cta && sk_ws && sk_flags;
-  const int bn = two_cta ? choose_bn2(g.M, g.N, stream_k) : choose_bn(g.M, g.N);
+namespace {
+
+// Tensor maps and kernel parameters of one problem for a given tile width (two_cta: 256 x bn tiles of a CTA pair).
+bool setup_problem(const GemmArgs& g, bool two_cta, int bn, int* err_flag, CUtensorMap* maps, Tf32Params& p) {
   const int b_rows = two_cta ? bn / 2 : bn;      // B rows staged per CTA
-  CUtensorMap maps[4];
   const float* As[2] = {g.A1, g.A2};
   const float* Bs[2] = {g.B1, g.B2};
   const int Ks[2] = {g.K1, g.A2 ? g.K2 : 0};
@@ -1136,9 +1152,9 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
     if (g.b_kmajor)      ok = ok && make_map(&maps[2 * s + 1], Bs[src], g.N, Ks[src], ldb[src], BK, b_rows, kmaj);
     else if (g.mn_padded) ok = ok && make_map_mn3d(&maps[2 * s + 1], Bs[src], Ks[src], g.N, ldb[src], b_rows / 32);
     else                 ok = ok && make_map(&maps[2 * s + 1], Bs[src], Ks[src], g.N, ldb[src], 32, BK, mnmaj);
-    if (!ok) return -1;
+    if (!ok) return false;
   }
-  Tf32Params p{};
+  p = Tf32Params{};
   p.M = g.M; p.N = g.N;
   p.kblocks[0] = (Ks[0] + BK - 1) / BK;
   p.kblocks[1] = (Ks[1] + BK - 1) / BK;
@@ -1154,16 +1170,42 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
               (!g.cin || (aligned16(g.cin) && g.ld_cin % 4 == 0));
   p.bn = bn;
   p.tiles_n = (g.N + bn - 1) / bn;
+  p.tiles = ((g.M + (two_cta ? 2 : 1) * BM - 1) / ((two_cta ? 2 : 1) * BM)) * p.tiles_n;
   p.err = err_flag;
+  p.slices = 1;
+  return true;
+}
+
+void set_kernel_attributes() {
+  static bool done = false;
+  if (!done) {
+    cudaFuncSetAttribute(gemm_tf32_kernel<kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaFuncSetAttribute(gemm_tf32_2cta_kernel<kStages2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+    done = true;
+  }
+}
+
+inline bool suits_pair_kernel(const GemmArgs& g) { return g.M > BM && g.N >= 128; }
+
+}  // namespace
+
+int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st) {
+  set_kernel_attributes();
+  const bool two_cta = g.two_cta >= 0 ? g.two_cta != 0 : suits_pair_kernel(g);
+  const bool stream_k = two_cta && sk_ws && sk_flags;
+  const int bn = two_cta ? choose_bn2(g.M, g.N, stream_k) : choose_bn(g.M, g.N);
   if (two_cta) {
-    p.tiles = ((g.M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;   // tiles of 256 rows, one per CTA pair
+    GroupMaps gm;                              // (host copies; passed to the kernel by value)
+    GroupParams gp;
+    gp.n_prob = 1;
+    Tf32Params& p = gp.pr[0];
+    if (!setup_problem(g, true, bn, err_flag, gm.m[0], p)) return -1;
     const int pairs = num_sms() / 2;
     const int total_kb = p.kblocks[0] + p.kblocks[1];
     p.sk_ws = sk_ws; p.sk_flags = sk_flags;
     p.P = p.tiles < pairs ? p.tiles : pairs;
     p.waves = p.tiles / p.P;
     p.rem = p.tiles - p.waves * p.P;
-    p.slices = 1;
     int launch_pairs = p.P;
     if (stream_k && p.tiles < pairs) {
       // fewer tiles than pairs: there is no full wave; every tile is cut along K over pairs / tiles pairs
@@ -1176,13 +1218,97 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
       // a slice costs a store and a re-read of the tile on top of its MMAs: not worth it for short K
       if (sl >= 2 && total_kb / sl >= 4) p.slices = sl;
     }
-    if (p.waves == 0) launch_pairs = p.rem * p.slices;
-    gemm_tf32_2cta_kernel<kStages2><<<2 * launch_pairs, 320, kSmemBytes2, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+    if (p.waves == 0) launch_pairs = p.slices >= 2 ? p.rem * p.slices : p.rem;
+    for (int q = 0; q <= MAX_PAIRS_LAUNCH; ++q) gp.rstart[0][q] = (unsigned short)(q < p.rem ? q : p.rem);
+    gemm_tf32_2cta_kernel<kStages2><<<2 * launch_pairs, 320, kSmemBytes2, st>>>(gm, gp);
   } else {
-    p.tiles = ((g.M + BM - 1) / BM) * p.tiles_n;
+    CUtensorMap maps[4];
+    Tf32Params p;
+    if (!setup_problem(g, false, bn, err_flag, maps, p)) return -1;
     const int grid = p.tiles < num_sms() ? p.tiles : num_sms();
     gemm_tf32_kernel<kStages><<<grid, 320, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
   }
+  return 1;
+}
+
+bool gemm_tf32_group_eligible(const GemmArgs* gs, int n) {
+  if (n < 1 || n > MAX_GROUP || num_sms() / 2 > MAX_PAIRS_LAUNCH) return false;
+  for (int i = 0; i < n; ++i)
+    if (!gemm_tf32_eligible(gs[i]) || !suits_pair_kernel(gs[i]) || gs[i].two_cta == 0) return false;
+  return true;
+}
+
+// Several independent problems in one launch of the CTA-pair kernel.  The pairs' work is balanced on the host:
+// problems are taken longest tile first; each gets as many whole waves (tiles q, q + P, ... for every pair q)
+// as fit under the level that evens out the loads so far, and its left-over tiles go to the least loaded pairs.
+int launch_gemm_tf32_group(const GemmArgs* gs, int n, int* err_flag, cudaStream_t st) {
+  if (!gemm_tf32_group_eligible(gs, n)) return -1;
+  set_kernel_attributes();
+  GroupMaps gm;
+  GroupParams gp;
+  const int pairs = num_sms() / 2;
+  struct Item { int src; double cost; };
+  Item order[MAX_GROUP];
+  Tf32Params tmp[MAX_GROUP];
+  CUtensorMap tmaps[MAX_GROUP][4];
+  long long total_tiles = 0;
+  for (int i = 0; i < n; ++i) {
+    const int bn = choose_bn2(gs[i].M, gs[i].N, true);
+    if (!setup_problem(gs[i], true, bn, err_flag, tmaps[i], tmp[i])) return -1;
+    if (tmp[i].tiles > 60000) return -1;       // (left-over tile indices are 16-bit)
+    // time of one tile: operand bytes per k-block (the feed bounds the main loop) plus a fixed part
+    order[i].src = i;
+    order[i].cost = (tmp[i].kblocks[0] + tmp[i].kblocks[1]) * (256.0 + bn) / 512.0 + 8.0;
+    total_tiles += tmp[i].tiles;
+  }
+  for (int i = 1; i < n; ++i)                   // insertion sort, longest tile first (stable)
+    for (int j = i; j > 0 && order[j].cost > order[j - 1].cost; --j) { Item t = order[j]; order[j] = order[j - 1]; order[j - 1] = t; }
+  const int P = total_tiles < pairs ? (int)total_tiles : pairs;
+  double load[MAX_PAIRS_LAUNCH];
+  for (int q = 0; q < P; ++q) load[q] = 0.0;
+  gp.n_prob = n;
+  for (int k = 0; k < n; ++k) {
+    const int i = order[k].src;
+    const double cost = order[k].cost;
+    Tf32Params& p = gp.pr[k];
+    p = tmp[i];
+    for (int j = 0; j < 4; ++j) gm.m[k][j] = tmaps[i][j];
+    p.P = P;
+    // counts per pair: lowest level L with sum_q floor((L - load_q) / cost) >= tiles, by bisection on L
+    int cnt[MAX_PAIRS_LAUNCH];
+    double lo = 0.0, hi = 0.0;
+    for (int q = 0; q < P; ++q) if (load[q] > hi) hi = load[q];
+    hi += cost * (p.tiles / P + 2);
+    for (int iter = 0; iter < 60; ++iter) {
+      const double mid = 0.5 * (lo + hi);
+      long long have = 0;
+      for (int q = 0; q < P; ++q) if (mid > load[q]) have += (long long)((mid - load[q]) / cost);
+      if (have >= p.tiles) hi = mid; else lo = mid;
+    }
+    long long have = 0;
+    for (int q = 0; q < P; ++q) { cnt[q] = hi > load[q] ? (int)((hi - load[q]) / cost) : 0; have += cnt[q]; }
+    // more than needed (several pairs cross a multiple of `cost` at the same level): take back from the fullest
+    while (have > p.tiles) {
+      int worst = -1;
+      for (int q = 0; q < P; ++q)
+        if (cnt[q] > 0 && (worst < 0 || load[q] + cnt[q] * cost > load[worst] + cnt[worst] * cost)) worst = q;
+      --cnt[worst]; --have;
+    }
+    while (have < p.tiles) {                    // (rounding in the bisection)
+      int best = 0;
+      for (int q = 1; q < P; ++q)
+        if (load[q] + cnt[q] * cost < load[best] + cnt[best] * cost) best = q;
+      ++cnt[best]; ++have;
+    }
+    int waves = cnt[0];
+    for (int q = 1; q < P; ++q) if (cnt[q] < waves) waves = cnt[q];
+    p.waves = waves;
+    p.rem = p.tiles - waves * P;
+    int run = 0;
+    for (int q = 0; q < P; ++q) { gp.rstart[k][q] = (unsigned short)run; run += cnt[q] - waves; load[q] += cnt[q] * cost; }
+    for (int q = P; q <= MAX_PAIRS_LAUNCH; ++q) gp.rstart[k][q] = (unsigned short)run;
+  }
+  gemm_tf32_2cta_kernel<kStages2><<<2 * P, 320, kSmemBytes2, st>>>(gm, gp);
   return 1;
 }
 

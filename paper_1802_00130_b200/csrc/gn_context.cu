@@ -56,6 +56,7 @@ struct gn_ctx {
   float* thin_scratch = nullptr; int64_t thin_cap = 0;
   float* sk_ws = nullptr; int* sk_flags = nullptr;   // stream-K workspace of the tensor-core kernel
   bool sk_enabled = true;
+  bool group_enabled = true;   // independent contractions of a layer as one launch (TF32 mode)
   // FP32-accurate mode on the tensor cores (3 x TF32): hi / lo parts of the operands
   int acc_method = 0;        // 0 choose (tensor cores where the shape allows), 1 FP32 FMA only, 2 as 0
   bool x3_usable = true;     // cleared if the error-compensated kernel could not be launched
@@ -335,6 +336,52 @@ void run_gemm(gn_ctx* c, const GemmArgs& g) {
   run_gemm_kind(c, g, (c->prec == GN_TF32 && gemm_tf32_eligible(g)) ? 0 : 1);
 }
 
+// Independent contractions issued together (any order is allowed).  In TF32 mode those that suit the CTA-pair
+// kernel go out in launches of up to three problems with a common work list (the tiles of one fill the partial
+// last wave of another); everything else runs one after the other, in the order given.
+void run_gemm_group(gn_ctx* c, const GemmArgs* gs, int n) {
+  constexpr int kMax = 3;
+  bool taken[16] = {false};
+  if (n >= 2 && n <= 16 && c->prec == GN_TF32 && c->group_enabled) {
+    GemmArgs pick[kMax];
+    int idx[kMax], np = 0;
+    auto flush = [&]() {
+      if (np >= 2 && gemm_tf32_group_eligible(pick, np)) {
+        c->gemm_seq += (uint64_t)np;
+        gn_ctx::EvPair* e = nullptr;
+        if (c->profiling) {
+          if (c->ev_used == c->ev.size()) {
+            gn_ctx::EvPair p{};
+            if (cudaEventCreate(&p.a) == cudaSuccess && cudaEventCreate(&p.b) == cudaSuccess) c->ev.push_back(p);
+          }
+          if (c->ev_used < c->ev.size()) {
+            e = &c->ev[c->ev_used++];
+            e->flop = 0.0;
+            for (int i = 0; i < np; ++i)
+              e->flop += 2.0 * pick[i].M * (double)pick[i].N * ((double)pick[i].K1 + (pick[i].A2 ? (double)pick[i].K2 : 0.0));
+            e->kind = 0;
+            cudaEventRecord(e->a, c->st);
+          }
+        }
+        const int r = launch_gemm_tf32_group(pick, np, c->err_flag + 1, c->st);
+        if (r < 0) { c->sticky = GN_ECUDA; c->err = "cuTensorMapEncodeTiled failed"; }
+        else c->launches += r;
+        if (e) cudaEventRecord(e->b, c->st);
+        for (int i = 0; i < np; ++i) taken[idx[i]] = true;
+      }
+      np = 0;
+    };
+    for (int i = 0; i < n; ++i) {
+      if (gemm_thin_kind(gs[i]) != THIN_NONE || !gemm_tf32_group_eligible(&gs[i], 1)) continue;
+      pick[np] = gs[i]; idx[np] = i; ++np;
+      if (np == kMax) flush();
+    }
+    flush();
+  }
+  for (int i = 0; i < n; ++i)
+    if (i >= 16 || !taken[i]) run_gemm(c, gs[i]);
+}
+
 gn_status ensure_partials(gn_ctx* c, int64_t count) {
   if (count <= c->partial_cap) return GN_OK;
   dev_free(c, c->partial, c->partial_cap);
@@ -377,8 +424,8 @@ void forward_pass(gn_ctx* c, const float* Z0, int64_t rows, std::vector<float*>&
 
 // Parameter-space half of the backward pass for one layer (Eqs. xtow-g, xtow-g-bias, and their
 // Jacobian twins of Section 4.2): out_W = alpha ds^T Zprev + beta cin_W, out_b = alpha 1^T ds + beta cin_b.
-gn_status weight_block(gn_ctx* c, int m, const float* ds, const float* Zprev, int64_t rows, float alpha,
-                       const float* cin, float beta, float* out, bool padded = true) {
+GemmArgs weight_block_args(const gn_ctx* c, int m, const float* ds, const float* Zprev, int64_t rows, float alpha,
+                           const float* cin, float beta, float* out, bool padded = true) {
   GemmArgs g;
   g.mn_padded = padded;   // ds and Zprev are context-owned (padded) unless the caller says otherwise
   g.M = c->w[m]; g.N = c->w[m - 1];
@@ -388,17 +435,27 @@ gn_status weight_block(gn_ctx* c, int m, const float* ds, const float* Zprev, in
   g.alpha = alpha;
   g.cin = cin + c->w_off[m]; g.ld_cin = c->w[m - 1]; g.beta = beta;
   g.D = out + c->w_off[m]; g.ldd = c->w[m - 1];
-  run_gemm(c, g);
+  return g;
+}
+
+gn_status bias_block(gn_ctx* c, int m, const float* ds, int64_t rows, float alpha, const float* cin, float beta,
+                     float* out) {
   GN_TRY(ensure_colsum(c, rows, c->w[m]));
   c->launches += launch_colsum(ds, rows, c->w[m], c->w[m], alpha, cin + c->b_off[m], beta, out + c->b_off[m],
                                c->colsum_scratch, c->st);
   return GN_OK;
 }
 
+gn_status weight_block(gn_ctx* c, int m, const float* ds, const float* Zprev, int64_t rows, float alpha,
+                       const float* cin, float beta, float* out, bool padded = true) {
+  run_gemm(c, weight_block_args(c, m, ds, Zprev, rows, alpha, cin, beta, out, padded));
+  return bias_block(c, m, ds, rows, alpha, cin, beta, out);
+}
+
 // Activation-space half (Eq. communi-g / communi-jaco followed by Eq. ztox-g):
 // dst = (ds W^mT) * sigma'(z^{m-1}), rows stacked modulo z_rows.
-void backward_data(gn_ctx* c, int m, const float* ds, int64_t rows, const float* Zprev, int64_t z_rows, float* dst,
-                   bool ds_just_used = false) {
+GemmArgs backward_data_args(const gn_ctx* c, int m, const float* ds, int64_t rows, const float* Zprev, int64_t z_rows,
+                            float* dst, bool ds_just_used = false) {
   GemmArgs g;
   g.a1_split_fresh = ds_just_used;   // the weight block of the same layer has just read these very rows of ds
   g.M = (int)rows; g.N = c->w[m - 1];
@@ -408,7 +465,20 @@ void backward_data(gn_ctx* c, int m, const float* ds, int64_t rows, const float*
   g.dsig = Zprev; g.ld_dsig = c->w[m - 1]; g.dsig_rows = (int)z_rows;
   g.D = dst; g.ldd = c->w[m - 1];
   g.mn_padded = true;     // B is the context's own (padded) copy of theta
-  run_gemm(c, g);
+  return g;
+}
+
+// Both halves for layer m from the same ds: the weight block over `w_rows` rows starting at ds_w, and (above the
+// first layer) the activation gradient over `d_rows` rows starting at ds_d.  The two contractions are independent.
+gn_status layer_backward(gn_ctx* c, int m, const float* ds_w, int64_t w_rows, const float* ds_d, int64_t d_rows,
+                         const float* Zprev, int64_t z_rows, float alpha, const float* cin, float beta, float* out,
+                         float* dst, bool w_padded = true) {
+  GemmArgs gs[2];
+  int n = 0;
+  gs[n++] = weight_block_args(c, m, ds_w, Zprev, w_rows, alpha, cin, beta, out, w_padded);
+  if (m > 1) gs[n++] = backward_data_args(c, m, ds_d, d_rows, Zprev, z_rows, dst, ds_w == ds_d && w_rows == d_rows);
+  run_gemm_group(c, gs, n);
+  return bias_block(c, m, ds_w, w_rows, alpha, cin, beta, out);
 }
 
 // out = coef v + (1/|S|) J^T (2 J v) over the stored subsample (Eq. sampled-Gauss).
@@ -433,11 +503,8 @@ gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
   const float* ds = c->RZ[L];
   const float inv = (float)(1.0 / (double)nS);
   for (int m = L; m >= 1; --m) {
-    GN_TRY(weight_block(c, m, ds, c->Z[m - 1], nS, inv, v, coef, out));
-    if (m > 1) {
-      backward_data(c, m, ds, nS, c->Z[m - 1], nS, c->DS[m - 1], true);
-      ds = c->DS[m - 1];
-    }
+    GN_TRY(layer_backward(c, m, ds, nS, ds, nS, c->Z[m - 1], nS, inv, v, coef, out, m > 1 ? c->DS[m - 1] : nullptr));
+    if (m > 1) ds = c->DS[m - 1];
   }
   return check_launch(c, "G v");
 }
@@ -471,11 +538,9 @@ gn_status product_blockdiag(gn_ctx* c, const float* v, float* out, float coef) {
   const float inv = (float)(1.0 / (double)nS);
   for (int k = L; k >= 1; --k) {
     const float* dsk = cur + (k - 1) * nS * c->w[k];
-    GN_TRY(weight_block(c, k, dsk, c->Z[k - 1], nS, inv, v, coef, out));
-    if (k > 1) {
-      backward_data(c, k, cur, (k - 1) * nS, c->Z[k - 1], nS, c->DS[k - 1]);
-      cur = c->DS[k - 1];
-    }
+    GN_TRY(layer_backward(c, k, dsk, nS, cur, (k - 1) * nS, c->Z[k - 1], nS, inv, v, coef, out,
+                          k > 1 ? c->DS[k - 1] : nullptr));
+    if (k > 1) cur = c->DS[k - 1];
   }
   return check_launch(c, "block-diagonal G v");
 }
@@ -523,22 +588,35 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
   const int L = c->L, nL = c->w[L];
   const int64_t nS = c->nS;
   const float inv = (float)(1.0 / (double)nS);
-  for (int m = 1; m <= L; ++m) {
-    // u_i = V^{mT} z^{m-1,i} + c^m for every row (the inner sum of Eq. direct-JV-cost); at m = L, D = I and B = 2I
-    GemmArgs g;
-    g.M = (int)nS; g.N = c->w[m];
-    g.A1 = c->Z[m - 1]; g.lda1 = c->w[m - 1]; g.B1 = Wm(c, v, m); g.ldb1 = c->w[m - 1]; g.K1 = c->w[m - 1];
-    g.bias = bm(c, v, m);
-    if (m == L) g.alpha = 2.f;
-    g.D = c->RZ[m]; g.ldd = c->w[m];
-    run_gemm(c, g);
-    const float* ds = c->RZ[m];
-    if (m < L) {
-      c->launches += launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], 1, 1, 0, c->DS[m], c->st);
-      ds = c->DS[m];
+  constexpr int kGroup = 3;
+  // The layers' chains are independent of one another, so each stage is issued for all layers together.
+  // 1. u_i = V^{mT} z^{m-1,i} + c^m for every row (the inner sum of Eq. direct-JV-cost); at m = L, D = I and B = 2I
+  for (int m0 = 1; m0 <= L; m0 += kGroup) {
+    GemmArgs gs[kGroup];
+    int n = 0;
+    for (int m = m0; m <= L && m < m0 + kGroup; ++m) {
+      GemmArgs& g = gs[n++];
+      g.M = (int)nS; g.N = c->w[m];
+      g.A1 = c->Z[m - 1]; g.lda1 = c->w[m - 1]; g.B1 = Wm(c, v, m); g.ldb1 = c->w[m - 1]; g.K1 = c->w[m - 1];
+      g.bias = bm(c, v, m);
+      if (m == L) g.alpha = 2.f;
+      g.D = c->RZ[m]; g.ldd = c->w[m];
     }
-    GN_TRY(weight_block(c, m, ds, c->Z[m - 1], nS, inv, v, coef, out));
+    run_gemm_group(c, gs, n);
   }
+  // 2. q_i = D_i^T 2 D_i u_i per sample (Eqs. direct-JV-cost, JTv)
+  for (int m = 1; m < L; ++m)
+    c->launches += launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], 1, 1, 0, c->DS[m], c->st);
+  // 3. the weight and bias blocks
+  for (int m0 = 1; m0 <= L; m0 += kGroup) {
+    GemmArgs gs[kGroup];
+    int n = 0;
+    for (int m = m0; m <= L && m < m0 + kGroup; ++m)
+      gs[n++] = weight_block_args(c, m, m < L ? c->DS[m] : c->RZ[m], c->Z[m - 1], nS, inv, v, coef, out);
+    run_gemm_group(c, gs, n);
+  }
+  for (int m = 1; m <= L; ++m)
+    GN_TRY(bias_block(c, m, m < L ? c->DS[m] : c->RZ[m], nS, inv, v, coef, out));
   return check_launch(c, "block-diagonal G v (stored factors)");
 }
 
@@ -669,10 +747,12 @@ gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
           const int64_t head = rows - 32;
           GN_TRY(weight_block(c, 1, c->Db[1], X0, head, inv_l, cin0, beta0, d_grad, true));
           GN_TRY(weight_block(c, 1, c->Db[1] + head * c->w[1], X0 + head * c->w[0], 32, inv_l, d_grad, 1.f, d_grad, false));
+        } else if (m == 1) {
+          GN_TRY(weight_block(c, 1, c->Db[1], Zprev, rows, inv_l, cin0, beta0, d_grad, r0 + rows != c->l));
         } else {
-          GN_TRY(weight_block(c, m, c->Db[m], Zprev, rows, inv_l, cin0, beta0, d_grad, !(m == 1 && r0 + rows == c->l)));
+          GN_TRY(layer_backward(c, m, c->Db[m], rows, c->Db[m], rows, c->Zb[m - 1], rows, inv_l, cin0, beta0, d_grad,
+                                c->Db[m - 1]));
         }
-        if (m > 1) backward_data(c, m, c->Db[m], rows, c->Zb[m - 1], rows, c->Db[m - 1], true);
       }
     }
   }
@@ -1212,6 +1292,14 @@ gn_status gn_newton_iter(gn_ctx* c, float* d_theta, const int32_t* d_idx, int64_
   rep->f_before = f0; rep->f_after = f1; rep->alpha = alpha; rep->beta1 = beta1; rep->beta2 = beta2;
   rep->rho = rho; rep->gTd = gTd; rep->dGd = dGd; rep->lambda_next = lam;
   rep->cg_iters = its; rep->backtracks = backtracks;
+  return GN_OK;
+}
+
+gn_status gn_debug_option(gn_ctx* c, int option, int value) {
+  if (!c) return GN_EINVAL;
+  if (option == 0) c->group_enabled = value != 0;
+  else if (option == 1) c->sk_enabled = value != 0 && c->sk_enabled;
+  else return fail(c, GN_EINVAL, "unknown option");
   return GN_OK;
 }
 

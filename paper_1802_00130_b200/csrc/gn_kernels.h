@@ -59,6 +59,11 @@ int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st);
 int64_t gemm_tf32_workspace_floats();
 int gemm_tf32_workspace_flags();
 int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st);
+// Up to three independent problems, each suited to the CTA-pair kernel (M > 128, N >= 128), as ONE launch whose
+// pairs walk a common, host-balanced work list: the tiles of one problem fill the partial last wave of another.
+// Whole tiles only.  Returns launches made, or -1 if the group cannot run this way (run the problems one by one).
+bool gemm_tf32_group_eligible(const GemmArgs* gs, int n);
+int launch_gemm_tf32_group(const GemmArgs* gs, int n, int* err_flag, cudaStream_t st);
 
 // Streaming FP32 kernels for contractions with one dimension <= 16 (the n_L-wide output layer).
 // gemm_thin_kind says which of them (if any) takes a problem; THIN_M needs a scratch buffer of

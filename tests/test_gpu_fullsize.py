@@ -34,8 +34,9 @@ def test_svhn1000_products_and_cg():
     ctx.set_subsample(dev(p["idx"]))
     XS = p["X"][p["idx"]]
     v = dev(p["v"])
-    product_error = relb(ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"]), p["widths"])
-    assert product_error <= 1.5e-6           # far inside the 1e-5 of the mode; the CG bound below builds on it
+    out, ref = ctx.Gv(v).cpu().numpy(), orc.Gv(p["theta"], p["widths"], p["C"], XS, p["v"])
+    assert relb(out, ref, p["widths"]) <= TOL["fp32"]
+    assert rel(out, ref) <= 1e-6             # the whole vector is what CG sees; the CG bound below builds on this
     assert relb(ctx.Gv_blockdiag(v).cpu().numpy(),
                orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"]), p["widths"]) <= TOL["fp32"]
     g = ctx.grad()
@@ -45,7 +46,7 @@ def test_svhn1000_products_and_cg():
     # On this system a product error eps moves the iterates by up to AMPLIFICATION_BOUND * eps from the third step
     # on (tests/test_oracle_cg_sensitivity.py shows it with the checker alone), so the 1e-4 that holds on the small
     # configurations is out of reach of any FP32 product here; the bound is that factor times the error asserted above.
-    bound = AMPLIFICATION_BOUND * 1.5e-6
+    bound = AMPLIFICATION_BOUND * 1e-6
     g32 = g_ref.astype(np.float32)
     _, its_ref, res_ref = orc.cg_solve(p["theta"], p["widths"], p["C"], XS, g32, 1.0, False, 20, 0.0)
     d, its, res, iterates = ctx.cg_solve(dev(g32), 1.0, blockdiag=False, max_iter=20, tol=0.0, keep_iterates=True)

@@ -1,0 +1,50 @@
+"""Independent contractions of a layer issued as one launch of the CTA-pair kernel (TF32 mode): same bits as one
+launch per contraction, and the usual bound against the float64 checker."""
+import numpy as np
+import pytest
+
+import gn_workloads as wl
+from oracle import gn_oracle as orc
+from test_gpu_parity import TOL, dev, make_ctx, relb
+
+pytestmark = pytest.mark.gpu
+
+CASES = {
+    "mid": lambda: wl.make("mid"),
+    "ragged_wide": lambda: wl.make_custom([300, 520, 392, 10], l=1500, nS=1100, C=15.0, seed=41, x="sparse80"),
+    "mnist2000_5": lambda: wl.make("mnist2000_5", l=6000),
+    "svhn1000": lambda: wl.make("svhn1000", l=5000),
+    "deep": lambda: wl.make_custom([256, 384, 256, 512, 256, 8], l=2000, nS=1300, C=20.0, seed=43, x="uniform"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(CASES))
+def test_grouped_launches_give_the_bits_of_single_launches(name):
+    import torch
+    p = CASES[name]()
+    outs = []
+    for grouped in (0, 1):
+        ctx = make_ctx(p, "tf32")
+        ctx.debug_option(1, 0)                  # whole tiles only in both runs: K slices change the order of sums
+        ctx.debug_option(0, grouped)
+        ctx.set_subsample(dev(p["idx"]))
+        v = dev(p["v"])
+        res = [ctx.Gv(v).clone()]
+        for method in (1, 2):
+            ctx.set_blockdiag_method(method)
+            res.append(ctx.Gv_blockdiag(v).clone())
+        res.append(ctx.grad().clone())
+        launches = ctx.kernel_launches
+        outs.append((res, launches))
+        ctx.close()
+    for a, b in zip(outs[0][0], outs[1][0]):
+        assert torch.equal(a, b)
+    assert outs[1][1] < outs[0][1]              # fewer launches: something was in fact grouped
+    XS = p["X"][p["idx"]]
+    th, w, C = p["theta"], p["widths"], p["C"]
+    res = [r.cpu().numpy() for r in outs[1][0]]
+    assert relb(res[0], orc.Gv(th, w, C, XS, p["v"]), w) <= TOL["tf32"]
+    ref_b = orc.Gv_blockdiag(th, w, C, XS, p["v"])
+    assert relb(res[1], ref_b, w) <= TOL["tf32"]
+    assert relb(res[2], ref_b, w) <= TOL["tf32"]
+    assert relb(res[3], orc.grad(th, w, C, p["X"], p["Y"]), w) <= TOL["tf32"]
