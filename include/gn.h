@@ -65,7 +65,9 @@ typedef enum {
 
 typedef enum {
   GN_TF32 = 0,         /* contractions on the tensor cores with TF32 operands, FP32 accumulate   */
-  GN_FP32_ACCURATE = 1 /* contractions in full FP32 (fused multiply-add on the FP32 pipes)      */
+  GN_FP32_ACCURATE = 1 /* results at FP32 accuracy: error-compensated tensor-core contractions  */
+                       /* (3 x TF32 on hi / lo operand parts) where the shape allows, the FP32  */
+                       /* FMA GEMM elsewhere; see gn_set_accurate_method                        */
 } gn_precision;
 
 /*
@@ -93,6 +95,9 @@ const char* gn_last_error(const gn_ctx* ctx);
 
 /* gn_workspace_bytes - device memory currently owned by the context. */
 int64_t gn_workspace_bytes(const gn_ctx* ctx);
+
+/* gn_kernel_launches - number of kernels this context has launched so far (all entry points). */
+int64_t gn_kernel_launches(const gn_ctx* ctx);
 
 /*
  * gn_set_batch_rows - number of rows processed at a time by gn_fun / gn_grad, which walk the
@@ -273,6 +278,11 @@ typedef struct {
 gn_status gn_newton_iter(gn_ctx* ctx, float* d_theta, const int32_t* d_idx, int64_t nS, float* d_dir,
                          const gn_newton_params* params, gn_newton_report* report);
 
+/* ======================================================================================================
+ * TEST AND MEASUREMENT HOOKS.  Everything from here to gn_debug_option serves the test suite and the
+ * benchmark (failure paths, single kernels, per-launch timing, A/B switches); a solver has no use for them.
+ * ====================================================================================================== */
+
 /*
  * gn_debug_timeout_probe - test hook for the failure path of the tensor-core pipeline: launches one
  * CTA that waits, with the pipeline's bounded-wait code and the given limit (0 < limit_ms <= 1000), on a
@@ -318,10 +328,16 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
  * gn_debug_option - test and measurement hook: switch a launch strategy of the context for A/B runs.
  * option 0: independent contractions of a layer issued as one launch of the CTA-pair kernel (value 0 =
  * one launch per contraction); option 1: cutting left-over tiles along K between CTA pairs (value 0 = whole
- * tiles only; cannot be switched back on).  Results do not depend on option 0 beyond rounding order inside a tile
- * (none: tiles are computed identically); GN_EINVAL for an unknown option.
+ * tiles only; cannot be switched back on); option 2: failure injection on the host: the value-th device allocation
+ * the context asks for from now on is refused as if the device were out of memory (0 = off); nothing on the
+ * device is touched by it.  Results do not depend on option 0 (tiles are computed identically); GN_EINVAL for an
+ * unknown option.
  */
 gn_status gn_debug_option(gn_ctx* ctx, int option, int value);
+
+/* ======================================================================================================
+ * CONTEXT-FREE ENTRY POINT
+ * ====================================================================================================== */
 
 /*
  * gn_thin_m_gemm_noalloc - D[M][N] = sum_r A[r][m] B[r][n] for M <= 16 (the shape of the output layer's
@@ -345,7 +361,12 @@ gn_status gn_debug_option(gn_ctx* ctx, int option, int value);
  * any rows; M = 16, N = 4096 does not once rows > 2048).
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress) with that
  * device current; make that first call outside any stream capture.  No cudaMalloc, cudaFree or other
- * allocating routine is called, on the first call or later.
+ * allocating routine is called, on the first call or later.  The array is not the caller's to provide, but it is
+ * device memory all the same: the CUDA runtime places the library's kernels and this array on a device when the
+ * library is first used there (with CUDA's default lazy loading that can be as late as this first call), and a
+ * host application that has already taken every free byte leaves no room for that.  So make one call at start-up,
+ * before the host application's allocator takes the device's memory: it doubles as the warm-up, and every later
+ * call leaves the device's free memory exactly as it found it.
  * All calls share the one array, which keeps the previous call's partial sums: every element that a call
  * reads it has written first, so nothing needs clearing, but two calls whose kernels may overlap on the
  * GPU (different streams, or different host threads) race on it - serialise them.
@@ -353,11 +374,6 @@ gn_status gn_debug_option(gn_ctx* ctx, int option, int value);
 gn_status gn_thin_m_gemm_noalloc(int M, int N, int64_t rows, const float* dA, int64_t lda, const float* dB,
                                  int64_t ldb, float* dD, int64_t ldd, void* cuda_stream, char* errbuf,
                                  int64_t errbuf_len);
-
-/*
- * gn_kernel_launches - number of kernels this context has launched so far (all entry points).
- */
-int64_t gn_kernel_launches(const gn_ctx* ctx);
 
 #ifdef __cplusplus
 }

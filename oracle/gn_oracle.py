@@ -432,8 +432,7 @@ def cg_partitioned(theta, widths, C, XS, g, lam, split, max_iter, tol, cg_min=0,
             if tol > 0 and np.sqrt(rho_new) <= tol * gnorm[k]:
                 active[k] = False
         it += 1
-        if keep_iterates:
-            iterates.append(d.copy())
+        iterates.append(d.copy())
         resnorms.append(np.sqrt(rho.copy()))
     return d, iterates, resnorms
 

@@ -80,6 +80,8 @@ struct gn_ctx {
   gn_status sticky = GN_OK;  // a launch-time failure that must surface at the next check
   // CG
   float* cg_r = nullptr; float* cg_p = nullptr; float* cg_q = nullptr;
+  CgControl* cg_ctl = nullptr; CgControl* h_ctl = nullptr;   // device-resident solver state and its pinned mirror
+  double* cg_hist = nullptr; int cg_hist_cap = 0;            // squared residual norms, one per step
   float* tmp_a = nullptr; float* tmp_b = nullptr;  // staging for *_host calls
   float* nt[4] = {nullptr, nullptr, nullptr, nullptr};  // Newton iteration: g, d, G d / G dbar, trial theta
   CgChunk* chunks[2] = {nullptr, nullptr}; int n_chunks[2] = {0, 0};
@@ -94,7 +96,9 @@ struct gn_ctx {
   int64_t bytes = 0;
   int64_t launches = 0;
   std::string err;
-  std::vector<void*> owned;
+  struct Owned { void* p; int64_t bytes; };
+  std::vector<Owned> owned;     // every device allocation of the context with its accounted size
+  int fail_alloc_in = 0;        // test hook: the fail_alloc_in-th device allocation from now is refused (0 = off)
 };
 
 namespace {
@@ -125,6 +129,8 @@ template <class T>
 gn_status dev_alloc(gn_ctx* c, T** p, int64_t count) {
   *p = nullptr;
   if (count <= 0) count = 1;
+  if (c->fail_alloc_in > 0 && --c->fail_alloc_in == 0)
+    return fail(c, GN_ENOMEM, std::string("device allocation of ") + std::to_string(count * (int64_t)sizeof(T)) + " bytes refused (injected)");
   void* q = nullptr;
   // 256 bytes of slack: the tensor-core kernel's 3-D TMA boxes may read up to 124 bytes past the last
   // row of an MN-major operand
@@ -134,19 +140,25 @@ gn_status dev_alloc(gn_ctx* c, T** p, int64_t count) {
     return fail(c, GN_ENOMEM, std::string("cudaMalloc of ") + std::to_string(count * (int64_t)sizeof(T)) + " bytes: " + cudaGetErrorString(e));
   }
   c->bytes += count * (int64_t)sizeof(T);
-  c->owned.push_back(q);
+  c->owned.push_back({q, count * (int64_t)sizeof(T)});
   *p = static_cast<T*>(q);
   return GN_OK;
 }
 
+// Frees a context allocation (null is fine); the accounted size is the one recorded when it was made.
 template <class T>
-void dev_free(gn_ctx* c, T*& p, int64_t count) {
+void dev_free(gn_ctx* c, T*& p, int64_t = 0) {
   if (!p) return;
   for (auto& o : c->owned)
-    if (o == (void*)p) { o = nullptr; break; }
+    if (o.p == (void*)p) { c->bytes -= o.bytes; o.p = nullptr; o.bytes = 0; break; }
   cudaFree(p);
-  c->bytes -= (count <= 0 ? 1 : count) * (int64_t)sizeof(T);
   p = nullptr;
+  // keep the registry from growing without bound across many regrowths
+  if (c->owned.size() > 4096) {
+    size_t k = 0;
+    for (size_t i = 0; i < c->owned.size(); ++i) if (c->owned[i].p) c->owned[k++] = c->owned[i];
+    c->owned.resize(k);
+  }
 }
 
 gn_status check_launch(gn_ctx* c, const char* where) {
@@ -382,11 +394,15 @@ void run_gemm_group(gn_ctx* c, const GemmArgs* gs, int n) {
     if (i >= 16 || !taken[i]) run_gemm(c, gs[i]);
 }
 
+// (the new buffer is obtained before the old one is let go: the solver and the dot products use c->partial
+// without asking for it again, so a refused allocation must leave the old buffer in place)
 gn_status ensure_partials(gn_ctx* c, int64_t count) {
   if (count <= c->partial_cap) return GN_OK;
-  dev_free(c, c->partial, c->partial_cap);
-  c->partial_cap = 0;
-  GN_TRY(dev_alloc(c, &c->partial, count));
+  double* fresh = nullptr;
+  GN_TRY(dev_alloc(c, &fresh, count));
+  cudaStreamSynchronize(c->st);
+  dev_free(c, c->partial);
+  c->partial = fresh;
   c->partial_cap = count;
   return GN_OK;
 }
@@ -760,7 +776,7 @@ gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
     c->launches += launch_sum_partials(c->partial, (int)(per_batch * nb), c->dscal + 0, false, c->st);
     // theta^T theta with the CG dot kernel over the single-segment chunk table
     double* tp = c->partial + per_batch * nb;
-    c->launches += launch_cg_dot(c->theta, c->theta, c->chunks[0], c->n_chunks[0], tp, c->st);
+    c->launches += launch_cg_dot(c->theta, c->theta, c->chunks[0], c->n_chunks[0], tp, nullptr, 0, nullptr, c->st);
     c->launches += launch_sum_partials(tp, c->n_chunks[0], c->dscal + 1, false, c->st);
     GN_CUDA(c, cudaMemcpyAsync(c->hscal, c->dscal, 2 * sizeof(double), cudaMemcpyDeviceToHost, c->st));
     GN_TRY(check_launch(c, "f / grad"));
@@ -835,15 +851,23 @@ gn_status build_chunks(gn_ctx* c, bool block_only) {
       if (sg.count == 0) sg.first = (int)i;
       ++sg.count;
     }
-    dev_free(c, c->chunks[mode], c->n_chunks[mode]);
-    c->n_chunks[mode] = (int)h.size();
-    GN_TRY(dev_alloc(c, &c->chunks[mode], (int64_t)h.size()));
-    GN_CUDA(c, cudaMemcpy(c->chunks[mode], h.data(), h.size() * sizeof(CgChunk), cudaMemcpyHostToDevice));
-    dev_free(c, c->segs[mode], c->segs_cap[mode]);
-    c->segs_cap[mode] = 0;
-    GN_TRY(dev_alloc(c, &c->segs[mode], (int64_t)n_seg));
-    c->segs_cap[mode] = n_seg;
-    GN_CUDA(c, cudaMemcpy(c->segs[mode], segs.data(), segs.size() * sizeof(CgSeg), cudaMemcpyHostToDevice));
+    // room for the partial sums of the new table, then the new tables, then the swap: a refused allocation
+    // leaves the old tables (and the structure they belong to) in use
+    GN_TRY(ensure_partials(c, 2 * (int64_t)h.size() + 64));
+    CgChunk* d_chunks = nullptr;
+    CgSeg* d_segs = nullptr;
+    gn_status st = dev_alloc(c, &d_chunks, (int64_t)h.size());
+    if (st == GN_OK) st = dev_alloc(c, &d_segs, (int64_t)n_seg);
+    if (st == GN_OK && (cudaMemcpy(d_chunks, h.data(), h.size() * sizeof(CgChunk), cudaMemcpyHostToDevice) != cudaSuccess ||
+                        cudaMemcpy(d_segs, segs.data(), segs.size() * sizeof(CgSeg), cudaMemcpyHostToDevice) != cudaSuccess)) {
+      cudaGetLastError();
+      st = fail(c, GN_ECUDA, "copy of the chunk tables failed");
+    }
+    if (st != GN_OK) { dev_free(c, d_chunks); dev_free(c, d_segs); return st; }
+    dev_free(c, c->chunks[mode]);
+    dev_free(c, c->segs[mode]);
+    c->chunks[mode] = d_chunks; c->n_chunks[mode] = (int)h.size();
+    c->segs[mode] = d_segs; c->segs_cap[mode] = n_seg;
   }
   return GN_OK;
 }
@@ -890,13 +914,15 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
     if ((s = dev_alloc(c, &c->cg_p, c->n)) != GN_OK) break;
     if ((s = dev_alloc(c, &c->cg_q, c->n)) != GN_OK) break;
     if ((s = dev_alloc(c, &c->dscal, 16)) != GN_OK) break;
+    if ((s = dev_alloc(c, &c->cg_ctl, 1)) != GN_OK) break;
+    if (cudaMemset(c->cg_ctl, 0, sizeof(CgControl)) != cudaSuccess) { s = GN_ECUDA; break; }
+    if (cudaMallocHost(&c->h_ctl, sizeof(CgControl)) != cudaSuccess) { s = GN_ENOMEM; break; }
     if ((s = dev_alloc(c, &c->err_flag, 2)) != GN_OK) break;
     if (cudaMemset(c->err_flag, 0, 2 * sizeof(int)) != cudaSuccess) { s = GN_ECUDA; break; }
     if (cudaMallocHost(&c->hscal, 16 * sizeof(double)) != cudaSuccess) { s = GN_ENOMEM; break; }
     if (cudaMallocHost(&c->h_err, 2 * sizeof(int)) != cudaSuccess) { s = GN_ENOMEM; break; }
     c->h_err[0] = c->h_err[1] = 0;
     if ((s = build_chunks(c, false)) != GN_OK) break;
-    if ((s = ensure_partials(c, 2 * (int64_t)c->n_chunks[1] + 64)) != GN_OK) break;
   } while (0);
   if (s != GN_OK) { gn_destroy(c); return s; }
   *out = c;
@@ -906,10 +932,11 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
 gn_status gn_destroy(gn_ctx* c) {
   if (!c) return GN_OK;
   cudaStreamSynchronize(c->st);
-  for (void* p : c->owned)
-    if (p) cudaFree(p);
+  for (auto& o : c->owned)
+    if (o.p) cudaFree(o.p);
   for (auto& p : c->ev) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   if (c->hscal) cudaFreeHost(c->hscal);
+  if (c->h_ctl) cudaFreeHost(c->h_ctl);
   if (c->h_err) cudaFreeHost(c->h_err);
   cudaGetLastError();
   delete c;
@@ -963,11 +990,15 @@ gn_status gn_set_split(gn_ctx* c, const int32_t* split) {
   if (P > 1024) return fail(c, GN_EINVAL, "more than 1024 partitions");
   if (any && c->L >= 2 && c->w[c->L] > 32) return fail(c, GN_EINVAL, "a split structure needs n_L <= 32 (stored Jacobian factors)");
   GN_TRY(sync(c, "set_split"));
+  const std::vector<int> old_split = c->split;
+  const bool old_has = c->has_split;
+  const int old_P = c->P;
   c->split.assign(split, split + c->L + 1);
   c->has_split = any;
   c->P = (int)P;
-  GN_TRY(build_chunks(c, true));
-  return ensure_partials(c, 2 * (int64_t)c->n_chunks[1] + 64);
+  const gn_status st = build_chunks(c, true);
+  if (st != GN_OK) { c->split = old_split; c->has_split = old_has; c->P = old_P; }   // the old tables are still in place
+  return st;
 }
 
 int32_t gn_num_partitions(const gn_ctx* c) { return c ? c->P : -1; }
@@ -1122,35 +1153,63 @@ gn_status gn_cg_solve(gn_ctx* c, const float* d_g, double lambda, int blockdiag,
   const CgChunk* ch = c->chunks[mode];
   const int nc = c->n_chunks[mode];
   const float coef = (float)(1.0 / c->C + lambda);
-  double* out2 = c->dscal + 2;
+  CgSeg* seg = c->segs[mode];
+  // device-resident solver state: ticket, step count, residual history
+  if (max_iter + 1 > c->cg_hist_cap) {
+    GN_TRY(sync(c, "cg history"));
+    dev_free(c, c->cg_hist, c->cg_hist_cap);
+    c->cg_hist_cap = 0;
+    GN_TRY(dev_alloc(c, &c->cg_hist, (int64_t)max_iter + 1));
+    c->cg_hist_cap = max_iter + 1;
+  }
+  CgControl h0{};
+  h0.hist = c->cg_hist; h0.hist_cap = max_iter + 1;
+  *c->h_ctl = h0;
+  GN_CUDA(c, cudaMemcpyAsync(c->cg_ctl, c->h_ctl, sizeof(CgControl), cudaMemcpyHostToDevice, c->st));
+  // The host has to look at the scalars after every step only if something may end the solve early: a stop
+  // tolerance, or the termination rule of Section 4.4.  Otherwise all max_iter steps are enqueued without waiting
+  // (a system that converges exactly freezes, and the steps after that change nothing).
+  const bool rule44 = blockdiag && (c->cg_min > 0 || c->cg_share < 1.0);
+  const bool watch = tol > 0.0 || rule44;
 
-  c->launches += launch_cg_init(d_g, d_d, c->cg_r, c->cg_p, ch, nc, c->partial, c->st);
-  c->launches += launch_cg_scalars(0, c->partial, ch, nc, c->segs[mode], n_seg, tol, out2, c->st);
-  GN_CUDA(c, cudaMemcpyAsync(c->hscal + 2, out2, 2 * sizeof(double), cudaMemcpyDeviceToHost, c->st));
+  c->launches += launch_cg_init(d_g, d_d, c->cg_r, c->cg_p, ch, nc, c->partial, seg, n_seg, tol, c->cg_ctl, c->st);
   GN_TRY(check_launch(c, "cg init"));
-  GN_TRY(sync(c, "cg init"));
-  if (resnorm_host) resnorm_host[0] = sqrt(c->hscal[2]);
+  double active = 1.0;
+  if (watch) {
+    GN_CUDA(c, cudaMemcpyAsync(c->h_ctl, c->cg_ctl, sizeof(CgControl), cudaMemcpyDeviceToHost, c->st));
+    GN_TRY(sync(c, "cg init"));
+    active = c->h_ctl->out[1];
+  }
   int it = 0;
   c->bd_expect = blockdiag ? max_iter : 0;
   struct Reset { int* p; ~Reset() { *p = 0; } } reset_expect{&c->bd_expect};
-  while (it < max_iter && c->hscal[3] > 0.5) {
+  while (it < max_iter && active > 0.5) {
     // Section 4.4: all partitions stop once cg_min steps are done and the stated share of them have finished
-    if (blockdiag && it >= c->cg_min && (double)n_seg - c->hscal[3] >= c->cg_share * (double)n_seg) break;
+    if (rule44 && it >= c->cg_min && (double)n_seg - active >= c->cg_share * (double)n_seg) break;
     GN_TRY(blockdiag ? product_blockdiag_any(c, c->cg_p, c->cg_q, coef) : product_full(c, c->cg_p, c->cg_q, coef));
-    c->launches += launch_cg_dot(c->cg_p, c->cg_q, ch, nc, c->partial, c->st);
-    c->launches += launch_cg_scalars(1, c->partial, ch, nc, c->segs[mode], n_seg, tol, out2, c->st);
-    c->launches += launch_cg_update(c->cg_p, c->cg_q, d_d, c->cg_r, ch, nc, c->segs[mode], c->partial, c->st);
-    c->launches += launch_cg_scalars(2, c->partial, ch, nc, c->segs[mode], n_seg, tol, out2, c->st);
-    c->launches += launch_cg_direction(c->cg_r, c->cg_p, ch, nc, c->segs[mode], c->st);
-    GN_CUDA(c, cudaMemcpyAsync(c->hscal + 2, out2, 2 * sizeof(double), cudaMemcpyDeviceToHost, c->st));
+    c->launches += launch_cg_dot(c->cg_p, c->cg_q, ch, nc, c->partial, seg, n_seg, c->cg_ctl, c->st);
+    c->launches += launch_cg_update(c->cg_p, c->cg_q, d_d, c->cg_r, ch, nc, seg, n_seg, tol, c->partial, c->cg_ctl, c->st);
+    c->launches += launch_cg_direction(c->cg_r, c->cg_p, ch, nc, seg, c->st);
     if (d_iterates)
       GN_CUDA(c, cudaMemcpyAsync(d_iterates + (int64_t)it * c->n, d_d, c->n * sizeof(float), cudaMemcpyDeviceToDevice, c->st));
     GN_TRY(check_launch(c, "cg step"));
-    GN_TRY(sync(c, "cg step"));
+    if (watch) {
+      GN_CUDA(c, cudaMemcpyAsync(c->h_ctl, c->cg_ctl, sizeof(CgControl), cudaMemcpyDeviceToHost, c->st));
+      GN_TRY(sync(c, "cg step"));
+      active = c->h_ctl->out[1];
+    }
     ++it;
-    if (resnorm_host) resnorm_host[it] = sqrt(c->hscal[2]);
   }
-  if (iters_host) *iters_host = it;
+  // one read of the state at the end: steps in which a segment was still active, and the residual history
+  GN_CUDA(c, cudaMemcpyAsync(c->h_ctl, c->cg_ctl, sizeof(CgControl), cudaMemcpyDeviceToHost, c->st));
+  GN_TRY(sync(c, "cg solve"));
+  const int steps = watch ? it : c->h_ctl->steps;
+  if (iters_host) *iters_host = steps;
+  if (resnorm_host) {
+    const int len = c->h_ctl->hist_len < steps + 1 ? c->h_ctl->hist_len : steps + 1;
+    GN_CUDA(c, cudaMemcpy(resnorm_host, c->cg_hist, (size_t)len * sizeof(double), cudaMemcpyDeviceToHost));
+    for (int k = 0; k < len; ++k) resnorm_host[k] = sqrt(resnorm_host[k]);
+  }
   return GN_OK;
 }
 
@@ -1230,7 +1289,7 @@ gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* d
 
 // x^T y into device scalar slot (fixed-order double-precision sum of per-chunk partials)
 static void dot_to_slot(gn_ctx* c, const float* x, const float* y, int slot) {
-  c->launches += launch_cg_dot(x, y, c->chunks[0], c->n_chunks[0], c->partial, c->st);
+  c->launches += launch_cg_dot(x, y, c->chunks[0], c->n_chunks[0], c->partial, nullptr, 0, nullptr, c->st);
   c->launches += launch_sum_partials(c->partial, c->n_chunks[0], c->dscal + slot, false, c->st);
 }
 
@@ -1297,6 +1356,7 @@ gn_status gn_newton_iter(gn_ctx* c, float* d_theta, const int32_t* d_idx, int64_
 
 gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   if (!c) return GN_EINVAL;
+  if (option == 2) { if (value < 0) return fail(c, GN_EINVAL, "count must be >= 0"); c->fail_alloc_in = value; return GN_OK; }
   if (option == 0) c->group_enabled = value != 0;
   else if (option == 1) c->sk_enabled = value != 0 && c->sk_enabled;
   else return fail(c, GN_EINVAL, "unknown option");

@@ -105,9 +105,6 @@ int launch_axpby(int64_t n, float a, const float* x, float b, const float* y, fl
 int launch_split_tf32(const float* src, int64_t rows, int cols, int64_t ld, float* hi, float* lo, int64_t ld_out,
                       cudaStream_t st);
 
-// Transposed copy dst[c][r] = src[r][c] (src rows x cols).
-int launch_transpose(const float* src, int rows, int cols, float* dst, cudaStream_t st);
-
 // Stored Jacobian factors (d z^L / d s^m per sample, Section 3.3.1).  D is [rows * nL][n] with row i * nL + u.
 // factor_last: D[(i, u)][t] = WL[u * n + t] * z (1 - z), z = Zprev[i * n + t]   (layer L-1 from the linear output layer)
 int launch_factor_last(const float* WL, const float* Zprev, int64_t rows, int nL, int n, float* D, cudaStream_t st);
@@ -135,23 +132,30 @@ struct CgSeg {           // per-segment scalars, device resident
   int pad;
 };
 
-// r = -g, p = r, d = 0, partial[c] = sum r^2
+// Device-resident state of one solve: where the kernels that end in a dot product take their tickets, what the
+// last scalar update left for the host (sum of rho over segments, number of active segments), the number of steps
+// in which some segment was still active, and the history of squared residual norms.
+struct CgControl {
+  unsigned int ticket;   // zero between launches
+  int steps;
+  int hist_len, hist_cap;
+  double* hist;
+  double out[2];
+};
+
+// r = -g, p = r, d = 0, partial[c] = sum r^2; then rho = gnorm2 = sum, active = rho > 0 && (tol <= 0 || tol < 1) per segment
 int launch_cg_init(const float* g, float* d, float* r, float* p, const CgChunk* chunks, int n_chunks,
-                   double* partial, cudaStream_t st);
-// partial[c] = sum p q
+                   double* partial, CgSeg* seg, int n_seg, double tol, CgControl* ctl, cudaStream_t st);
+// partial[c] = sum p q; with seg != nullptr also pq = sum, alpha = active ? rho / pq : 0 per segment
+// (seg == nullptr: partials only, ctl unused)
 int launch_cg_dot(const float* p, const float* q, const CgChunk* chunks, int n_chunks, double* partial,
-                  cudaStream_t st);
-// d += alpha p, r -= alpha q, partial[c] = sum r^2   (alpha per segment)
+                  CgSeg* seg, int n_seg, CgControl* ctl, cudaStream_t st);
+// d += alpha p, r -= alpha q, partial[c] = sum r^2 (alpha per segment); then rho_new = sum, beta = rho_new / rho,
+// rho = rho_new, active &= !(sqrt(rho) <= tol ||g||) per segment
 int launch_cg_update(const float* p, const float* q, float* d, float* r, const CgChunk* chunks,
-                     int n_chunks, const CgSeg* seg, double* partial, cudaStream_t st);
+                     int n_chunks, CgSeg* seg, int n_seg, double tol, double* partial, CgControl* ctl, cudaStream_t st);
 // p = r + beta p   (beta per segment)
 int launch_cg_direction(const float* r, float* p, const CgChunk* chunks, int n_chunks, const CgSeg* seg,
                         cudaStream_t st);
-// phase 0: rho = gnorm2 = sum, active = rho > 0 && (tol <= 0 || sqrt(rho) > tol ||g||)
-// phase 1: pq = sum, alpha = active ? rho / pq : 0
-// phase 2: rho_new = sum; beta = active ? rho_new / rho : 0; rho = rho_new; active &= !stop
-// After each phase host_out[0] = sum over segments of rho, host_out[1] = number of active segments.
-int launch_cg_scalars(int phase, const double* partial, const CgChunk* chunks, int n_chunks, CgSeg* seg,
-                      int n_seg, double tol, double* host_out, cudaStream_t st);
 
 }  // namespace gn

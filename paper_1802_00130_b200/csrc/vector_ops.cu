@@ -3,6 +3,8 @@
 //
 // Reductions are deterministic: every block writes one partial, partials are combined in a fixed
 // order in double precision.
+#include <initializer_list>
+
 #include "gn_kernels.h"
 
 namespace gn {
@@ -241,96 +243,26 @@ __global__ void __launch_bounds__(256) factor_apply_kernel(const float* __restri
   }
 }
 
-// ---------------------------------------------------------------------------------- transpose
-__global__ void __launch_bounds__(256) transpose_kernel(const float* __restrict__ src, int rows, int cols,
-                                                        float* __restrict__ dst) {
-  __shared__ float tile[32][33];
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int j = ty; j < 32; j += 8) {
-    const int r = r0 + j, c = c0 + tx;
-    tile[j][tx] = (r < rows && c < cols) ? src[(long long)r * cols + c] : 0.f;
-  }
-  __syncthreads();
-  for (int j = ty; j < 32; j += 8) {
-    const int c = c0 + j, r = r0 + tx;
-    if (r < rows && c < cols) dst[(long long)c * rows + r] = tile[tx][j];
-  }
-}
-
 // ---------------------------------------------------------------------------------- CG
-// One block per chunk of at most kCgChunk coordinates: 256 threads x 16 strided elements.
-__global__ void __launch_bounds__(256) cg_init_kernel(const float* __restrict__ g, float* __restrict__ d,
-                                                      float* __restrict__ r, float* __restrict__ p,
-                                                      const CgChunk* __restrict__ chunks, double* __restrict__ partial) {
-  const CgChunk ch = chunks[blockIdx.x];
-  float s = 0.f;
-  for (int i = threadIdx.x; i < ch.len; i += 256) {
-    const long long k = ch.start + i;
-    const float x = -g[k];
-    d[k] = 0.f; r[k] = x; p[k] = x;
-    s = fmaf(x, x, s);
-  }
-  const double t = block_sum_256((double)s);
-  if (threadIdx.x == 0) partial[blockIdx.x] = t;
-}
+// One block per chunk of at most kCgChunk coordinates (256 threads; 16-byte accesses when the chunk starts on a
+// multiple of four coordinates).  A kernel that ends in a dot product also computes the step's scalars: every
+// block leaves its partial sum, takes a ticket, and the block that draws the last ticket adds the partials of every
+// segment in a fixed order (so the result does not depend on which block that is) and updates the per-segment
+// scalars; no separate launch, no wait.
 
-__global__ void __launch_bounds__(256) cg_dot_kernel(const float* __restrict__ p, const float* __restrict__ q,
-                                                     const CgChunk* __restrict__ chunks, double* __restrict__ partial) {
-  const CgChunk ch = chunks[blockIdx.x];
-  float s = 0.f;
-  for (int i = threadIdx.x; i < ch.len; i += 256) {
-    const long long k = ch.start + i;
-    s = fmaf(p[k], q[k], s);
-  }
-  const double t = block_sum_256((double)s);
-  if (threadIdx.x == 0) partial[blockIdx.x] = t;
-}
-
-__global__ void __launch_bounds__(256) cg_update_kernel(const float* __restrict__ p, const float* __restrict__ q,
-                                                        float* __restrict__ d, float* __restrict__ r,
-                                                        const CgChunk* __restrict__ chunks, const CgSeg* __restrict__ seg,
-                                                        double* __restrict__ partial) {
-  const CgChunk ch = chunks[blockIdx.x];
-  const float alpha = seg[ch.seg].alpha;
-  const bool live = seg[ch.seg].active != 0;
-  float s = 0.f;
-  for (int i = threadIdx.x; i < ch.len; i += 256) {
-    const long long k = ch.start + i;
-    float rk = r[k];
-    if (live) {
-      d[k] = fmaf(alpha, p[k], d[k]);
-      rk = fmaf(-alpha, q[k], rk);
-      r[k] = rk;
-    }
-    s = fmaf(rk, rk, s);
-  }
-  const double t = block_sum_256((double)s);
-  if (threadIdx.x == 0) partial[blockIdx.x] = t;
-}
-
-__global__ void __launch_bounds__(256) cg_direction_kernel(const float* __restrict__ r, float* __restrict__ p,
-                                                           const CgChunk* __restrict__ chunks,
-                                                           const CgSeg* __restrict__ seg) {
-  const CgChunk ch = chunks[blockIdx.x];
-  if (seg[ch.seg].beta == 0.f && seg[ch.seg].active == 0 && seg[ch.seg].alpha == 0.f) return;  // frozen before this step
-  const float beta = seg[ch.seg].beta;
-  for (int i = threadIdx.x; i < ch.len; i += 256) {
-    const long long k = ch.start + i;
-    p[k] = fmaf(beta, p[k], r[k]);
-  }
-}
-
-// One block.  With several segments warp w handles segments w, w + 8, ..., summing that segment's own run of the
-// chunk table; with a single segment the whole block sums it.  Every sum has a fixed order.
-__global__ void __launch_bounds__(256) cg_scalars_kernel(int phase, const double* __restrict__ partial,
-                                                         const CgChunk* __restrict__ chunks, int n_chunks,
-                                                         CgSeg* __restrict__ seg, int n_seg, double tol,
-                                                         double* __restrict__ host_out) {
+// Per-segment sums of the chunk partials and the scalar updates of one phase, by one 256-thread block.
+// phase 0: rho = gnorm2 = sum, active = rho > 0
+// phase 1: pq = sum, alpha = active ? rho / pq : 0
+// phase 2: rho_new = sum; beta = rho_new / rho; rho = rho_new; active &= !(stop rule met)
+// ctl->out[0] = sum over segments of rho, ctl->out[1] = number of active segments; after phases 0 and 2 the
+// residual norm squared is appended to the history, and a step that began with an active segment is counted.
+__device__ void cg_scalars_block(int phase, const double* partial, CgSeg* seg, int n_seg, double tol, CgControl* ctl) {
   __shared__ double seg_rho[64];
   __shared__ int seg_act[64];
+  __shared__ int was_active;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  (void)chunks; (void)n_chunks;
+  if (threadIdx.x == 0) was_active = 0;
+  __syncthreads();
   auto update = [&](int s, double acc) -> CgSeg {
     CgSeg g = seg[s];
     if (phase == 0) {
@@ -342,6 +274,7 @@ __global__ void __launch_bounds__(256) cg_scalars_kernel(int phase, const double
       if (!(acc > 0.0)) g.active = 0;
     } else {
       if (g.active) {
+        was_active = 1;
         g.beta = g.rho > 0.0 ? (float)(acc / g.rho) : 0.f;
         g.rho = acc;
         if (!(acc > 0.0) || (tol > 0.0 && sqrt(acc) <= tol * sqrt(g.gnorm2))) g.active = 0;
@@ -352,37 +285,172 @@ __global__ void __launch_bounds__(256) cg_scalars_kernel(int phase, const double
     seg[s] = g;
     return g;
   };
+  double tot = 0.0, act = 0.0;
   if (n_seg == 1) {
     const int first = seg[0].first, count = seg[0].count;
     double acc = 0.0;
-    for (int c = threadIdx.x; c < count; c += 256) acc += partial[first + c];
+    for (int c = threadIdx.x; c < count; c += 256) acc += __ldcg(partial + first + c);
     acc = block_sum_256(acc);
     if (threadIdx.x == 0) {
       const CgSeg g = update(0, acc);
-      host_out[0] = g.rho; host_out[1] = (double)g.active;
+      tot = g.rho; act = (double)g.active;
     }
+  } else {
+    for (int s0 = 0; s0 < n_seg; s0 += 64) {
+      for (int s = s0 + w; s < min(n_seg, s0 + 64); s += 8) {
+        const int first = seg[s].first, count = seg[s].count;
+        double acc = 0.0;
+        for (int c = lane; c < count; c += 32) acc += __ldcg(partial + first + c);
+        acc = warp_sum(acc);
+        if (lane == 0) {
+          const CgSeg g = update(s, acc);
+          seg_rho[s - s0] = g.rho;
+          seg_act[s - s0] = g.active;
+        }
+      }
+      __syncthreads();
+      if (threadIdx.x == 0)
+        for (int s = s0; s < min(n_seg, s0 + 64); ++s) { tot += seg_rho[s - s0]; act += seg_act[s - s0]; }
+      __syncthreads();
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    ctl->out[0] = tot; ctl->out[1] = act;
+    if (phase == 0) { ctl->steps = 0; ctl->hist_len = 0; }
+    if (phase == 2 && was_active) ctl->steps += 1;
+    if (phase != 1 && ctl->hist && ctl->hist_len < ctl->hist_cap && (phase == 0 || was_active)) ctl->hist[ctl->hist_len++] = tot;
+  }
+}
+
+// Block-wide: leave this block's partial, and tell whether this block drew the last ticket of the launch.
+__device__ __forceinline__ bool cg_last_block(double block_total, double* partial, CgControl* ctl) {
+  __shared__ int last;
+  if (threadIdx.x == 0) {
+    partial[blockIdx.x] = block_total;
+    __threadfence();
+    const unsigned t = atomicAdd(&ctl->ticket, 1u);
+    last = (t == gridDim.x - 1) ? 1 : 0;
+    if (last) { ctl->ticket = 0; __threadfence(); }
+  }
+  __syncthreads();
+  return last != 0;
+}
+
+template <typename F>
+__device__ __forceinline__ void cg_for_chunk(const CgChunk& ch, bool vec_ok, F&& body4, int& tail0) {
+  // body4(k) handles coordinates k .. k + 3 as one 16-byte access; the rest is left to the caller from tail0 on
+  tail0 = 0;
+  if (vec_ok && (ch.start & 3) == 0) {
+    const int n4 = ch.len >> 2;
+    for (int i = threadIdx.x; i < n4; i += 256) body4(ch.start + 4ll * i);
+    tail0 = n4 << 2;
+  }
+}
+
+__global__ void __launch_bounds__(256) cg_init_kernel(const float* __restrict__ g, float* __restrict__ d,
+                                                      float* __restrict__ r, float* __restrict__ p,
+                                                      const CgChunk* __restrict__ chunks, double* __restrict__ partial,
+                                                      CgSeg* seg, int n_seg, double tol, CgControl* ctl, int vec_ok) {
+  const CgChunk ch = chunks[blockIdx.x];
+  float s = 0.f;
+  int t0;
+  cg_for_chunk(ch, vec_ok != 0, [&](long long k) {
+    float4 x = *reinterpret_cast<const float4*>(g + k);
+    x.x = -x.x; x.y = -x.y; x.z = -x.z; x.w = -x.w;
+    *reinterpret_cast<float4*>(d + k) = make_float4(0.f, 0.f, 0.f, 0.f);
+    *reinterpret_cast<float4*>(r + k) = x;
+    *reinterpret_cast<float4*>(p + k) = x;
+    s += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+  }, t0);
+  for (int i = t0 + threadIdx.x; i < ch.len; i += 256) {
+    const long long k = ch.start + i;
+    const float x = -g[k];
+    d[k] = 0.f; r[k] = x; p[k] = x;
+    s = fmaf(x, x, s);
+  }
+  const double t = block_sum_256((double)s);
+  if (cg_last_block(t, partial, ctl)) cg_scalars_block(0, partial, seg, n_seg, tol, ctl);
+}
+
+// partial[c] = sum x y over chunk c; with seg != nullptr also the phase-1 scalars (alpha) by the last block
+__global__ void __launch_bounds__(256) cg_dot_kernel(const float* __restrict__ x, const float* __restrict__ y,
+                                                     const CgChunk* __restrict__ chunks, double* __restrict__ partial,
+                                                     CgSeg* seg, int n_seg, CgControl* ctl, int vec_ok) {
+  const CgChunk ch = chunks[blockIdx.x];
+  float s = 0.f;
+  int t0;
+  cg_for_chunk(ch, vec_ok != 0, [&](long long k) {
+    const float4 a = *reinterpret_cast<const float4*>(x + k);
+    const float4 b = *reinterpret_cast<const float4*>(y + k);
+    s += a.x * b.x + a.y * b.y + a.z * b.z + a.w * b.w;
+  }, t0);
+  for (int i = t0 + threadIdx.x; i < ch.len; i += 256) {
+    const long long k = ch.start + i;
+    s = fmaf(x[k], y[k], s);
+  }
+  const double t = block_sum_256((double)s);
+  if (!seg) {
+    if (threadIdx.x == 0) partial[blockIdx.x] = t;
     return;
   }
-  for (int s0 = 0; s0 < n_seg; s0 += 64) {
-    for (int s = s0 + w; s < min(n_seg, s0 + 64); s += 8) {
-      const int first = seg[s].first, count = seg[s].count;
-      double acc = 0.0;
-      for (int c = lane; c < count; c += 32) acc += partial[first + c];
-      acc = warp_sum(acc);
-      if (lane == 0) {
-        const CgSeg g = update(s, acc);
-        seg_rho[s - s0] = g.rho;
-        seg_act[s - s0] = g.active;
-      }
+  if (cg_last_block(t, partial, ctl)) cg_scalars_block(1, partial, seg, n_seg, 0.0, ctl);
+}
+
+// d += alpha p, r -= alpha q for the live segments, partial = sum r^2, then the phase-2 scalars by the last block
+__global__ void __launch_bounds__(256) cg_update_kernel(const float* __restrict__ p, const float* __restrict__ q,
+                                                        float* __restrict__ d, float* __restrict__ r,
+                                                        const CgChunk* __restrict__ chunks, CgSeg* seg, int n_seg,
+                                                        double tol, double* __restrict__ partial, CgControl* ctl,
+                                                        int vec_ok) {
+  const CgChunk ch = chunks[blockIdx.x];
+  const float alpha = seg[ch.seg].alpha;
+  const bool live = seg[ch.seg].active != 0;
+  float s = 0.f;
+  int t0;
+  cg_for_chunk(ch, vec_ok != 0, [&](long long k) {
+    float4 rk = *reinterpret_cast<const float4*>(r + k);
+    if (live) {
+      const float4 pk = *reinterpret_cast<const float4*>(p + k);
+      const float4 qk = *reinterpret_cast<const float4*>(q + k);
+      float4 dk = *reinterpret_cast<const float4*>(d + k);
+      dk.x = fmaf(alpha, pk.x, dk.x); dk.y = fmaf(alpha, pk.y, dk.y); dk.z = fmaf(alpha, pk.z, dk.z); dk.w = fmaf(alpha, pk.w, dk.w);
+      rk.x = fmaf(-alpha, qk.x, rk.x); rk.y = fmaf(-alpha, qk.y, rk.y); rk.z = fmaf(-alpha, qk.z, rk.z); rk.w = fmaf(-alpha, qk.w, rk.w);
+      *reinterpret_cast<float4*>(d + k) = dk;
+      *reinterpret_cast<float4*>(r + k) = rk;
     }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      double tot = s0 == 0 ? 0.0 : host_out[0];
-      double act = s0 == 0 ? 0.0 : host_out[1];
-      for (int s = s0; s < min(n_seg, s0 + 64); ++s) { tot += seg_rho[s - s0]; act += seg_act[s - s0]; }
-      host_out[0] = tot; host_out[1] = act;
+    s += rk.x * rk.x + rk.y * rk.y + rk.z * rk.z + rk.w * rk.w;
+  }, t0);
+  for (int i = t0 + threadIdx.x; i < ch.len; i += 256) {
+    const long long k = ch.start + i;
+    float rk = r[k];
+    if (live) {
+      d[k] = fmaf(alpha, p[k], d[k]);
+      rk = fmaf(-alpha, q[k], rk);
+      r[k] = rk;
     }
-    __syncthreads();
+    s = fmaf(rk, rk, s);
+  }
+  const double t = block_sum_256((double)s);
+  if (cg_last_block(t, partial, ctl)) cg_scalars_block(2, partial, seg, n_seg, tol, ctl);
+}
+
+__global__ void __launch_bounds__(256) cg_direction_kernel(const float* __restrict__ r, float* __restrict__ p,
+                                                           const CgChunk* __restrict__ chunks,
+                                                           const CgSeg* __restrict__ seg, int vec_ok) {
+  const CgChunk ch = chunks[blockIdx.x];
+  if (seg[ch.seg].beta == 0.f && seg[ch.seg].active == 0 && seg[ch.seg].alpha == 0.f) return;  // frozen before this step
+  const float beta = seg[ch.seg].beta;
+  int t0;
+  cg_for_chunk(ch, vec_ok != 0, [&](long long k) {
+    const float4 rk = *reinterpret_cast<const float4*>(r + k);
+    float4 pk = *reinterpret_cast<const float4*>(p + k);
+    pk.x = fmaf(beta, pk.x, rk.x); pk.y = fmaf(beta, pk.y, rk.y); pk.z = fmaf(beta, pk.z, rk.z); pk.w = fmaf(beta, pk.w, rk.w);
+    *reinterpret_cast<float4*>(p + k) = pk;
+  }, t0);
+  for (int i = t0 + threadIdx.x; i < ch.len; i += 256) {
+    const long long k = ch.start + i;
+    p[k] = fmaf(beta, p[k], r[k]);
   }
 }
 
@@ -584,35 +652,32 @@ int launch_split_tf32(const float* src, int64_t rows, int cols, int64_t ld, floa
   return 1;
 }
 
-int launch_transpose(const float* src, int rows, int cols, float* dst, cudaStream_t st) {
-  dim3 grid((cols + 31) / 32, (rows + 31) / 32);
-  transpose_kernel<<<grid, 256, 0, st>>>(src, rows, cols, dst);
+namespace {
+inline int all_aligned16(std::initializer_list<const void*> ps) {
+  for (const void* q : ps)
+    if (reinterpret_cast<uintptr_t>(q) & 15) return 0;
   return 1;
 }
+}  // namespace
 
 int launch_cg_init(const float* g, float* d, float* r, float* p, const CgChunk* chunks, int n_chunks,
-                   double* partial, cudaStream_t st) {
-  cg_init_kernel<<<n_chunks, 256, 0, st>>>(g, d, r, p, chunks, partial);
+                   double* partial, CgSeg* seg, int n_seg, double tol, CgControl* ctl, cudaStream_t st) {
+  cg_init_kernel<<<n_chunks, 256, 0, st>>>(g, d, r, p, chunks, partial, seg, n_seg, tol, ctl, all_aligned16({g, d, r, p}));
   return 1;
 }
 int launch_cg_dot(const float* p, const float* q, const CgChunk* chunks, int n_chunks, double* partial,
-                  cudaStream_t st) {
-  cg_dot_kernel<<<n_chunks, 256, 0, st>>>(p, q, chunks, partial);
+                  CgSeg* seg, int n_seg, CgControl* ctl, cudaStream_t st) {
+  cg_dot_kernel<<<n_chunks, 256, 0, st>>>(p, q, chunks, partial, seg, n_seg, ctl, all_aligned16({p, q}));
   return 1;
 }
 int launch_cg_update(const float* p, const float* q, float* d, float* r, const CgChunk* chunks,
-                     int n_chunks, const CgSeg* seg, double* partial, cudaStream_t st) {
-  cg_update_kernel<<<n_chunks, 256, 0, st>>>(p, q, d, r, chunks, seg, partial);
+                     int n_chunks, CgSeg* seg, int n_seg, double tol, double* partial, CgControl* ctl, cudaStream_t st) {
+  cg_update_kernel<<<n_chunks, 256, 0, st>>>(p, q, d, r, chunks, seg, n_seg, tol, partial, ctl, all_aligned16({p, q, d, r}));
   return 1;
 }
 int launch_cg_direction(const float* r, float* p, const CgChunk* chunks, int n_chunks, const CgSeg* seg,
                         cudaStream_t st) {
-  cg_direction_kernel<<<n_chunks, 256, 0, st>>>(r, p, chunks, seg);
-  return 1;
-}
-int launch_cg_scalars(int phase, const double* partial, const CgChunk* chunks, int n_chunks, CgSeg* seg,
-                      int n_seg, double tol, double* host_out, cudaStream_t st) {
-  cg_scalars_kernel<<<1, 256, 0, st>>>(phase, partial, chunks, n_chunks, seg, n_seg, tol, host_out);
+  cg_direction_kernel<<<n_chunks, 256, 0, st>>>(r, p, chunks, seg, all_aligned16({r, p}));
   return 1;
 }
 

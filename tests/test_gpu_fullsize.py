@@ -123,26 +123,47 @@ def test_wide4096_reduced_rows_all_quantities(wide4096_reduced, mode):
 
 def test_wide4096_fifty_cg_steps(wide4096_reduced):
     """Eq. sample-gaussnewton with the stop rule of Eq. CG-stopping-cond switched off: 50 steps on the full system of
-    the 1024-4096-4096-4096-4096-100 network over 256 subsample rows; iterates 1..10 and all 51 residual norms."""
+    the 1024-4096-4096-4096-4096-100 network over 256 subsample rows; iterates 1..10 and all 51 residual norms.
+
+    Like the 3072-1000-1000-10 system, this one has an ill-conditioned third step (its residual norm goes up there),
+    which multiplies any error in the products.  How much is measured here with the checker alone: its CG is run once
+    more with every product perturbed by a seeded relative error of the size asserted for the device's product and
+    rounded to float32; twice the deviation that run shows is the bound for the device's iterates."""
     p, ref = wide4096_reduced
     idx = np.ascontiguousarray(p["idx"][:256])
     XS = p["X"][idx]
+    th, w, C = p["theta"], p["widths"], p["C"]
     ctx = make_ctx(p)
     ctx.set_subsample(dev(idx))
+    eps = 1e-6
+    assert rel(ctx.Gv(dev(p["v"])).cpu().numpy(), orc.Gv(th, w, C, XS, p["v"])) <= eps
     g32 = ref["grad"].astype(np.float32)
-    matvec = lambda x: orc.Gv(p["theta"], p["widths"], p["C"], XS, x)
+    matvec = lambda x: orc.Gv(th, w, C, XS, x)
     _, its_ref, _ = orc.cg(matvec, g32, 1.0, 10, 0.0)
-    _, _, res_ref = orc.cg(matvec, g32, 1.0, 50, 0.0, keep_iterates=False)
+    rng = np.random.Generator(np.random.PCG64(5))
+
+    def perturbed(x):
+        q = matvec(x.astype(np.float32).astype(np.float64))
+        return (q * (1.0 + eps * rng.standard_normal(q.size))).astype(np.float32).astype(np.float64)
+
+    _, moved, _ = orc.cg(perturbed, g32, 1.0, 6, 0.0)
+    moved_by = [rel(moved[k], its_ref[k]) for k in range(6)]
+    del moved
+    bound = [max(1e-4, 2.0 * max(moved_by[: k + 1])) for k in range(6)]
+    bound += [bound[-1]] * 4
+    assert bound[-1] <= 5e-3                   # (the system amplifies by about a thousand, not more)
     _, its, _, iterates = ctx.cg_solve(dev(g32), 1.0, blockdiag=False, max_iter=10, tol=0.0, keep_iterates=True)
     assert its == 10
     for k in range(10):
-        assert rel(iterates[k].cpu().numpy(), its_ref[k]) <= 1e-4, k
-    del iterates
+        assert rel(iterates[k].cpu().numpy(), its_ref[k]) <= bound[k], (k, bound[k])
+    del iterates, its_ref
+    _, _, res_ref = orc.cg(matvec, g32, 1.0, 50, 0.0, keep_iterates=False)
     d, its, res = ctx.cg_solve(dev(g32), 1.0, blockdiag=False, max_iter=50, tol=0.0)
     assert its == 50
+    # r_k = -g - A d_k: an iterate that is off by `bound` relative moves the residual by at most about bound * ||g||
     tot = [float(r[0]) for r in res_ref]
     for k in range(51):
-        assert abs(res[k] - tot[k]) <= 1e-3 * tot[k] + 1e-4 * tot[0], k
+        assert abs(res[k] - tot[k]) <= 1e-3 * tot[k] + bound[-1] * tot[0], k
     ctx.close()
 
 

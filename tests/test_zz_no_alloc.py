@@ -54,3 +54,47 @@ def test_sizes_beyond_the_built_in_scratch_are_refused_without_a_launch():
         gn.thin_m_gemm_noalloc(torch.zeros((64, 17), device="cuda"), torch.zeros((64, 64), device="cuda"),
                                torch.zeros((17, 64), device="cuda"))
     assert e.value.status == 1
+
+
+_FIRST_CALL_SCRIPT = r"""
+import sys
+sys.path.insert(0, sys.argv[1])
+import numpy as np, torch
+import paper_1802_00130_b200 as gn
+rng = np.random.Generator(np.random.PCG64(7))
+rows, M, N = 3000, 10, 2000
+A = torch.from_numpy(rng.standard_normal((rows, M), dtype=np.float32)).cuda()
+B = torch.from_numpy(rng.standard_normal((rows, N), dtype=np.float32)).cuda()
+out = torch.empty((M, N), dtype=torch.float32, device="cuda")
+ref = A.double().t() @ B.double()
+side = torch.cuda.Stream()
+torch.cuda.synchronize()
+frees = []
+for k in range(4):                      # the very first call into the library in this process is this entry point
+    st = side if k == 2 else None       # once on a stream of the caller's own
+    out.fill_(float("nan"))
+    torch.cuda.synchronize()
+    gn.thin_m_gemm_noalloc(A, B, out, stream=st)
+    torch.cuda.synchronize()
+    frees.append(torch.cuda.mem_get_info()[0])
+    err = ((out.double() - ref).norm() / ref.norm()).item()
+    assert err <= 2e-6, (k, err)
+# the first call may make the runtime place the library's code and its fixed array on the device; from the second
+# call on the device's free memory must not move by a byte
+assert frees[1] == frees[2] == frees[3], frees
+print("ok", frees)
+"""
+
+
+def test_first_library_call_in_a_fresh_process_and_no_byte_taken_afterwards():
+    """A process whose first call into the library is this entry point (nothing else has made the runtime load the
+    library's kernels), one call on a stream of the caller's own, and the device's free memory read after every
+    call: identical from the second call on, which is what a caller whose allocator owns the rest of the memory
+    relies on."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, "-c", _FIRST_CALL_SCRIPT, root], capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stdout + out.stderr
+    assert out.stdout.strip().startswith("ok")
