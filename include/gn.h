@@ -300,12 +300,13 @@ gn_status gn_debug_activations(gn_ctx* ctx, int m, float* d_out);
 /*
  * gn_profile - switch per-launch timing of the contraction kernels on (enable != 0) or off.  While on,
  * every GEMM launch is bracketed by a pair of CUDA events on the context's stream.
- * gn_profile_read - synchronise the stream and return, for the tensor-core kernel (index 0), the
- * FP32 FMA GEMM (index 1), the streaming kernels for n_L-wide shapes (index 2) and the error-compensated
- * tensor-core kernel of GN_FP32_ACCURATE contexts (index 3): summed device time in milliseconds,
- * floating-point operations of the contractions (2 M N K per launch; for index 3 the three TF32 products
- * per term count once) and number of launches; then reset the counters.  Each output is an array of four
- * entries and may be NULL.
+ * gn_profile_read - synchronise the stream and return, for the CTA-pair tensor-core kernel that carries the large
+ * contractions (index 0), the FP32 FMA GEMM (index 1), the streaming kernels for n_L-wide shapes (index 2), the
+ * error-compensated tensor-core kernel of GN_FP32_ACCURATE contexts (index 3) and the one-CTA tensor-core kernel
+ * that takes the n_L-wide and small-M shapes in TF32 mode (index 4): summed device time in milliseconds,
+ * floating-point operations of the contractions (2 M N K per launch, summed over the problems of a grouped
+ * launch; for index 3 the three TF32 products per term count once) and number of launches; then reset the
+ * counters.  Each output is an array of FIVE entries and may be NULL.
  */
 gn_status gn_profile(gn_ctx* ctx, int enable);
 gn_status gn_profile_read(gn_ctx* ctx, double* gemm_ms, double* gemm_flop, int64_t* gemm_launches);
@@ -330,8 +331,9 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
  * one launch per contraction); option 1: cutting left-over tiles along K between CTA pairs (value 0 = whole
  * tiles only; cannot be switched back on); option 2: failure injection on the host: the value-th device allocation
  * the context asks for from now on is refused as if the device were out of memory (0 = off); nothing on the
- * device is touched by it.  Results do not depend on option 0 (tiles are computed identically); GN_EINVAL for an
- * unknown option.
+ * device is touched by it; option 3: the bias column sums and the n_L-row weight block of a layer on a side stream
+ * next to the layer's large contractions (value 0 = everything on the context's stream).  Results do not depend on
+ * options 0 and 3 (tiles and sums are computed identically); GN_EINVAL for an unknown option.
  */
 gn_status gn_debug_option(gn_ctx* ctx, int option, int value);
 

@@ -304,11 +304,12 @@ class GnContext:
         self._check(self._lib.gn_profile(self._h, int(bool(enable))))
 
     def profile_read(self):
-        """Per-kernel GEMM timing since the last read: {"tensor": {...}, "ffma": {...}, "thin": {...}, "tensor_x3": {...}}."""
-        ms, flop, cnt = (_dbl * 4)(), (_dbl * 4)(), (_i64 * 4)()
+        """Per-kernel GEMM timing since the last read: {"tensor": {...}, "ffma": {...}, "thin": {...}, "tensor_x3": {...},
+        "tensor_1cta": {...}} ("tensor" = the CTA-pair kernel)."""
+        ms, flop, cnt = (_dbl * 5)(), (_dbl * 5)(), (_i64 * 5)()
         self._check(self._lib.gn_profile_read(self._h, ms, flop, cnt))
         return {name: {"ms": ms[k], "flop": flop[k], "launches": cnt[k]}
-                for k, name in enumerate(("tensor", "ffma", "thin", "tensor_x3"))}
+                for k, name in enumerate(("tensor", "ffma", "thin", "tensor_x3", "tensor_1cta"))}
 
     def debug_gemm(self, kind, A, B, a_kmajor=True, b_kmajor=True):
         """Test hook: D[M][N] from A ([M][K] or [K][M]) and B ([N][K] or [K][N]); kind 0 tensor-core, 1 FMA."""

@@ -22,6 +22,12 @@ struct gn_ctx {
   const float* dY = nullptr;
   gn_precision prec = GN_FP32_ACCURATE;
   cudaStream_t st = nullptr;
+  // side stream: the bias column sums and the n_L-row weight block of a layer are independent of the layer's large
+  // contractions and small enough to run beside them; they are forked off after the layer's delta is ready and
+  // joined before the product (or row batch) ends
+  cudaStream_t st2 = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  bool side_enabled = true, side_open = false;
   int64_t n = 0;
   std::vector<int64_t> w_off, b_off;  // [m], m = 1..L (entry 0 unused)
   int64_t batch_rows = 32768;
@@ -168,6 +174,29 @@ gn_status check_launch(gn_ctx* c, const char* where) {
   return GN_OK;
 }
 
+// Side stream: everything enqueued on the main stream so far happens before what follows on the side stream.
+cudaStream_t side_fork(gn_ctx* c) {
+  if (!c->side_enabled || !c->st2) return c->st;
+  cudaEventRecord(c->ev_fork, c->st);
+  cudaStreamWaitEvent(c->st2, c->ev_fork, 0);
+  c->side_open = true;
+  return c->st2;
+}
+// ... and everything on the side stream so far happens before what follows on the main stream.
+void side_join(gn_ctx* c) {
+  if (!c->side_open) return;
+  cudaEventRecord(c->ev_join, c->st2);
+  cudaStreamWaitEvent(c->st, c->ev_join, 0);
+  c->side_open = false;
+}
+struct SideJoin { gn_ctx* c; ~SideJoin() { side_join(c); } };   // joins on every way out of a launch sequence
+
+// Before a workspace that side-stream kernels may still read is released.
+void quiesce(gn_ctx* c) {
+  cudaStreamSynchronize(c->st);
+  if (c->st2) cudaStreamSynchronize(c->st2);
+}
+
 // Synchronise the stream; also fetch the tensor-core pipeline's timeout word.
 gn_status sync(gn_ctx* c, const char* where) {
   cudaError_t e = cudaMemcpyAsync(c->h_err + 1, c->err_flag + 1, sizeof(int), cudaMemcpyDeviceToHost, c->st);
@@ -186,7 +215,8 @@ gn_status sync(gn_ctx* c, const char* where) {
 
 gn_status ensure_sk_workspace(gn_ctx* c);
 
-void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
+void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind, cudaStream_t st = nullptr) {
+  if (!st) st = c->st;
   gn_ctx::EvPair* e = nullptr;
   if (c->profiling) {
     if (c->ev_used == c->ev.size()) {
@@ -196,8 +226,10 @@ void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
     if (c->ev_used < c->ev.size()) {
       e = &c->ev[c->ev_used++];
       e->flop = 2.0 * g.M * (double)g.N * ((double)g.K1 + (g.A2 ? (double)g.K2 : 0.0));
-      e->kind = kind;
-      cudaEventRecord(e->a, c->st);
+      // the one-CTA tensor-core kernel (n_L-wide and small-M shapes, bound by memory) is counted apart from the
+      // CTA-pair kernel that carries the large contractions
+      e->kind = (kind == 0 && !(g.two_cta >= 0 ? g.two_cta != 0 : (g.M > 128 && g.N >= 128))) ? 4 : kind;
+      cudaEventRecord(e->a, st);
     }
   }
   if (kind == 0) {
@@ -205,19 +237,19 @@ void run_gemm_kind(gn_ctx* c, const GemmArgs& g, int kind) {
     const bool sk = c->sk_enabled && g.two_cta != 2;
     GemmArgs g2 = g;
     if (g2.two_cta == 2) g2.two_cta = 1;
-    const int r = launch_gemm_tf32(g2, c->err_flag + 1, sk ? c->sk_ws : nullptr, sk ? c->sk_flags : nullptr, c->st);
+    const int r = launch_gemm_tf32(g2, c->err_flag + 1, sk ? c->sk_ws : nullptr, sk ? c->sk_flags : nullptr, st);
     if (r < 0) { c->sticky = GN_ECUDA; c->err = "cuTensorMapEncodeTiled failed"; }
     else c->launches += r;
   } else if (kind == 3) {
-    const int r = launch_gemm_tf32x3(g, c->err_flag + 1, c->st);
+    const int r = launch_gemm_tf32x3(g, c->err_flag + 1, st);
     if (r < 0) { c->sticky = GN_ECUDA; c->err = "the error-compensated tensor-core kernel could not be launched"; c->x3_usable = false; }
     else c->launches += r;
   } else if (kind == 2) {
-    c->launches += launch_gemm_thin(g, c->thin_scratch, c->st);
+    c->launches += launch_gemm_thin(g, c->thin_scratch, st);
   } else {
-    c->launches += launch_gemm_ffma(g, c->st);
+    c->launches += launch_gemm_ffma(g, st);
   }
-  if (e) cudaEventRecord(e->b, c->st);
+  if (e) cudaEventRecord(e->b, st);
 }
 
 gn_status ensure_sk_workspace(gn_ctx* c) {
@@ -326,7 +358,7 @@ bool run_gemm_x3(gn_ctx* c, const GemmArgs& g) {
 // Kernel choice: streaming kernels for the n_L-wide shapes (both precisions: they are exact FP32),
 // the tensor-core kernel in TF32 mode when TMA can address the operands and, in its error-compensated
 // form, in FP32-accurate mode when the shape suits the CTA-pair kernel; else the FP32 FMA GEMM.
-void run_gemm(gn_ctx* c, const GemmArgs& g) {
+void run_gemm(gn_ctx* c, const GemmArgs& g, cudaStream_t st = nullptr) {
   ++c->gemm_seq;
   const ThinKind thin = gemm_thin_kind(g);
   // In TF32 mode the n_L-wide forward products go to the tensor-core kernel as one 32- or 64-column
@@ -335,17 +367,17 @@ void run_gemm(gn_ctx* c, const GemmArgs& g) {
   if (thin != THIN_NONE && !thin_n_on_tensor) {
     const int64_t need = gemm_thin_scratch_floats(g);
     if (need > c->thin_cap) {
-      cudaStreamSynchronize(c->st);
+      quiesce(c);
       dev_free(c, c->thin_scratch, c->thin_cap);
       c->thin_cap = 0;
       if (dev_alloc(c, &c->thin_scratch, need) != GN_OK) { c->sticky = GN_ENOMEM; return; }
       c->thin_cap = need;
     }
-    run_gemm_kind(c, g, 2);
+    run_gemm_kind(c, g, 2, st);
     return;
   }
   if (c->prec == GN_FP32_ACCURATE && c->acc_method != 1 && run_gemm_x3(c, g)) return;
-  run_gemm_kind(c, g, (c->prec == GN_TF32 && gemm_tf32_eligible(g)) ? 0 : 1);
+  run_gemm_kind(c, g, (c->prec == GN_TF32 && gemm_tf32_eligible(g)) ? 0 : 1, st);
 }
 
 // Independent contractions issued together (any order is allowed).  In TF32 mode those that suit the CTA-pair
@@ -410,6 +442,7 @@ gn_status ensure_partials(gn_ctx* c, int64_t count) {
 gn_status ensure_colsum(gn_ctx* c, int64_t rows, int cols) {
   const int64_t need = colsum_scratch_floats(rows, cols);
   if (need <= c->colsum_cap) return GN_OK;
+  quiesce(c);
   dev_free(c, c->colsum_scratch, c->colsum_cap);
   c->colsum_cap = 0;
   GN_TRY(dev_alloc(c, &c->colsum_scratch, need));
@@ -458,7 +491,7 @@ gn_status bias_block(gn_ctx* c, int m, const float* ds, int64_t rows, float alph
                      float* out) {
   GN_TRY(ensure_colsum(c, rows, c->w[m]));
   c->launches += launch_colsum(ds, rows, c->w[m], c->w[m], alpha, cin + c->b_off[m], beta, out + c->b_off[m],
-                               c->colsum_scratch, c->st);
+                               c->colsum_scratch, side_fork(c));
   return GN_OK;
 }
 
@@ -493,12 +526,21 @@ gn_status layer_backward(gn_ctx* c, int m, const float* ds_w, int64_t w_rows, co
   int n = 0;
   gs[n++] = weight_block_args(c, m, ds_w, Zprev, w_rows, alpha, cin, beta, out, w_padded);
   if (m > 1) gs[n++] = backward_data_args(c, m, ds_d, d_rows, Zprev, z_rows, dst, ds_w == ds_d && w_rows == d_rows);
+  if (n == 2 && gemm_thin_kind(gs[0]) == THIN_M && c->side_enabled && c->st2) {
+    // the n_L-row weight block streams the same rows as the activation gradient but shares nothing else with it
+    GN_TRY(bias_block(c, m, ds_w, w_rows, alpha, cin, beta, out));
+    run_gemm(c, gs[0], side_fork(c));
+    run_gemm(c, gs[1]);
+    return GN_OK;
+  }
+  GN_TRY(bias_block(c, m, ds_w, w_rows, alpha, cin, beta, out));
   run_gemm_group(c, gs, n);
-  return bias_block(c, m, ds_w, w_rows, alpha, cin, beta, out);
+  return GN_OK;
 }
 
 // out = coef v + (1/|S|) J^T (2 J v) over the stored subsample (Eq. sampled-Gauss).
 gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
+  SideJoin side_guard{c};
   const int L = c->L;
   const int64_t nS = c->nS;
   for (int m = 1; m <= L; ++m) {
@@ -529,6 +571,7 @@ gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
 // pulled back to layer k only; the L streams are stacked along rows, stream j occupying rows
 // [(j-1)|S|, j|S|) of every buffer at or above layer j, so each layer runs one stacked GEMM.
 gn_status product_blockdiag(gn_ctx* c, const float* v, float* out, float coef) {
+  SideJoin side_guard{c};
   const int L = c->L;
   const int64_t nS = c->nS;
   for (int k = 1; k <= L; ++k) {
@@ -600,6 +643,7 @@ gn_status ensure_factors(gn_ctx* c) {
 }
 
 gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float coef) {
+  SideJoin side_guard{c};
   GN_TRY(ensure_factors(c));
   const int L = c->L, nL = c->w[L];
   const int64_t nS = c->nS;
@@ -642,6 +686,7 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
 // Q_a[:, T_b] = D[:, :, T_b]^T 2 D[:, :, T_b] U_a[:, T_b]; then out_W[T_a, :] = Z_{m-1}[:, T_a]^T Q_a / |S|.
 // At the output layer D = I, so Q_a = 2 U_a.
 gn_status product_split(gn_ctx* c, const float* v, float* out, float coef) {
+  SideJoin side_guard{c};
   const int L = c->L, nL = c->w[L];
   const int64_t nS = c->nS;
   if (L >= 2) {
@@ -753,6 +798,7 @@ gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
         GN_CUDA(c, cudaMemsetAsync(c->partial + b * per_batch + used, 0, (per_batch - used) * sizeof(double), c->st));
     }
     if (d_grad) {
+      SideJoin side_guard{c};     // the next batch overwrites what the side stream reads
       for (int m = L; m >= 1; --m) {
         const float* Zprev = m == 1 ? X0 : c->Zb[m - 1];
         const float* cin0 = b == 0 ? c->theta : d_grad;
@@ -920,6 +966,9 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
     if ((s = dev_alloc(c, &c->err_flag, 2)) != GN_OK) break;
     if (cudaMemset(c->err_flag, 0, 2 * sizeof(int)) != cudaSuccess) { s = GN_ECUDA; break; }
     if (cudaMallocHost(&c->hscal, 16 * sizeof(double)) != cudaSuccess) { s = GN_ENOMEM; break; }
+    if (cudaStreamCreateWithFlags(&c->st2, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) { s = GN_ECUDA; break; }
     if (cudaMallocHost(&c->h_err, 2 * sizeof(int)) != cudaSuccess) { s = GN_ENOMEM; break; }
     c->h_err[0] = c->h_err[1] = 0;
     if ((s = build_chunks(c, false)) != GN_OK) break;
@@ -931,7 +980,10 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
 
 gn_status gn_destroy(gn_ctx* c) {
   if (!c) return GN_OK;
-  cudaStreamSynchronize(c->st);
+  quiesce(c);
+  if (c->st2) cudaStreamDestroy(c->st2);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
   for (auto& o : c->owned)
     if (o.p) cudaFree(o.p);
   for (auto& p : c->ev) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
@@ -1234,16 +1286,16 @@ gn_status gn_profile(gn_ctx* c, int enable) {
 gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t* gemm_launches) {
   if (!c) return GN_EINVAL;
   GN_TRY(sync(c, "profile_read"));
-  double ms[4] = {0.0, 0.0, 0.0, 0.0}, flop[4] = {0.0, 0.0, 0.0, 0.0};
-  int64_t cnt[4] = {0, 0, 0, 0};
+  double ms[5] = {0.0, 0.0, 0.0, 0.0, 0.0}, flop[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
+  int64_t cnt[5] = {0, 0, 0, 0, 0};
   for (size_t i = 0; i < c->ev_used; ++i) {
     float t = 0.f;
-    const int k = c->ev[i].kind < 0 || c->ev[i].kind > 3 ? 1 : c->ev[i].kind;
+    const int k = c->ev[i].kind < 0 || c->ev[i].kind > 4 ? 1 : c->ev[i].kind;
     if (cudaEventElapsedTime(&t, c->ev[i].a, c->ev[i].b) == cudaSuccess) ms[k] += t;
     flop[k] += c->ev[i].flop;
     cnt[k] += 1;
   }
-  for (int k = 0; k < 4; ++k) {
+  for (int k = 0; k < 5; ++k) {
     if (gemm_ms) gemm_ms[k] = ms[k];
     if (gemm_flop) gemm_flop[k] = flop[k];
     if (gemm_launches) gemm_launches[k] = cnt[k];
@@ -1357,6 +1409,7 @@ gn_status gn_newton_iter(gn_ctx* c, float* d_theta, const int32_t* d_idx, int64_
 gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   if (!c) return GN_EINVAL;
   if (option == 2) { if (value < 0) return fail(c, GN_EINVAL, "count must be >= 0"); c->fail_alloc_in = value; return GN_OK; }
+  if (option == 3) { quiesce(c); c->side_enabled = value != 0; return GN_OK; }
   if (option == 0) c->group_enabled = value != 0;
   else if (option == 1) c->sk_enabled = value != 0 && c->sk_enabled;
   else return fail(c, GN_EINVAL, "unknown option");

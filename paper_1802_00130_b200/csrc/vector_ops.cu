@@ -85,8 +85,9 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const float* __rest
 }
 
 // 16-byte version: grid (ceil(cols/128), ceil(rows/CS_ROWS)); a warp covers 128 columns of a row,
-// 8 warps stride rows with four rows in flight per thread.
-__global__ void __launch_bounds__(256) colsum_partial_vec_kernel(const float* __restrict__ A, long long rows, int cols,
+// 8 warps stride rows with four rows in flight per thread.  Held to 40 registers so that a block fits on an SM
+// beside a CTA of the tensor-core kernel (320 threads x 168 registers): the sums run on a side stream under it.
+__global__ void __launch_bounds__(256, 6) colsum_partial_vec_kernel(const float* __restrict__ A, long long rows, int cols,
                                                                  long long lda, float* __restrict__ scratch) {
   __shared__ float4 sh[8][32];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -96,16 +97,18 @@ __global__ void __launch_bounds__(256) colsum_partial_vec_kernel(const float* __
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
   if (c < cols) {
     long long r = r0 + w;
-    for (; r + 24 < r1; r += 32) {
-      const float4 x0 = __ldg(reinterpret_cast<const float4*>(A + r * lda + c));
-      const float4 x1 = __ldg(reinterpret_cast<const float4*>(A + (r + 8) * lda + c));
-      const float4 x2 = __ldg(reinterpret_cast<const float4*>(A + (r + 16) * lda + c));
-      const float4 x3 = __ldg(reinterpret_cast<const float4*>(A + (r + 24) * lda + c));
+    const float4* ptr = reinterpret_cast<const float4*>(A + r * lda + c);
+    const long long step = 2 * lda;                       // eight rows, in 16-byte units
+    for (; r + 24 < r1; r += 32, ptr += 4 * step) {
+      const float4 x0 = __ldg(ptr);
+      const float4 x1 = __ldg(ptr + step);
+      const float4 x2 = __ldg(ptr + 2 * step);
+      const float4 x3 = __ldg(ptr + 3 * step);
       s.x += (x0.x + x1.x) + (x2.x + x3.x); s.y += (x0.y + x1.y) + (x2.y + x3.y);
       s.z += (x0.z + x1.z) + (x2.z + x3.z); s.w += (x0.w + x1.w) + (x2.w + x3.w);
     }
-    for (; r < r1; r += 8) {
-      const float4 x = __ldg(reinterpret_cast<const float4*>(A + r * lda + c));
+    for (; r < r1; r += 8, ptr += step) {
+      const float4 x = __ldg(ptr);
       s.x += x.x; s.y += x.y; s.z += x.z; s.w += x.w;
     }
   }

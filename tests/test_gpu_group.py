@@ -1,5 +1,6 @@
-"""Independent contractions of a layer issued as one launch of the CTA-pair kernel (TF32 mode): same bits as one
-launch per contraction, and the usual bound against the float64 checker."""
+"""Independent work of a layer issued together: its large contractions as one launch of the CTA-pair kernel (TF32
+mode), its bias column sums and n_L-row weight block on a side stream.  Same bits as one launch after the other on
+one stream, and the usual bound against the float64 checker."""
 import numpy as np
 import pytest
 
@@ -23,10 +24,11 @@ def test_grouped_launches_give_the_bits_of_single_launches(name):
     import torch
     p = CASES[name]()
     outs = []
-    for grouped in (0, 1):
+    for grouped, side in ((0, 0), (1, 1), (1, 0), (0, 1)):
         ctx = make_ctx(p, "tf32")
-        ctx.debug_option(1, 0)                  # whole tiles only in both runs: K slices change the order of sums
+        ctx.debug_option(1, 0)                  # whole tiles only in every run: K slices change the order of sums
         ctx.debug_option(0, grouped)
+        ctx.debug_option(3, side)
         ctx.set_subsample(dev(p["idx"]))
         v = dev(p["v"])
         res = [ctx.Gv(v).clone()]
@@ -37,8 +39,9 @@ def test_grouped_launches_give_the_bits_of_single_launches(name):
         launches = ctx.kernel_launches
         outs.append((res, launches))
         ctx.close()
-    for a, b in zip(outs[0][0], outs[1][0]):
-        assert torch.equal(a, b)
+    for other in outs[1:]:
+        for a, b in zip(outs[0][0], other[0]):
+            assert torch.equal(a, b)
     assert outs[1][1] < outs[0][1]              # fewer launches: something was in fact grouped
     XS = p["X"][p["idx"]]
     th, w, C = p["theta"], p["widths"], p["C"]
