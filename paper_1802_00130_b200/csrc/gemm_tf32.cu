@@ -25,6 +25,8 @@
 // code in global memory and the CTA drains and exits (tensor memory is always released).
 #include <cuda.h>
 
+#include <utility>
+
 #include "gn_kernels.h"
 
 namespace gn {
@@ -76,6 +78,14 @@ __device__ __forceinline__ unsigned long long globaltimer() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+
+// Programmatic dependent launch.  The kernels below are launched with the stream-serialisation attribute, so
+// their CTAs may become resident, set up their barriers and allocate tensor memory while the kernel before
+// them in the stream is still draining; nothing of global memory is touched before grid_dep_wait() returns,
+// which is when that kernel has completed and its writes are visible.  grid_dep_launch() lets the kernel
+// after this one do the same.  Without the attribute both are no-ops.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
@@ -160,6 +170,25 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Accumulator read in the 16 x 256-bit fragment shape: one instruction covers 16 tensor-memory lanes (rows) and
+// 32 columns; thread t of the warp receives, in register 4j + 2e + i (j = 0..3, e = 0..1, i = 0..1), the element
+// of row (t / 4) + 8 e and column 8 j + 2 (t mod 4) + i.  Four neighbouring threads hold 32 contiguous bytes of a
+// row, so a warp-wide 8-byte access to global memory touches 8 rows x one full 32-byte sector each, where the
+// 32 x 32-bit shape (lane = row) makes every access touch 32 rows x half a sector: half the requests per byte
+// on the load/store unit, which is what the epilogue is bound by.  The caller waits (tmem_ld_wait) before use.
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -217,6 +246,8 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dep_wait();
+  grid_dep_launch();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer (TMA issue spread over lanes)
@@ -517,6 +548,8 @@ gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constan
   cluster_sync_all();      // barriers of both CTAs are initialised before anyone signals across the pair
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dep_wait();
+  grid_dep_launch();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer (both CTAs)
@@ -605,9 +638,11 @@ gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constan
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    // Fragment layout of tmem_ld_16x256b_x4: this thread's 32 values of a 32 x 32 chunk are v[h][4j + 2e + i] =
+    // element (row 16h + 8e + lane/4, column 8j + 2 (lane%4) + i) of the warp's quadrant.
     const int quad = warp & 3;
     const int half = (warp - 2) >> 2;
-    const int row = quad * 32 + lane;                          // row of this CTA's 128-row block
+    const int rsub = lane >> 2, csub = (lane & 3) * 2;
     int ti = 0;
     Work w;
     for (int wi = 0; next_work(gp, pair, wi, w); ++wi, ++ti) {
@@ -623,18 +658,26 @@ gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constan
       if (!good) break;
       tc_fence_after();
       const int n_chunks = min(bn / 32, (p.N - n0 + 31) / 32);   // column chunks of this tile that exist
+      const uint32_t tq = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX);
       int sl = 0, grp = 0;                                       // slice index and first pair of the tile's group
       if (w.sliced) {
         grp = (pair / p.slices) * p.slices;
         sl = pair - grp;
         // 1. raw accumulator of this slice to the workspace slot of this pair
-        float* wsw = p.sk_ws + (((long long)pair * 2 + rank) * BM + row) * BN_MAX;
+        float* wsw = p.sk_ws + (((long long)pair * 2 + rank) * BM + quad * 32 + rsub) * BN_MAX + csub;
         for (int c = half; c < n_chunks; c += 2) {
-          float v[32];
-          tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
+          float v[2][16];
+          tmem_ld_16x256b_x4(tq + (uint32_t)(c * 32), v[0]);
+          tmem_ld_16x256b_x4(tq + (16u << 16) + (uint32_t)(c * 32), v[1]);
+          tmem_ld_wait();
 #pragma unroll
-          for (int q = 0; q < 8; ++q)
-            __stcg(reinterpret_cast<float4*>(wsw + c * 32) + q, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
+          for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                __stcg(reinterpret_cast<float2*>(wsw + (long long)(16 * h + 8 * e) * BN_MAX + c * 32 + 8 * j),
+                       make_float2(v[h][4 * j + 2 * e], v[h][4 * j + 2 * e + 1]));
         }
         // the accumulator is free again; the tensor pipe has no further use for it in this pair
         tc_fence_before();
@@ -662,74 +705,107 @@ gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constan
         if (!good) break;
       }
       {
-        const int m = m0 + row;
-        const bool m_ok = m < p.M;
-        const float* zrow = p.dsig ? p.dsig + (long long)((m / p.dsig_div) % p.dsig_rows) * p.ld_dsig : nullptr;
-        const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
-        float* drow = p.D + (long long)m * p.ldd;
+        const int mq = m0 + quad * 32 + rsub;                    // this thread's rows are mq + 16h + 8e
+        const float* const dsig = p.dsig;
+        const float* const cin = p.cin;
         const float* const bias = p.bias;
+        float* const D = p.D;
+        const long long ldd = p.ldd, ld_dsig = p.ld_dsig, ld_cin = p.ld_cin;
+        const int dsig_rows = p.dsig_rows, dsig_div = p.dsig_div;
         const float alpha = p.alpha, beta = p.beta;
-        const int N = p.N, sigm = p.sigmoid, vec_epi = p.vec_epi;
+        const int M = p.M, N = p.N, sigm = p.sigmoid, vec_epi = p.vec_epi;
         // whole tile: this warp's chunks are half, half + 2, ...; sliced tile: the pair's share of the
         // chunks is sl, sl + slices, ..., dealt alternately to the two warps of a quadrant
         const int c_first = w.sliced ? sl + half * p.slices : half;
         const int c_step = w.sliced ? 2 * p.slices : 2;
         for (int c = c_first; c < n_chunks; c += c_step) {
-          const int nb = n0 + c * 32;
-          const bool fullc = vec_epi && nb + 32 <= N;
-          float4 zc[8], ci[8];
-          if (fullc && m_ok) {
+          const int nb = n0 + c * 32 + csub;                     // this thread's columns are nb + 8j, nb + 8j + 1
+          const bool fullc = vec_epi && n0 + c * 32 + 32 <= N;   // warp-uniform: whole chunk in range, 16-byte aligned rows
+          float2 zc[2][8], ci[2][8];                             // [h][4e + j]
+          if (fullc) {                        // all global reads of the chunk in flight before anything waits
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              zc[q] = zrow ? __ldg(reinterpret_cast<const float4*>(zrow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-              ci[q] = crow ? __ldg(reinterpret_cast<const float4*>(crow + nb) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const int m = mq + 16 * h + 8 * e;
+                const bool m_ok = m < M;
+                const float* zrow = (dsig && m_ok) ? dsig + (long long)((m / dsig_div) % dsig_rows) * ld_dsig + nb : nullptr;
+                const float* crow = (cin && m_ok) ? cin + (long long)m * ld_cin + nb : nullptr;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  zc[h][4 * e + j] = zrow ? __ldg(reinterpret_cast<const float2*>(zrow + 8 * j)) : make_float2(0.f, 0.f);
+                  ci[h][4 * e + j] = crow ? __ldg(reinterpret_cast<const float2*>(crow + 8 * j)) : make_float2(0.f, 0.f);
+                }
+              }
           }
-          float v[32];
-          if (!w.sliced) {
-            tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN_MAX + c * 32), v);
-          } else {
-            // sum of the slices' partials, slice 0 first
+          float2 bz[4];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = 0.f;
-            for (int s2 = 0; s2 < p.slices; ++s2) {
-              const float* wsr = p.sk_ws + (((long long)(grp + s2) * 2 + rank) * BM + row) * BN_MAX + c * 32;
+          for (int j = 0; j < 4; ++j)
+            bz[j] = (bias && fullc) ? __ldg(reinterpret_cast<const float2*>(bias + nb + 8 * j)) : make_float2(0.f, 0.f);
 #pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                const float4 x = __ldcg(reinterpret_cast<const float4*>(wsr) + q);
-                v[4 * q] += x.x; v[4 * q + 1] += x.y; v[4 * q + 2] += x.z; v[4 * q + 3] += x.w;
+          for (int h = 0; h < 2; ++h) {         // one 16-row half of the chunk at a time (16 accumulator registers live)
+            float v[16];
+            if (!w.sliced) {
+              tmem_ld_16x256b_x4(tq + ((uint32_t)(16 * h) << 16) + (uint32_t)(c * 32), v);
+              tmem_ld_wait();
+            } else {
+              // sum of the slices' partials, slice 0 first
+#pragma unroll
+              for (int i = 0; i < 16; ++i) v[i] = 0.f;
+              for (int s2 = 0; s2 < p.slices; ++s2) {
+                const float* wsr = p.sk_ws + (((long long)(grp + s2) * 2 + rank) * BM + quad * 32 + rsub + 16 * h) * BN_MAX + csub + c * 32;
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    const float2 x = __ldcg(reinterpret_cast<const float2*>(wsr + (long long)(8 * e) * BN_MAX + 8 * j));
+                    v[4 * j + 2 * e] += x.x; v[4 * j + 2 * e + 1] += x.y;
+                  }
               }
             }
-          }
-          if (!m_ok) continue;
-          if (fullc) {
+            if (fullc) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (bias) bz = __ldg(reinterpret_cast<const float4*>(bias + nb) + q);
-              float x[4] = {v[4 * q] + bz.x, v[4 * q + 1] + bz.y, v[4 * q + 2] + bz.z, v[4 * q + 3] + bz.w};
-              const float z[4] = {zc[q].x, zc[q].y, zc[q].z, zc[q].w};
-              const float cc[4] = {ci[q].x, ci[q].y, ci[q].z, ci[q].w};
+              for (int e = 0; e < 2; ++e) {
+                const int m = mq + 16 * h + 8 * e;
+                if (m >= M) continue;
+                float* drow = D + (long long)m * ldd + nb;
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                if (sigm) x[j] = 1.f / (1.f + __expf(-x[j]));
-                if (zrow) x[j] *= z[j] * (1.f - z[j]);
-                x[j] *= alpha;
-                if (crow) x[j] = fmaf(beta, cc[j], x[j]);
+                for (int j = 0; j < 4; ++j) {
+                  float x[2] = {v[4 * j + 2 * e] + bz[j].x, v[4 * j + 2 * e + 1] + bz[j].y};
+                  const float z[2] = {zc[h][4 * e + j].x, zc[h][4 * e + j].y};
+                  const float cc[2] = {ci[h][4 * e + j].x, ci[h][4 * e + j].y};
+#pragma unroll
+                  for (int i = 0; i < 2; ++i) {
+                    if (sigm) x[i] = 1.f / (1.f + __expf(-x[i]));
+                    if (dsig) x[i] *= z[i] * (1.f - z[i]);
+                    x[i] *= alpha;
+                    if (cin) x[i] = fmaf(beta, cc[i], x[i]);
+                  }
+                  *reinterpret_cast<float2*>(drow + 8 * j) = make_float2(x[0], x[1]);
+                }
               }
-              reinterpret_cast<float4*>(drow + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
-            }
-          } else {
+            } else {                             // ragged or unaligned chunk: element by element
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int n = nb + j;
-              if (n < N) {
-                float x = v[j] + (bias ? __ldg(bias + n) : 0.f);
-                if (sigm) x = 1.f / (1.f + __expf(-x));
-                if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
-                x *= alpha;
-                if (crow) x = fmaf(beta, __ldg(crow + n), x);
-                drow[n] = x;
+              for (int e = 0; e < 2; ++e) {
+                const int m = mq + 16 * h + 8 * e;
+                if (m >= M) continue;
+                const float* zrow = dsig ? dsig + (long long)((m / dsig_div) % dsig_rows) * ld_dsig : nullptr;
+                const float* crow = cin ? cin + (long long)m * ld_cin : nullptr;
+                float* drow = D + (long long)m * ldd;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                  for (int i = 0; i < 2; ++i) {
+                    const int n = nb + 8 * j + i;
+                    if (n < N) {
+                      float x = v[4 * j + 2 * e + i] + (bias ? __ldg(bias + n) : 0.f);
+                      if (sigm) x = 1.f / (1.f + __expf(-x));
+                      if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
+                      x *= alpha;
+                      if (crow) x = fmaf(beta, __ldg(crow + n), x);
+                      drow[n] = x;
+                    }
+                  }
               }
             }
           }
@@ -815,6 +891,8 @@ gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, cons
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dep_wait();
+  grid_dep_launch();
 
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(X3_REGS_LOW));
@@ -1135,6 +1213,22 @@ int gemm_tf32_workspace_flags() { return num_sms() / 2; }
 
 namespace {
 
+// Launch with the programmatic stream-serialisation attribute (see grid_dep_wait above).
+template <class... KArgs, class... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, int smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3((unsigned)block, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 // Tensor maps and kernel parameters of one problem for a given tile width (two_cta: 256 x bn tiles of a CTA pair).
 bool setup_problem(const GemmArgs& g, bool two_cta, int bn, int* err_flag, CUtensorMap* maps, Tf32Params& p) {
   const int b_rows = two_cta ? bn / 2 : bn;      // B rows staged per CTA
@@ -1189,44 +1283,65 @@ inline bool suits_pair_kernel(const GemmArgs& g) { return g.M > BM && g.N >= 128
 
 }  // namespace
 
+namespace {
+// K slices for the tiles left over after the whole waves of a problem with `tiles` tiles of `total_kb` k-blocks on
+// `pairs` CTA pairs (1 = whole tiles).  A sliced tile pays for a store and a re-read of its partial accumulators
+// and for the wait between them, about as much as 25 to 30 k-blocks of main loop (measured: a 25-k-block tile is
+// faster whole even when its wave is nearly empty, a 63-k-block tile gains from 2 slices on), so a tile is cut only
+// if that saves more than this.
+int choose_slices(int tiles, int total_kb, int pairs) {
+  int rem = tiles % pairs;
+  if (tiles < pairs) rem = tiles;
+  if (rem == 0) return 1;
+  int sl = pairs / rem;
+  if (sl > kMaxSlices) sl = kMaxSlices;
+  if (sl > total_kb) sl = total_kb;
+  while (sl >= 2 && total_kb / sl < 4) --sl;
+  if (sl < 2) return 1;
+  return (double)total_kb * (1.0 - 1.0 / sl) >= 30.0 ? sl : 1;
+}
+}  // namespace
+
 int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st) {
   set_kernel_attributes();
   const bool two_cta = g.two_cta >= 0 ? g.two_cta != 0 : suits_pair_kernel(g);
-  const bool stream_k = two_cta && sk_ws && sk_flags;
-  const int bn = two_cta ? choose_bn2(g.M, g.N, stream_k) : choose_bn(g.M, g.N);
+  bool stream_k = two_cta && sk_ws && sk_flags;
+  const int pairs = num_sms() / 2;
+  const int total_kb_all = (g.K1 + BK - 1) / BK + (g.A2 ? (g.K2 + BK - 1) / BK : 0);
+  int bn = two_cta ? choose_bn2(g.M, g.N, stream_k) : choose_bn(g.M, g.N);
+  if (stream_k) {
+    // the width chosen for an even split of the work only stands if the left-over tiles will in fact be cut
+    const int tiles = ((g.M + 2 * BM - 1) / (2 * BM)) * ((g.N + bn - 1) / bn);
+    if (choose_slices(tiles, total_kb_all, pairs) < 2) { stream_k = false; bn = choose_bn2(g.M, g.N, false); }
+  }
   if (two_cta) {
     GroupMaps gm;                              // (host copies; passed to the kernel by value)
     GroupParams gp;
     gp.n_prob = 1;
     Tf32Params& p = gp.pr[0];
     if (!setup_problem(g, true, bn, err_flag, gm.m[0], p)) return -1;
-    const int pairs = num_sms() / 2;
     const int total_kb = p.kblocks[0] + p.kblocks[1];
     p.sk_ws = sk_ws; p.sk_flags = sk_flags;
     p.P = p.tiles < pairs ? p.tiles : pairs;
     p.waves = p.tiles / p.P;
     p.rem = p.tiles - p.waves * p.P;
     int launch_pairs = p.P;
-    if (stream_k && p.tiles < pairs) {
-      // fewer tiles than pairs: there is no full wave; every tile is cut along K over pairs / tiles pairs
-      p.P = pairs; p.waves = 0; p.rem = p.tiles;
+    if (stream_k) {
+      const int sl = choose_slices(p.tiles, total_kb, pairs);
+      if (sl >= 2) {
+        if (p.tiles < pairs) { p.P = pairs; p.waves = 0; p.rem = p.tiles; }   // no full wave: every tile is cut
+        p.slices = sl;
+        if (p.waves == 0) launch_pairs = p.rem * p.slices;
+      }
     }
-    if (stream_k && p.rem > 0) {
-      int sl = pairs / p.rem;
-      if (sl > kMaxSlices) sl = kMaxSlices;
-      if (sl > total_kb) sl = total_kb;
-      // a slice costs a store and a re-read of the tile on top of its MMAs: not worth it for short K
-      if (sl >= 2 && total_kb / sl >= 4) p.slices = sl;
-    }
-    if (p.waves == 0) launch_pairs = p.slices >= 2 ? p.rem * p.slices : p.rem;
     for (int q = 0; q <= MAX_PAIRS_LAUNCH; ++q) gp.rstart[0][q] = (unsigned short)(q < p.rem ? q : p.rem);
-    gemm_tf32_2cta_kernel<kStages2><<<2 * launch_pairs, 320, kSmemBytes2, st>>>(gm, gp);
+    launch_pdl(gemm_tf32_2cta_kernel<kStages2>, 2 * launch_pairs, 320, kSmemBytes2, st, gm, gp);
   } else {
     CUtensorMap maps[4];
     Tf32Params p;
     if (!setup_problem(g, false, bn, err_flag, maps, p)) return -1;
     const int grid = p.tiles < num_sms() ? p.tiles : num_sms();
-    gemm_tf32_kernel<kStages><<<grid, 320, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+    launch_pdl(gemm_tf32_kernel<kStages>, grid, 320, kSmemBytes, st, maps[0], maps[1], maps[2], maps[3], p);
   }
   return 1;
 }
@@ -1308,7 +1423,7 @@ int launch_gemm_tf32_group(const GemmArgs* gs, int n, int* err_flag, cudaStream_
     for (int q = 0; q < P; ++q) { gp.rstart[k][q] = (unsigned short)run; run += cnt[q] - waves; load[q] += cnt[q] * cost; }
     for (int q = P; q <= MAX_PAIRS_LAUNCH; ++q) gp.rstart[k][q] = (unsigned short)run;
   }
-  gemm_tf32_2cta_kernel<kStages2><<<2 * P, 320, kSmemBytes2, st>>>(gm, gp);
+  launch_pdl(gemm_tf32_2cta_kernel<kStages2>, 2 * P, 320, kSmemBytes2, st, gm, gp);
   return 1;
 }
 
@@ -1389,7 +1504,7 @@ int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   p.waves = p.tiles / p.P;
   p.rem = p.tiles - p.waves * p.P;
   p.slices = 1;
-  gemm_tf32x3_kernel<X3_STAGES><<<2 * p.P, X3_THREADS, kSmemBytes3, st>>>(maps, p, xp);
+  launch_pdl(gemm_tf32x3_kernel<X3_STAGES>, 2 * p.P, X3_THREADS, kSmemBytes3, st, maps, p, xp);
   return 1;
 }
 

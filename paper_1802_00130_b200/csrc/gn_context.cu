@@ -27,7 +27,7 @@ struct gn_ctx {
   // joined before the product (or row batch) ends
   cudaStream_t st2 = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
-  bool side_enabled = true, side_open = false;
+  bool side_enabled = true, side_open = false, side_region = false;
   int64_t n = 0;
   std::vector<int64_t> w_off, b_off;  // [m], m = 1..L (entry 0 unused)
   int64_t batch_rows = 32768;
@@ -189,7 +189,14 @@ void side_join(gn_ctx* c) {
   cudaStreamWaitEvent(c->st, c->ev_join, 0);
   c->side_open = false;
 }
-struct SideJoin { gn_ctx* c; ~SideJoin() { side_join(c); } };   // joins on every way out of a launch sequence
+// A launch sequence that uses the side stream: inside it, every kernel that works in the side stream's scratch
+// buffers (column sums, the n_L-row weight block) goes to the side stream, so those buffers have one user at a
+// time; the join happens on every way out.
+struct SideJoin {
+  gn_ctx* c;
+  explicit SideJoin(gn_ctx* ctx) : c(ctx) { c->side_region = true; }
+  ~SideJoin() { side_join(c); c->side_region = false; }
+};
 
 // Before a workspace that side-stream kernels may still read is released.
 void quiesce(gn_ctx* c) {
@@ -373,6 +380,8 @@ void run_gemm(gn_ctx* c, const GemmArgs& g, cudaStream_t st = nullptr) {
       if (dev_alloc(c, &c->thin_scratch, need) != GN_OK) { c->sticky = GN_ENOMEM; return; }
       c->thin_cap = need;
     }
+    // the n_L-row weight block streams its operands once and shares nothing with the layer's other contraction
+    if (thin == THIN_M && c->side_region && !st) st = side_fork(c);
     run_gemm_kind(c, g, 2, st);
     return;
   }
@@ -526,13 +535,6 @@ gn_status layer_backward(gn_ctx* c, int m, const float* ds_w, int64_t w_rows, co
   int n = 0;
   gs[n++] = weight_block_args(c, m, ds_w, Zprev, w_rows, alpha, cin, beta, out, w_padded);
   if (m > 1) gs[n++] = backward_data_args(c, m, ds_d, d_rows, Zprev, z_rows, dst, ds_w == ds_d && w_rows == d_rows);
-  if (n == 2 && gemm_thin_kind(gs[0]) == THIN_M && c->side_enabled && c->st2) {
-    // the n_L-row weight block streams the same rows as the activation gradient but shares nothing else with it
-    GN_TRY(bias_block(c, m, ds_w, w_rows, alpha, cin, beta, out));
-    run_gemm(c, gs[0], side_fork(c));
-    run_gemm(c, gs[1]);
-    return GN_OK;
-  }
   GN_TRY(bias_block(c, m, ds_w, w_rows, alpha, cin, beta, out));
   run_gemm_group(c, gs, n);
   return GN_OK;
@@ -540,7 +542,7 @@ gn_status layer_backward(gn_ctx* c, int m, const float* ds_w, int64_t w_rows, co
 
 // out = coef v + (1/|S|) J^T (2 J v) over the stored subsample (Eq. sampled-Gauss).
 gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
-  SideJoin side_guard{c};
+  SideJoin side_guard(c);
   const int L = c->L;
   const int64_t nS = c->nS;
   for (int m = 1; m <= L; ++m) {
@@ -571,7 +573,7 @@ gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
 // pulled back to layer k only; the L streams are stacked along rows, stream j occupying rows
 // [(j-1)|S|, j|S|) of every buffer at or above layer j, so each layer runs one stacked GEMM.
 gn_status product_blockdiag(gn_ctx* c, const float* v, float* out, float coef) {
-  SideJoin side_guard{c};
+  SideJoin side_guard(c);
   const int L = c->L;
   const int64_t nS = c->nS;
   for (int k = 1; k <= L; ++k) {
@@ -643,7 +645,7 @@ gn_status ensure_factors(gn_ctx* c) {
 }
 
 gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float coef) {
-  SideJoin side_guard{c};
+  SideJoin side_guard(c);
   GN_TRY(ensure_factors(c));
   const int L = c->L, nL = c->w[L];
   const int64_t nS = c->nS;
@@ -686,7 +688,6 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
 // Q_a[:, T_b] = D[:, :, T_b]^T 2 D[:, :, T_b] U_a[:, T_b]; then out_W[T_a, :] = Z_{m-1}[:, T_a]^T Q_a / |S|.
 // At the output layer D = I, so Q_a = 2 U_a.
 gn_status product_split(gn_ctx* c, const float* v, float* out, float coef) {
-  SideJoin side_guard{c};
   const int L = c->L, nL = c->w[L];
   const int64_t nS = c->nS;
   if (L >= 2) {
@@ -798,7 +799,7 @@ gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
         GN_CUDA(c, cudaMemsetAsync(c->partial + b * per_batch + used, 0, (per_batch - used) * sizeof(double), c->st));
     }
     if (d_grad) {
-      SideJoin side_guard{c};     // the next batch overwrites what the side stream reads
+      SideJoin side_guard(c);     // the next batch overwrites what the side stream reads
       for (int m = L; m >= 1; --m) {
         const float* Zprev = m == 1 ? X0 : c->Zb[m - 1];
         const float* cin0 = b == 0 ? c->theta : d_grad;
