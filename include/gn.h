@@ -332,8 +332,11 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
  * tiles only; cannot be switched back on); option 2: failure injection on the host: the value-th device allocation
  * the context asks for from now on is refused as if the device were out of memory (0 = off); nothing on the
  * device is touched by it; option 3: the bias column sums and the n_L-row weight block of a layer on a side stream
- * next to the layer's large contractions (value 0 = everything on the context's stream).  Results do not depend on
- * options 0 and 3 (tiles and sums are computed identically); GN_EINVAL for an unknown option.
+ * next to the layer's large contractions (value 0 = everything on the context's stream); option 4: consecutive
+ * layers of a pass as one launch whose tiles wait for the tiles they read (value 0 = one launch per layer, 1 = the
+ * stored forward pass, the default, 2 = also the forward R pass of a product).  Option 5 (GN_FP32_ACCURATE contexts): the error-compensated kernel also writes the hi / lo parts
+ * of a result that a later contraction takes as an operand (value 0 = a separate pass splits it).  Results do not
+ * depend on options 0, 3, 4 and 5 (tiles, sums and parts are computed identically); GN_EINVAL for an unknown option.
  */
 gn_status gn_debug_option(gn_ctx* ctx, int option, int value);
 

@@ -47,6 +47,9 @@ struct Tf32Params {
   float alpha;
   const float* cin; long long ld_cin; float beta;
   int vec_epi;          // D, bias, dsig, cin all 16-byte aligned with leading dimensions % 4 == 0
+  // error-compensated kernel only: also write the two-term TF32 split of every stored value (hi = value rounded to
+  // TF32, lo = value - hi rounded to TF32) to these matrices, for the contraction that takes D as an operand next
+  float* Dhi; float* Dlo; long long ld_parts;
   int bn;               // tile width: multiple of 32, 32 <= bn <= 256
   int tiles_n, tiles;
   int* err;
@@ -62,12 +65,24 @@ struct Tf32Params {
 // its tiles of the problem's whole waves (q, q + P, ...) and then tiles rstart[g][q] .. rstart[g][q + 1] - 1 of the
 // tiles left over after those waves; the host deals the left-over tiles so that the pairs' total loads come out even
 // (longest tiles first), which lets the short tiles of one problem fill the partial last wave of another.
-constexpr int MAX_GROUP = 3;
+constexpr int MAX_GROUP = 5;
 constexpr int MAX_PAIRS_LAUNCH = 80;        // >= SMs / 2
 struct GroupParams {
   int n_prob;
   Tf32Params pr[MAX_GROUP];
   unsigned short rstart[MAX_GROUP][MAX_PAIRS_LAUNCH + 1];
+  // Dependent problems in one launch (a chain of layers): problem g may read, as an operand, what problem
+  // dep_prob[g] (earlier in the list) writes.  dep_all[g] == 0: a tile of g needs the producer's tiles of the
+  // same 256-row panel (its A rows are the producer's output rows); dep_all[g] == 1: it needs all of them (its
+  // K runs over the producer's rows).  The epilogue warps of a producer count finished tiles per panel
+  // (signal bit 0) and in total (bit 1) in `done`; the TMA warps of a consumer wait, bounded, for the count.
+  // Every pair works through the problems in list order and all pairs are resident, so a wait is always for
+  // work that is running or about to run on another pair.
+  int dep_prob[MAX_GROUP];
+  int dep_all[MAX_GROUP];
+  int signal[MAX_GROUP];
+  int* done;                 // [n_prob][done_stride]: entry i < done_stride - 1 counts panel i, the last entry all tiles
+  int done_stride;
 };
 struct GroupMaps { CUtensorMap m[MAX_GROUP][4]; };   // per problem: A0, B0, A1, B1
 
@@ -86,6 +101,12 @@ __device__ __forceinline__ unsigned long long globaltimer() {
 // after this one do the same.  Without the attribute both are no-ops.
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+__device__ __forceinline__ float round_tf32(float x) {
+  uint32_t u;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+  return __uint_as_float(u);
+}
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
@@ -188,6 +209,12 @@ __device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -563,6 +590,24 @@ gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constan
       const int t = w.tile, kb0 = w.kb0, kb1 = w.kb1;
       const int m0 = (t / p.tiles_n) * (2 * BM) + (int)rank * BM;
       const int n0 = (t % p.tiles_n) * bn + (int)rank * hb;
+      if (gp.dep_prob[w.prob] >= 0) {
+        // an operand of this tile is written by an earlier problem of this launch: wait until its tiles are stored
+        const int d = gp.dep_prob[w.prob];
+        const int* ctr = gp.done + (long long)d * gp.done_stride + (gp.dep_all[w.prob] ? gp.done_stride - 1 : t / p.tiles_n);
+        const int want = 16 * (gp.dep_all[w.prob] ? gp.pr[d].tiles : gp.pr[d].tiles_n);
+        int good = 1;
+        if (lane == 0) {
+          const unsigned long long t0 = globaltimer();
+          while (ld_acquire_gpu(ctr) < want) {
+            if (*abort_flag || globaltimer() - t0 > WAIT_LIMIT_NS) { atomicCAS(err, 0, 6); *abort_flag = 1; good = 0; break; }
+            __nanosleep(100);
+          }
+        }
+        good = __shfl_sync(0xffffffffu, good, 0);
+        if (!good) { ok = false; break; }
+        asm volatile("fence.proxy.async.global;" ::: "memory");   // the stores were generic, the loads below are TMA's
+        __syncwarp();
+      }
       for (int kb = kb0; kb < kb1; ++kb, ++it) {
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1;
@@ -816,6 +861,17 @@ gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constan
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
       }
+      if (gp.signal[w.prob]) {
+        // a later problem of this launch reads this tile: publish this warp's stores, then count the warp in
+        __threadfence();
+        asm volatile("fence.proxy.async.global;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          int* base = gp.done + (long long)w.prob * gp.done_stride;
+          if (gp.signal[w.prob] & 1) atomicAdd(base + t / p.tiles_n, 1);
+          if (gp.signal[w.prob] & 2) atomicAdd(base + gp.done_stride - 1, 1);
+        }
+      }
     }
   }
   tc_fence_before();
@@ -1043,6 +1099,13 @@ gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, cons
               if (crow) x[e] = fmaf(p.beta, cv[e], x[e]);
             }
             reinterpret_cast<float4*>(drow + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
+            if (p.Dhi) {
+              float h[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) { h[e] = round_tf32(x[e]); x[e] = round_tf32(x[e] - h[e]); }
+              reinterpret_cast<float4*>(p.Dhi + (long long)m * p.ld_parts + nb)[q] = make_float4(h[0], h[1], h[2], h[3]);
+              reinterpret_cast<float4*>(p.Dlo + (long long)m * p.ld_parts + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
+            }
             // the running sums leave few registers: keep the loads of at most two steps in flight
             if (q & 1) asm volatile("" ::: "memory");
           }
@@ -1057,6 +1120,11 @@ gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, cons
               x *= p.alpha;
               if (crow) x = fmaf(p.beta, __ldg(crow + n), x);
               drow[n] = x;
+              if (p.Dhi) {
+                const float h = round_tf32(x);
+                p.Dhi[(long long)m * p.ld_parts + n] = h;
+                p.Dlo[(long long)m * p.ld_parts + n] = round_tf32(x - h);
+              }
             }
           }
         }
@@ -1316,7 +1384,8 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
   }
   if (two_cta) {
     GroupMaps gm;                              // (host copies; passed to the kernel by value)
-    GroupParams gp;
+    GroupParams gp = {};                       // (no dependencies, no signals)
+    for (int k = 0; k < MAX_GROUP; ++k) gp.dep_prob[k] = -1;
     gp.n_prob = 1;
     Tf32Params& p = gp.pr[0];
     if (!setup_problem(g, true, bn, err_flag, gm.m[0], p)) return -1;
@@ -1353,14 +1422,67 @@ bool gemm_tf32_group_eligible(const GemmArgs* gs, int n) {
   return true;
 }
 
-// Several independent problems in one launch of the CTA-pair kernel.  The pairs' work is balanced on the host:
-// problems are taken longest tile first; each gets as many whole waves (tiles q, q + P, ... for every pair q)
-// as fit under the level that evens out the loads so far, and its left-over tiles go to the least loaded pairs.
-int launch_gemm_tf32_group(const GemmArgs* gs, int n, int* err_flag, cudaStream_t st) {
+namespace {
+
+// Tiles of problem slot k of a group (cost `cost` each) dealt to the P pairs on top of the loads they carry
+// already: as many whole waves (tiles q, q + P, ... for every pair q) as every pair takes anyway, the rest as
+// contiguous runs of the left-over tiles, so that the loads come out as even as whole tiles allow.
+void deal_tiles(GroupParams& gp, int k, double cost, int P, double* load) {
+  Tf32Params& p = gp.pr[k];
+  p.P = P;
+  int cnt[MAX_PAIRS_LAUNCH];
+  // lowest level L with sum_q floor((L - load_q) / cost) >= tiles, by bisection on L
+  double lo = 0.0, hi = 0.0;
+  for (int q = 0; q < P; ++q) if (load[q] > hi) hi = load[q];
+  hi += cost * (p.tiles / P + 2);
+  for (int iter = 0; iter < 60; ++iter) {
+    const double mid = 0.5 * (lo + hi);
+    long long have = 0;
+    for (int q = 0; q < P; ++q) if (mid > load[q]) have += (long long)((mid - load[q]) / cost);
+    if (have >= p.tiles) hi = mid; else lo = mid;
+  }
+  long long have = 0;
+  for (int q = 0; q < P; ++q) { cnt[q] = hi > load[q] ? (int)((hi - load[q]) / cost) : 0; have += cnt[q]; }
+  // more than needed (several pairs cross a multiple of `cost` at the same level): take back from the fullest
+  while (have > p.tiles) {
+    int worst = -1;
+    for (int q = 0; q < P; ++q)
+      if (cnt[q] > 0 && (worst < 0 || load[q] + cnt[q] * cost > load[worst] + cnt[worst] * cost)) worst = q;
+    --cnt[worst]; --have;
+  }
+  while (have < p.tiles) {                    // (rounding in the bisection)
+    int best = 0;
+    for (int q = 1; q < P; ++q)
+      if (load[q] + cnt[q] * cost < load[best] + cnt[best] * cost) best = q;
+    ++cnt[best]; ++have;
+  }
+  int waves = cnt[0];
+  for (int q = 1; q < P; ++q) if (cnt[q] < waves) waves = cnt[q];
+  p.waves = waves;
+  p.rem = p.tiles - waves * P;
+  int run = 0;
+  for (int q = 0; q < P; ++q) { gp.rstart[k][q] = (unsigned short)run; run += cnt[q] - waves; load[q] += cnt[q] * cost; }
+  for (int q = P; q <= MAX_PAIRS_LAUNCH; ++q) gp.rstart[k][q] = (unsigned short)run;
+}
+
+// time of one tile in k-blocks of a 256-wide tile: operand bytes per k-block (the feed bounds the main loop) plus a fixed part
+double tile_cost(const Tf32Params& p) { return (p.kblocks[0] + p.kblocks[1]) * (256.0 + p.bn) / 512.0 + 8.0; }
+
+}  // namespace
+
+// Several problems in one launch of the CTA-pair kernel.
+//   Independent problems (dep_prob == nullptr): taken longest tile first, the pairs' loads evened out on the host,
+//   so the short tiles of one problem fill the partial last wave of another.
+//   A chain (dep_prob[i] = index of the earlier problem whose output problem i reads, or -1; dep_all[i] != 0 if it
+//   needs all of that output rather than the 256-row panel of its own tile): kept in the given order, every pair
+//   works through the problems one after the other, and the head of a problem overlaps the tail of the one before.
+//   `done` is a zeroed-by-this-call array of n * done_stride ints, done_stride > the number of 256-row panels.
+int launch_gemm_tf32_group(const GemmArgs* gs, int n, const int* dep_prob, const int* dep_all, int* done,
+                           int done_stride, int* err_flag, cudaStream_t st) {
   if (!gemm_tf32_group_eligible(gs, n)) return -1;
   set_kernel_attributes();
   GroupMaps gm;
-  GroupParams gp;
+  GroupParams gp = {};
   const int pairs = num_sms() / 2;
   struct Item { int src; double cost; };
   Item order[MAX_GROUP];
@@ -1371,58 +1493,40 @@ int launch_gemm_tf32_group(const GemmArgs* gs, int n, int* err_flag, cudaStream_
     const int bn = choose_bn2(gs[i].M, gs[i].N, true);
     if (!setup_problem(gs[i], true, bn, err_flag, tmaps[i], tmp[i])) return -1;
     if (tmp[i].tiles > 60000) return -1;       // (left-over tile indices are 16-bit)
-    // time of one tile: operand bytes per k-block (the feed bounds the main loop) plus a fixed part
     order[i].src = i;
-    order[i].cost = (tmp[i].kblocks[0] + tmp[i].kblocks[1]) * (256.0 + bn) / 512.0 + 8.0;
+    order[i].cost = tile_cost(tmp[i]);
     total_tiles += tmp[i].tiles;
   }
-  for (int i = 1; i < n; ++i)                   // insertion sort, longest tile first (stable)
-    for (int j = i; j > 0 && order[j].cost > order[j - 1].cost; --j) { Item t = order[j]; order[j] = order[j - 1]; order[j - 1] = t; }
+  const bool chain = dep_prob != nullptr;
+  if (chain) {
+    if (!done) return -1;
+    for (int i = 0; i < n; ++i) {
+      if (dep_prob[i] >= i) return -1;
+      if (dep_prob[i] >= 0 && !dep_all[i] && gs[dep_prob[i]].M != gs[i].M) return -1;   // panels must coincide
+      if ((gs[i].M + 2 * BM - 1) / (2 * BM) + 1 > done_stride) return -1;
+    }
+  } else {
+    for (int i = 1; i < n; ++i)                 // insertion sort, longest tile first (stable)
+      for (int j = i; j > 0 && order[j].cost > order[j - 1].cost; --j) { Item t = order[j]; order[j] = order[j - 1]; order[j - 1] = t; }
+  }
   const int P = total_tiles < pairs ? (int)total_tiles : pairs;
   double load[MAX_PAIRS_LAUNCH];
   for (int q = 0; q < P; ++q) load[q] = 0.0;
   gp.n_prob = n;
+  gp.done = done; gp.done_stride = done_stride;
+  for (int k = 0; k < MAX_GROUP; ++k) { gp.dep_prob[k] = -1; gp.dep_all[k] = 0; gp.signal[k] = 0; }
   for (int k = 0; k < n; ++k) {
     const int i = order[k].src;
-    const double cost = order[k].cost;
-    Tf32Params& p = gp.pr[k];
-    p = tmp[i];
+    gp.pr[k] = tmp[i];
     for (int j = 0; j < 4; ++j) gm.m[k][j] = tmaps[i][j];
-    p.P = P;
-    // counts per pair: lowest level L with sum_q floor((L - load_q) / cost) >= tiles, by bisection on L
-    int cnt[MAX_PAIRS_LAUNCH];
-    double lo = 0.0, hi = 0.0;
-    for (int q = 0; q < P; ++q) if (load[q] > hi) hi = load[q];
-    hi += cost * (p.tiles / P + 2);
-    for (int iter = 0; iter < 60; ++iter) {
-      const double mid = 0.5 * (lo + hi);
-      long long have = 0;
-      for (int q = 0; q < P; ++q) if (mid > load[q]) have += (long long)((mid - load[q]) / cost);
-      if (have >= p.tiles) hi = mid; else lo = mid;
+    deal_tiles(gp, k, order[k].cost, P, load);
+    if (chain && dep_prob[i] >= 0) {            // (a chain keeps its order: slot == index)
+      gp.dep_prob[k] = dep_prob[i];
+      gp.dep_all[k] = dep_all[i] ? 1 : 0;
+      gp.signal[dep_prob[i]] |= dep_all[i] ? 2 : 1;
     }
-    long long have = 0;
-    for (int q = 0; q < P; ++q) { cnt[q] = hi > load[q] ? (int)((hi - load[q]) / cost) : 0; have += cnt[q]; }
-    // more than needed (several pairs cross a multiple of `cost` at the same level): take back from the fullest
-    while (have > p.tiles) {
-      int worst = -1;
-      for (int q = 0; q < P; ++q)
-        if (cnt[q] > 0 && (worst < 0 || load[q] + cnt[q] * cost > load[worst] + cnt[worst] * cost)) worst = q;
-      --cnt[worst]; --have;
-    }
-    while (have < p.tiles) {                    // (rounding in the bisection)
-      int best = 0;
-      for (int q = 1; q < P; ++q)
-        if (load[q] + cnt[q] * cost < load[best] + cnt[best] * cost) best = q;
-      ++cnt[best]; ++have;
-    }
-    int waves = cnt[0];
-    for (int q = 1; q < P; ++q) if (cnt[q] < waves) waves = cnt[q];
-    p.waves = waves;
-    p.rem = p.tiles - waves * P;
-    int run = 0;
-    for (int q = 0; q < P; ++q) { gp.rstart[k][q] = (unsigned short)run; run += cnt[q] - waves; load[q] += cnt[q] * cost; }
-    for (int q = P; q <= MAX_PAIRS_LAUNCH; ++q) gp.rstart[k][q] = (unsigned short)run;
   }
+  if (chain && cudaMemsetAsync(done, 0, sizeof(int) * (size_t)n * done_stride, st) != cudaSuccess) return -1;
   launch_pdl(gemm_tf32_2cta_kernel<kStages2>, 2 * P, 320, kSmemBytes2, st, gm, gp);
   return 1;
 }
@@ -1495,6 +1599,8 @@ int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st) {
   p.vec_epi = aligned16(g.D) && (g.ldd % 4 == 0) && (!g.bias || aligned16(g.bias)) &&
               (!g.dsig || (aligned16(g.dsig) && g.ld_dsig % 4 == 0)) &&
               (!g.cin || (aligned16(g.cin) && g.ld_cin % 4 == 0));
+  p.Dhi = g.Dhi; p.Dlo = g.Dlo; p.ld_parts = g.ld_parts;
+  if (p.Dhi && !(aligned16(g.Dhi) && aligned16(g.Dlo) && g.ld_parts % 4 == 0)) return -1;
   p.bn = bn;
   p.tiles_n = (g.N + bn - 1) / bn;
   p.err = err_flag;

@@ -63,6 +63,11 @@ struct gn_ctx {
   float* sk_ws = nullptr; int* sk_flags = nullptr;   // stream-K workspace of the tensor-core kernel
   bool sk_enabled = true;
   bool group_enabled = true;   // independent contractions of a layer as one launch (TF32 mode)
+  // consecutive layers of a pass as one launch with tile-level dependencies (TF32 mode): 0 never, 1 the stored forward
+  // pass (where it measured 8 % faster), 2 also the forward R pass of a product (where cutting left-over tiles along K,
+  // which a chained launch does not do, measured as fast or faster)
+  int chain_level = 1;
+  int* chain_ctr = nullptr; int64_t chain_ctr_cap = 0;   // finished-tile counters of such a launch
   // FP32-accurate mode on the tensor cores (3 x TF32): hi / lo parts of the operands
   int acc_method = 0;        // 0 choose (tensor cores where the shape allows), 1 FP32 FMA only, 2 as 0
   bool x3_usable = true;     // cleared if the error-compensated kernel could not be launched
@@ -77,6 +82,13 @@ struct gn_ctx {
     uint64_t seq = 0;        // contraction (gemm_seq) that wrote these parts
   };
   SplitSlot split_slot[4];
+  // hi / lo parts written by the epilogue of the error-compensated kernel for a result that a later contraction of
+  // the SAME launch sequence takes as an operand (R z^m, delta s^m, and their row-batch twins): keyed by the result's
+  // address, valid only while parts_epoch stands (every launch sequence that may rewrite those buffers bumps it)
+  struct PartsEntry { const float* src = nullptr; int64_t rows = 0; int cols = 0; int64_t ld = 0; uint64_t epoch = 0; SplitBuf buf; };
+  std::vector<PartsEntry> parts;
+  uint64_t parts_epoch = 1;
+  bool parts_enabled = false;  // (measured 7 % slower than a separate splitting pass: off unless asked for)
   uint64_t gemm_seq = 0;     // counts contractions (run_gemm calls)
   double* partial = nullptr; int64_t partial_cap = 0;
   double* dscal = nullptr;   // device: [0] loss, [1] theta^T theta, [2] cg sum rho, [3] cg active
@@ -283,6 +295,13 @@ bool split_buf_reserve(gn_ctx* c, gn_ctx::SplitBuf& b, int64_t need) {
   return true;
 }
 
+// The results whose parts the epilogue writes live in the subsample and row-batch workspaces: when those move,
+// the parts kept for their old addresses go.
+void drop_parts(gn_ctx* c) {
+  for (auto& e : c->parts) { dev_free(c, e.buf.hi); dev_free(c, e.buf.lo); }
+  c->parts.clear();
+}
+
 // hi / lo parts of the stored matrix [rows][cols] (leading dimension ld) that serves as an operand.  Matrices
 // inside theta or inside the stored activations Z_m are split once per set_theta / set_subsample; anything
 // else goes through the slot of its operand role (0 = A1, 1 = B1, 2 = A2, 3 = B2) and is split again on every
@@ -324,6 +343,11 @@ bool split_operand(gn_ctx* c, const float* src, int64_t rows, int cols, int64_t 
     *hi = e->buf.hi; *lo = e->buf.lo;
     return true;
   }
+  for (auto& e : c->parts)
+    if (e.src == src && e.epoch == c->parts_epoch && e.rows == rows && e.cols == cols && e.ld == ld && e.buf.hi) {
+      *hi = e.buf.hi; *lo = e.buf.lo;      // written by the epilogue that produced this operand
+      return true;
+    }
   if (rows * ldo > kMaxTransientSplitFloats) return false;
   gn_ctx::SplitSlot& sl = c->split_slot[role];
   const bool same = reuse && sl.seq != 0 && sl.seq + 1 == c->gemm_seq && sl.src == src && sl.rows == rows &&
@@ -358,7 +382,23 @@ bool run_gemm_x3(gn_ctx* c, const GemmArgs& g) {
     h.B2 = hi; h.B2lo = lo; h.ldb2 = ldo;
   }
   h.mn_padded = true;     // the parts live in context allocations, which carry slack after their last row
+  gn_ctx::PartsEntry* pe = nullptr;
+  if (g.emit_parts && c->parts_enabled && (int64_t)g.M * round4(g.N) <= kMaxTransientSplitFloats) {
+    // the result is an operand later in this launch sequence: have the epilogue write its hi / lo parts as well
+    for (auto& e : c->parts)
+      if (e.src == g.D) { pe = &e; break; }
+    if (!pe && c->parts.size() < 1024) { c->parts.emplace_back(); pe = &c->parts.back(); pe->src = g.D; }
+    if (pe) {
+      pe->epoch = 0;
+      if (split_buf_reserve(c, pe->buf, (int64_t)g.M * round4(g.N))) {
+        h.Dhi = pe->buf.hi; h.Dlo = pe->buf.lo; h.ld_parts = round4(g.N);
+      } else {
+        pe = nullptr;
+      }
+    }
+  }
   run_gemm_kind(c, h, 3);
+  if (pe && c->x3_usable) { pe->rows = g.M; pe->cols = g.N; pe->ld = g.ldd; pe->epoch = c->parts_epoch; }
   return true;
 }
 
@@ -393,7 +433,7 @@ void run_gemm(gn_ctx* c, const GemmArgs& g, cudaStream_t st = nullptr) {
 // kernel go out in launches of up to three problems with a common work list (the tiles of one fill the partial
 // last wave of another); everything else runs one after the other, in the order given.
 void run_gemm_group(gn_ctx* c, const GemmArgs* gs, int n) {
-  constexpr int kMax = 3;
+  constexpr int kMax = 3;      // (more than three independent problems per launch gained nothing measurable)
   bool taken[16] = {false};
   if (n >= 2 && n <= 16 && c->prec == GN_TF32 && c->group_enabled) {
     GemmArgs pick[kMax];
@@ -416,7 +456,7 @@ void run_gemm_group(gn_ctx* c, const GemmArgs* gs, int n) {
             cudaEventRecord(e->a, c->st);
           }
         }
-        const int r = launch_gemm_tf32_group(pick, np, c->err_flag + 1, c->st);
+        const int r = launch_gemm_tf32_group(pick, np, nullptr, nullptr, nullptr, 0, c->err_flag + 1, c->st);
         if (r < 0) { c->sticky = GN_ECUDA; c->err = "cuTensorMapEncodeTiled failed"; }
         else c->launches += r;
         if (e) cudaEventRecord(e->b, c->st);
@@ -437,6 +477,64 @@ void run_gemm_group(gn_ctx* c, const GemmArgs* gs, int n) {
 
 // (the new buffer is obtained before the old one is let go: the solver and the dot products use c->partial
 // without asking for it again, so a refused allocation must leave the old buffer in place)
+// The layers of a pass, each reading what the one before it writes (dep[i] = index of that earlier problem, -1 for
+// none; dep_all[i]: it reads all of that output, not just the rows of its own tile).  In TF32 mode a run of
+// consecutive problems that suit the CTA-pair kernel goes out as ONE launch in which a tile starts as soon as the
+// tiles it reads are stored, so a layer's first tiles run beside the previous layer's last ones; everything else
+// runs one after the other, in the order given (which is a valid order by construction).
+void run_gemm_chain(gn_ctx* c, const GemmArgs* gs, const int* dep, const int* dep_all, int n, int level = 1) {
+  int i = 0;
+  while (i < n) {
+    int j = i;
+    if (c->prec == GN_TF32 && c->chain_level >= level) {
+      while (j < n && j - i < kGemmGroupMax && gemm_thin_kind(gs[j]) == THIN_NONE && gemm_tf32_group_eligible(&gs[j], 1)) ++j;
+    }
+    if (j - i >= 2) {
+      const int cnt = j - i;
+      int64_t panels = 0;
+      for (int k = i; k < j; ++k) panels = std::max<int64_t>(panels, (gs[k].M + 255) / 256);
+      const int stride = (int)panels + 1;
+      if (!c->chain_ctr || (int64_t)kGemmGroupMax * stride > c->chain_ctr_cap) {
+        quiesce(c);
+        dev_free(c, c->chain_ctr);
+        c->chain_ctr_cap = 0;
+        if (dev_alloc(c, &c->chain_ctr, (int64_t)kGemmGroupMax * stride) == GN_OK) c->chain_ctr_cap = (int64_t)kGemmGroupMax * stride;
+      }
+      int ldep[kGemmGroupMax], lall[kGemmGroupMax];
+      // (what an earlier launch wrote is complete by stream order: no dependency inside this launch)
+      for (int k = 0; k < cnt; ++k) { ldep[k] = dep[i + k] < i ? -1 : dep[i + k] - i; lall[k] = dep_all[i + k]; }
+      if (c->chain_ctr) {
+        gn_ctx::EvPair* e = nullptr;
+        if (c->profiling) {
+          if (c->ev_used == c->ev.size()) {
+            gn_ctx::EvPair pnew{};
+            if (cudaEventCreate(&pnew.a) == cudaSuccess && cudaEventCreate(&pnew.b) == cudaSuccess) c->ev.push_back(pnew);
+          }
+          if (c->ev_used < c->ev.size()) {
+            e = &c->ev[c->ev_used++];
+            e->flop = 0.0;
+            for (int k = i; k < j; ++k)
+              e->flop += 2.0 * gs[k].M * (double)gs[k].N * ((double)gs[k].K1 + (gs[k].A2 ? (double)gs[k].K2 : 0.0));
+            e->kind = 0;
+            cudaEventRecord(e->a, c->st);
+          }
+        }
+        const int r = launch_gemm_tf32_group(gs + i, cnt, ldep, lall, c->chain_ctr, stride, c->err_flag + 1, c->st);
+        if (e) cudaEventRecord(e->b, c->st);
+        if (r >= 0) {
+          c->launches += r + 1;             // (the clearing of the counters counts as a launch)
+          c->gemm_seq += (uint64_t)cnt;
+          i = j;
+          continue;
+        }
+        if (e) --c->ev_used;                // nothing was launched: drop the event pair
+      }
+    }
+    run_gemm(c, gs[i]);
+    ++i;
+  }
+}
+
 gn_status ensure_partials(gn_ctx* c, int64_t count) {
   if (count <= c->partial_cap) return GN_OK;
   double* fresh = nullptr;
@@ -466,9 +564,11 @@ const float* Wm(const gn_ctx* c, const float* vec, int m) { return vec + c->w_of
 const float* bm(const gn_ctx* c, const float* vec, int m) { return vec + c->b_off[m]; }
 
 // Eq. (xtoz): Zout[m] = sigma(Zout[m-1] W^m + 1 b^mT), m = 1..L, over `rows` rows; Zout[0] = Z0.
-void forward_pass(gn_ctx* c, const float* Z0, int64_t rows, std::vector<float*>& Zout) {
+void forward_pass(gn_ctx* c, const float* Z0, int64_t rows, std::vector<float*>& Zout, bool emit_parts = false) {
+  std::vector<GemmArgs> gs((size_t)c->L);
+  std::vector<int> dep((size_t)c->L), dep_all((size_t)c->L, 0);
   for (int m = 1; m <= c->L; ++m) {
-    GemmArgs g;
+    GemmArgs& g = gs[(size_t)m - 1];
     g.M = (int)rows; g.N = c->w[m];
     g.A1 = m == 1 ? Z0 : Zout[m - 1]; g.lda1 = c->w[m - 1];
     g.B1 = Wm(c, c->theta, m); g.ldb1 = c->w[m - 1]; g.K1 = c->w[m - 1];
@@ -476,8 +576,10 @@ void forward_pass(gn_ctx* c, const float* Z0, int64_t rows, std::vector<float*>&
     g.D = Zout[m]; g.ldd = c->w[m];
     g.bias = bm(c, c->theta, m);
     g.sigmoid = m < c->L;
-    run_gemm(c, g);
+    g.emit_parts = emit_parts && m < c->L;   // Z_m is an operand of layer m + 1 and of its weight block
+    dep[(size_t)m - 1] = m - 2;          // layer m reads the rows layer m - 1 writes
   }
+  run_gemm_chain(c, gs.data(), dep.data(), dep_all.data(), c->L);
 }
 
 // Parameter-space half of the backward pass for one layer (Eqs. xtow-g, xtow-g-bias, and their
@@ -523,6 +625,7 @@ GemmArgs backward_data_args(const gn_ctx* c, int m, const float* ds, int64_t row
   g.dsig = Zprev; g.ld_dsig = c->w[m - 1]; g.dsig_rows = (int)z_rows;
   g.D = dst; g.ldd = c->w[m - 1];
   g.mn_padded = true;     // B is the context's own (padded) copy of theta
+  g.emit_parts = ds_just_used;   // in the full product and the gradient, delta s^{m-1} feeds the two contractions of layer m - 1
   return g;
 }
 
@@ -543,22 +646,29 @@ gn_status layer_backward(gn_ctx* c, int m, const float* ds_w, int64_t w_rows, co
 // out = coef v + (1/|S|) J^T (2 J v) over the stored subsample (Eq. sampled-Gauss).
 gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
   SideJoin side_guard(c);
+  ++c->parts_epoch;
   const int L = c->L;
   const int64_t nS = c->nS;
-  for (int m = 1; m <= L; ++m) {
-    GemmArgs g;
-    g.M = (int)nS; g.N = c->w[m];
-    if (m == 1) {
-      g.A1 = c->Z[0]; g.lda1 = c->w[0]; g.B1 = Wm(c, v, 1); g.ldb1 = c->w[0]; g.K1 = c->w[0];
-    } else {
-      g.A1 = c->RZ[m - 1]; g.lda1 = c->w[m - 1]; g.B1 = Wm(c, c->theta, m); g.ldb1 = c->w[m - 1]; g.K1 = c->w[m - 1];
-      g.A2 = c->Z[m - 1];  g.lda2 = c->w[m - 1]; g.B2 = Wm(c, v, m);        g.ldb2 = c->w[m - 1]; g.K2 = c->w[m - 1];
+  {
+    std::vector<GemmArgs> gs((size_t)L);
+    std::vector<int> dep((size_t)L), dep_all((size_t)L, 0);
+    for (int m = 1; m <= L; ++m) {
+      GemmArgs& g = gs[(size_t)m - 1];
+      g.M = (int)nS; g.N = c->w[m];
+      if (m == 1) {
+        g.A1 = c->Z[0]; g.lda1 = c->w[0]; g.B1 = Wm(c, v, 1); g.ldb1 = c->w[0]; g.K1 = c->w[0];
+      } else {
+        g.A1 = c->RZ[m - 1]; g.lda1 = c->w[m - 1]; g.B1 = Wm(c, c->theta, m); g.ldb1 = c->w[m - 1]; g.K1 = c->w[m - 1];
+        g.A2 = c->Z[m - 1];  g.lda2 = c->w[m - 1]; g.B2 = Wm(c, v, m);        g.ldb2 = c->w[m - 1]; g.K2 = c->w[m - 1];
+      }
+      g.bias = bm(c, v, m);
+      if (m < L) { g.dsig = c->Z[m]; g.ld_dsig = c->w[m]; g.dsig_rows = (int)nS; }
+      else g.alpha = 2.f;                                   // B = 2I
+      g.D = c->RZ[m]; g.ldd = c->w[m];
+      g.emit_parts = m < L;              // R z^m is an operand of layer m + 1
+      dep[(size_t)m - 1] = m - 2;        // R z^{m-1} of the layer below
     }
-    g.bias = bm(c, v, m);
-    if (m < L) { g.dsig = c->Z[m]; g.ld_dsig = c->w[m]; g.dsig_rows = (int)nS; }
-    else g.alpha = 2.f;                                   // B = 2I
-    g.D = c->RZ[m]; g.ldd = c->w[m];
-    run_gemm(c, g);
+    run_gemm_chain(c, gs.data(), dep.data(), dep_all.data(), L, 2);
   }
   const float* ds = c->RZ[L];
   const float inv = (float)(1.0 / (double)nS);
@@ -574,6 +684,7 @@ gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
 // [(j-1)|S|, j|S|) of every buffer at or above layer j, so each layer runs one stacked GEMM.
 gn_status product_blockdiag(gn_ctx* c, const float* v, float* out, float coef) {
   SideJoin side_guard(c);
+  ++c->parts_epoch;
   const int L = c->L;
   const int64_t nS = c->nS;
   for (int k = 1; k <= L; ++k) {
@@ -619,6 +730,7 @@ bool stored_factors_applicable(const gn_ctx* c) {
 // (Eqs. communi-jaco, ztox-jaco, Jelement-store).  Done once per (theta, S).
 gn_status ensure_factors(gn_ctx* c) {
   if (c->factors_valid) return GN_OK;
+  ++c->parts_epoch;
   const int L = c->L, nL = c->w[L];
   const int64_t nS = c->nS;
   if (nS > c->capF) {
@@ -646,6 +758,7 @@ gn_status ensure_factors(gn_ctx* c) {
 
 gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float coef) {
   SideJoin side_guard(c);
+  ++c->parts_epoch;
   GN_TRY(ensure_factors(c));
   const int L = c->L, nL = c->w[L];
   const int64_t nS = c->nS;
@@ -688,6 +801,7 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
 // Q_a[:, T_b] = D[:, :, T_b]^T 2 D[:, :, T_b] U_a[:, T_b]; then out_W[T_a, :] = Z_{m-1}[:, T_a]^T Q_a / |S|.
 // At the output layer D = I, so Q_a = 2 U_a.
 gn_status product_split(gn_ctx* c, const float* v, float* out, float coef) {
+  ++c->parts_epoch;
   const int L = c->L, nL = c->w[L];
   const int64_t nS = c->nS;
   if (L >= 2) {
@@ -765,6 +879,8 @@ gn_status product_blockdiag_any(gn_ctx* c, const float* v, float* out, float coe
 gn_status ensure_batch(gn_ctx* c) {
   const int64_t rows = c->batch_rows < c->l ? c->batch_rows : c->l;
   if (rows <= c->capB) return GN_OK;
+  quiesce(c);
+  drop_parts(c);
   for (int m = 1; m <= c->L; ++m) { dev_free(c, c->Zb[m], c->capB * c->w[m]); dev_free(c, c->Db[m], c->capB * c->w[m]); }
   c->capB = 0;
   for (int m = 1; m <= c->L; ++m) {
@@ -789,7 +905,8 @@ gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
     const int64_t r0 = b * Rb;
     const int64_t rows = (c->l - r0 < Rb) ? c->l - r0 : Rb;
     const float* X0 = c->dX + r0 * c->w[0];
-    forward_pass(c, X0, rows, c->Zb);
+    ++c->parts_epoch;           // the batch buffers are rewritten
+    forward_pass(c, X0, rows, c->Zb, true);
     c->launches += launch_loss_delta(c->Zb[L], c->dY + r0 * c->w[L], rows * c->w[L], d_grad ? c->Db[L] : nullptr,
                                      c->partial + b * per_batch, c->st);
     {
@@ -1007,7 +1124,8 @@ gn_status gn_set_batch_rows(gn_ctx* c, int64_t rows) {
   c->batch_rows = rows;
   if ((rows < c->l ? rows : c->l) != c->capB && c->capB > 0) {
     // shrink or grow on next use: drop the old workspace now so memory stays bounded
-    cudaStreamSynchronize(c->st);
+    quiesce(c);
+    drop_parts(c);
     for (int m = 1; m <= c->L; ++m) { dev_free(c, c->Zb[m], c->capB * c->w[m]); dev_free(c, c->Db[m], c->capB * c->w[m]); }
     c->capB = 0;
   }
@@ -1095,6 +1213,7 @@ static gn_status set_subsample_impl(gn_ctx* c, const int32_t* idx, int64_t nS, c
   c->factors_valid = false;
   c->bd_count = 0;
   ++c->sub_epoch;             // the stored activations are about to be rewritten
+  ++c->parts_epoch;
   if (nS > c->capS) {
     GN_TRY(sync(c, "set_subsample"));
     // the stored activations move: the hi / lo parts kept for matrices inside the old buffers go with them
@@ -1107,6 +1226,7 @@ static gn_status set_subsample_impl(gn_ctx* c, const int32_t* idx, int64_t nS, c
         ++i;
       }
     }
+    drop_parts(c);
     dev_free(c, c->idx, c->capS);
     for (int m = 0; m <= c->L; ++m) dev_free(c, c->Z[m], c->capS * c->w[m]);
     for (int m = 1; m <= c->L; ++m) { dev_free(c, c->RZ[m], m * c->capS * c->w[m]); dev_free(c, c->DS[m], m * c->capS * c->w[m]); }
@@ -1318,6 +1438,7 @@ gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* d
   // kinds 3..6 are the tensor-core kernel with options: 3 = MN-major operands declared padded,
   // 4 = one CTA per tile forced, 5 = CTA pair per tile forced, 6 = as 5 without splitting tiles
   // between pairs (all with padded operands)
+  ++c->parts_epoch;
   if (kind == 7) {          // error-compensated tensor-core form (3 x TF32, chunked accumulation)
     ++c->gemm_seq;
     if (!run_gemm_x3(c, g)) return fail(c, GN_EINVAL, "the error-compensated tensor-core form does not take this problem");
@@ -1411,6 +1532,8 @@ gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   if (!c) return GN_EINVAL;
   if (option == 2) { if (value < 0) return fail(c, GN_EINVAL, "count must be >= 0"); c->fail_alloc_in = value; return GN_OK; }
   if (option == 3) { quiesce(c); c->side_enabled = value != 0; return GN_OK; }
+  if (option == 5) { c->parts_enabled = value != 0; return GN_OK; }
+  if (option == 4) { c->chain_level = value < 0 ? 0 : (value > 2 ? 2 : value); return GN_OK; }
   if (option == 0) c->group_enabled = value != 0;
   else if (option == 1) c->sk_enabled = value != 0 && c->sk_enabled;
   else return fail(c, GN_EINVAL, "unknown option");

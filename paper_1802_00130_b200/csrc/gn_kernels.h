@@ -27,6 +27,11 @@ struct GemmArgs {
   // layouts and leading dimensions for the lo parts), and acc = sum Alo Bhi + Ahi Blo + Ahi Bhi.
   const float* A1lo = nullptr; const float* B1lo = nullptr; const float* A2lo = nullptr; const float* B2lo = nullptr;
   bool a1_split_fresh = false;   // caller's word that A1 is, unchanged, the A1 of the previous contraction
+  // Error-compensated form: the result will itself be an operand of a later contraction (emit_parts, set by the
+  // caller), and where the hi / lo parts of every stored value go (Dhi, Dlo with leading dimension ld_parts,
+  // filled in by the host logic that owns the buffers).
+  bool emit_parts = false;
+  float* Dhi = nullptr; float* Dlo = nullptr; int64_t ld_parts = 0;
   bool a_kmajor = true, b_kmajor = true;
   bool mn_padded = false;  // every MN-major operand is followed by >= 128 readable bytes
   int two_cta = -1;        // tensor-core kernel: -1 choose, 0 one CTA per tile, 1 CTA pair per 256-row tile
@@ -59,11 +64,20 @@ int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st);
 int64_t gemm_tf32_workspace_floats();
 int gemm_tf32_workspace_flags();
 int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st);
-// Up to three independent problems, each suited to the CTA-pair kernel (M > 128, N >= 128), as ONE launch whose
-// pairs walk a common, host-balanced work list: the tiles of one problem fill the partial last wave of another.
-// Whole tiles only.  Returns launches made, or -1 if the group cannot run this way (run the problems one by one).
+// Up to five problems, each suited to the CTA-pair kernel (M > 128, N >= 128), as ONE launch whose pairs walk a
+// common, host-balanced work list.  Whole tiles only.
+//   dep_prob == nullptr: independent problems, longest tiles first; the tiles of one fill the partial last wave
+//   of another.
+//   dep_prob != nullptr: a chain in the given order; problem i reads, as its FIRST A operand (row panels) or, with
+//   dep_all[i] != 0, as an operand whose K runs over the producer's rows, the output of problem dep_prob[i] < i
+//   (-1: none).  The consumer's tiles wait (bounded) for the producer's, so the layers of a pass overlap instead
+//   of each draining the GPU.  `done`: device scratch of n * done_stride ints (done_stride > M / 256 + 1),
+//   cleared by the call.
+// Returns launches made, or -1 if the group cannot run this way (run the problems one by one, in order).
+constexpr int kGemmGroupMax = 5;
 bool gemm_tf32_group_eligible(const GemmArgs* gs, int n);
-int launch_gemm_tf32_group(const GemmArgs* gs, int n, int* err_flag, cudaStream_t st);
+int launch_gemm_tf32_group(const GemmArgs* gs, int n, const int* dep_prob, const int* dep_all, int* done,
+                           int done_stride, int* err_flag, cudaStream_t st);
 
 // Streaming FP32 kernels for contractions with one dimension <= 16 (the n_L-wide output layer).
 // gemm_thin_kind says which of them (if any) takes a problem; THIN_M needs a scratch buffer of

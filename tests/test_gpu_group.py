@@ -1,6 +1,7 @@
-"""Independent work of a layer issued together: its large contractions as one launch of the CTA-pair kernel (TF32
-mode), its bias column sums and n_L-row weight block on a side stream.  Same bits as one launch after the other on
-one stream, and the usual bound against the float64 checker."""
+"""Work issued together: the independent large contractions of a layer as one launch of the CTA-pair kernel (TF32
+mode), its bias column sums and n_L-row weight block on a side stream, and the consecutive layers of a pass as one
+launch whose tiles wait for the tiles they read.  Same bits as one launch after the other on one stream, and the
+usual bound against the float64 checker."""
 import numpy as np
 import pytest
 
@@ -24,11 +25,12 @@ def test_grouped_launches_give_the_bits_of_single_launches(name):
     import torch
     p = CASES[name]()
     outs = []
-    for grouped, side in ((0, 0), (1, 1), (1, 0), (0, 1)):
+    for grouped, side, chain in ((0, 0, 0), (1, 1, 2), (1, 0, 0), (0, 1, 1), (0, 0, 2)):
         ctx = make_ctx(p, "tf32")
         ctx.debug_option(1, 0)                  # whole tiles only in every run: K slices change the order of sums
         ctx.debug_option(0, grouped)
         ctx.debug_option(3, side)
+        ctx.debug_option(4, chain)
         ctx.set_subsample(dev(p["idx"]))
         v = dev(p["v"])
         res = [ctx.Gv(v).clone()]
@@ -36,6 +38,8 @@ def test_grouped_launches_give_the_bits_of_single_launches(name):
             ctx.set_blockdiag_method(method)
             res.append(ctx.Gv_blockdiag(v).clone())
         res.append(ctx.grad().clone())
+        for m in range(1, len(p["widths"])):        # the stored forward pass itself
+            res.append(ctx.debug_activations(m).clone())
         launches = ctx.kernel_launches
         outs.append((res, launches))
         ctx.close()
@@ -51,3 +55,37 @@ def test_grouped_launches_give_the_bits_of_single_launches(name):
     assert relb(res[1], ref_b, w) <= TOL["tf32"]
     assert relb(res[2], ref_b, w) <= TOL["tf32"]
     assert relb(res[3], orc.grad(th, w, C, p["X"], p["Y"]), w) <= TOL["tf32"]
+
+
+@pytest.mark.parametrize("name", ["mid", "deep", "mnist2000_5"])
+def test_parts_written_by_the_epilogue_are_the_parts_a_separate_pass_would_write(name):
+    """FP32-accurate mode: the error-compensated kernel writes the hi / lo TF32 parts of a result that a later
+    contraction of the same product (or row batch) takes as an operand.  Same bits as splitting that result in a pass
+    of its own, fewer launches, and the mode's bound against the float64 checker."""
+    import torch
+    p = CASES[name]()
+    outs = []
+    for emit in (0, 1):
+        ctx = make_ctx(p, "fp32")
+        ctx.debug_option(5, emit)
+        ctx.set_subsample(dev(p["idx"]))
+        v = dev(p["v"])
+        res = [ctx.Gv(v).clone(), ctx.grad().clone(), ctx.Gv(v).clone()]
+        for method in (1, 2):
+            ctx.set_blockdiag_method(method)
+            res.append(ctx.Gv_blockdiag(v).clone())
+        res.append(ctx.Gv(v).clone())           # after the block-diagonal products have rewritten the same buffers
+        outs.append((res, ctx.kernel_launches))
+        ctx.close()
+    for a, b in zip(outs[0][0], outs[1][0]):
+        assert torch.equal(a, b)
+    assert outs[1][1] < outs[0][1]
+    XS = p["X"][p["idx"]]
+    th, w, C = p["theta"], p["widths"], p["C"]
+    res = [r.cpu().numpy() for r in outs[1][0]]
+    ref = orc.Gv(th, w, C, XS, p["v"])
+    for k in (0, 2, 5):
+        assert relb(res[k], ref, w) <= TOL["fp32"]
+    assert relb(res[1], orc.grad(th, w, C, p["X"], p["Y"]), w) <= TOL["fp32"]
+    ref_b = orc.Gv_blockdiag(th, w, C, XS, p["v"])
+    assert relb(res[3], ref_b, w) <= TOL["fp32"] and relb(res[4], ref_b, w) <= TOL["fp32"]
