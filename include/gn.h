@@ -78,7 +78,9 @@ typedef enum {
  *   l            number of training rows, >= 1.
  *   dX, dY       device, [l][n_0] and [l][n_L], borrowed.
  *   prec         arithmetic of the contractions.
- *   cuda_stream  a cudaStream_t (NULL = the legacy default stream).
+ *   cuda_stream  a cudaStream_t.  NULL: the context creates a blocking stream of its own, which orders itself with
+ *                work on the legacy default stream as CUDA's blocking streams do (a stream that can be captured is
+ *                needed for the graph replay of small CG solves; the legacy default stream cannot).
  * Errors: GN_EINVAL for bad arguments, GN_ECUDA if no device / wrong architecture, GN_ENOMEM.
  */
 gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_t l,
@@ -96,8 +98,10 @@ const char* gn_last_error(const gn_ctx* ctx);
 /* gn_workspace_bytes - device memory currently owned by the context. */
 int64_t gn_workspace_bytes(const gn_ctx* ctx);
 
-/* gn_kernel_launches - number of kernels this context has launched so far (all entry points). */
+/* gn_kernel_launches - number of kernels this context has launched so far (all entry points; the kernels of a
+ * replayed graph count as if launched one by one).  gn_graph_replays - CG steps issued as one graph launch. */
 int64_t gn_kernel_launches(const gn_ctx* ctx);
+int64_t gn_graph_replays(const gn_ctx* ctx);
 
 /*
  * gn_set_batch_rows - number of rows processed at a time by gn_fun / gn_grad, which walk the
@@ -335,8 +339,9 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
  * next to the layer's large contractions (value 0 = everything on the context's stream); option 4: consecutive
  * layers of a pass as one launch whose tiles wait for the tiles they read (value 0 = one launch per layer, 1 = the
  * stored forward pass, the default, 2 = also the forward R pass of a product).  Option 5 (GN_FP32_ACCURATE contexts): the error-compensated kernel also writes the hi / lo parts
- * of a result that a later contraction takes as an operand (value 0 = a separate pass splits it).  Results do not
- * depend on options 0, 3, 4 and 5 (tiles, sums and parts are computed identically); GN_EINVAL for an unknown option.
+ * of a result that a later contraction takes as an operand (value 0 = a separate pass splits it).  Option 6: fixed-length
+ * CG solves of small problems replay one captured step as a CUDA graph (value 0 = plain launches).  Results do not
+ * depend on options 0, 3, 4, 5 and 6 (tiles, sums and parts are computed identically); GN_EINVAL for an unknown option.
  */
 gn_status gn_debug_option(gn_ctx* ctx, int option, int value);
 

@@ -20,6 +20,7 @@ _SIGNATURES = {
     "gn_last_error": (C.c_char_p, [_vp]),
     "gn_workspace_bytes": (_i64, [_vp]),
     "gn_kernel_launches": (_i64, [_vp]),
+    "gn_graph_replays": (_i64, [_vp]),
     "gn_set_batch_rows": (_i32, [_vp, _i64]),
     "gn_set_blockdiag_method": (_i32, [_vp, _i32]),
     "gn_set_accurate_method": (_i32, [_vp, _i32]),
@@ -193,6 +194,10 @@ class GnContext:
     @property
     def kernel_launches(self):
         return int(self._lib.gn_kernel_launches(self._h))
+
+    @property
+    def graph_replays(self):
+        return int(self._lib.gn_graph_replays(self._h))
 
     # ------------------------------------------------------------------ entry points
     def set_batch_rows(self, rows):

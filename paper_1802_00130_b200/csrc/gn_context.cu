@@ -100,6 +100,19 @@ struct gn_ctx {
   float* cg_r = nullptr; float* cg_p = nullptr; float* cg_q = nullptr;
   CgControl* cg_ctl = nullptr; CgControl* h_ctl = nullptr;   // device-resident solver state and its pinned mirror
   double* cg_hist = nullptr; int cg_hist_cap = 0;            // squared residual norms, one per step
+  // One CG step (product + the three vector kernels) as a CUDA graph, for problems small enough that issuing the
+  // step's ~20 launches from the host takes as long as running them: captured from the second step of a
+  // fixed-length solve and replayed for the rest; kept across solves while nothing it has baked in changes.
+  struct CgGraph {
+    cudaGraphExec_t exec = nullptr;
+    uint64_t alloc_gen = 0; int64_t nS = 0; float coef = 0.f; const float* d = nullptr; int stored = 0, method = 0, n_seg = 0;
+    int64_t launches = 0;
+  };
+  CgGraph cg_graph[2];
+  bool graph_enabled = true, graph_ok = true;
+  int64_t graph_replays = 0;
+  bool own_stream = false;     // no stream was given: the context made one (stream capture cannot use the legacy default stream)
+  uint64_t alloc_gen = 1;      // bumped by every device allocation and release of the context
   float* tmp_a = nullptr; float* tmp_b = nullptr;  // staging for *_host calls
   float* nt[4] = {nullptr, nullptr, nullptr, nullptr};  // Newton iteration: g, d, G d / G dbar, trial theta
   CgChunk* chunks[2] = {nullptr, nullptr}; int n_chunks[2] = {0, 0};
@@ -158,6 +171,7 @@ gn_status dev_alloc(gn_ctx* c, T** p, int64_t count) {
     return fail(c, GN_ENOMEM, std::string("cudaMalloc of ") + std::to_string(count * (int64_t)sizeof(T)) + " bytes: " + cudaGetErrorString(e));
   }
   c->bytes += count * (int64_t)sizeof(T);
+  ++c->alloc_gen;
   c->owned.push_back({q, count * (int64_t)sizeof(T)});
   *p = static_cast<T*>(q);
   return GN_OK;
@@ -171,6 +185,7 @@ void dev_free(gn_ctx* c, T*& p, int64_t = 0) {
     if (o.p == (void*)p) { c->bytes -= o.bytes; o.p = nullptr; o.bytes = 0; break; }
   cudaFree(p);
   p = nullptr;
+  ++c->alloc_gen;
   // keep the registry from growing without bound across many regrowths
   if (c->owned.size() > 4096) {
     size_t k = 0;
@@ -1060,6 +1075,12 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
   c->w.assign(widths, widths + L + 1);
   c->C = C; c->l = l; c->dX = dX; c->dY = dY; c->prec = prec;
   c->st = static_cast<cudaStream_t>(cuda_stream);
+  if (!c->st) {
+    // a blocking stream of the context's own: it orders itself with work on the legacy default stream the way
+    // CUDA's blocking streams do, so a caller that works on that stream sees no difference
+    if (cudaStreamCreate(&c->st) != cudaSuccess) { cudaGetLastError(); delete c; return GN_ECUDA; }
+    c->own_stream = true;
+  }
   c->w_off.assign(L + 2, 0); c->b_off.assign(L + 2, 0);
   int64_t off = 0;
   for (int m = 1; m <= L; ++m) {
@@ -1099,6 +1120,8 @@ gn_status gn_create(gn_ctx** out, int L, const int32_t* widths, double C, int64_
 gn_status gn_destroy(gn_ctx* c) {
   if (!c) return GN_OK;
   quiesce(c);
+  for (auto& g : c->cg_graph) if (g.exec) cudaGraphExecDestroy(g.exec);
+  if (c->own_stream) cudaStreamDestroy(c->st);
   if (c->st2) cudaStreamDestroy(c->st2);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
@@ -1117,6 +1140,7 @@ int64_t gn_num_params(const gn_ctx* c) { return c ? c->n : -1; }
 const char* gn_last_error(const gn_ctx* c) { return c ? c->err.c_str() : "null context"; }
 int64_t gn_workspace_bytes(const gn_ctx* c) { return c ? c->bytes : -1; }
 int64_t gn_kernel_launches(const gn_ctx* c) { return c ? c->launches : -1; }
+int64_t gn_graph_replays(const gn_ctx* c) { return c ? c->graph_replays : -1; }
 
 gn_status gn_set_batch_rows(gn_ctx* c, int64_t rows) {
   if (!c) return GN_EINVAL;
@@ -1356,16 +1380,65 @@ gn_status gn_cg_solve(gn_ctx* c, const float* d_g, double lambda, int blockdiag,
   int it = 0;
   c->bd_expect = blockdiag ? max_iter : 0;
   struct Reset { int* p; ~Reset() { *p = 0; } } reset_expect{&c->bd_expect};
-  while (it < max_iter && active > 0.5) {
-    // Section 4.4: all partitions stop once cg_min steps are done and the stated share of them have finished
-    if (rule44 && it >= c->cg_min && (double)n_seg - active >= c->cg_share * (double)n_seg) break;
+  auto one_step = [&]() -> gn_status {
     GN_TRY(blockdiag ? product_blockdiag_any(c, c->cg_p, c->cg_q, coef) : product_full(c, c->cg_p, c->cg_q, coef));
     c->launches += launch_cg_dot(c->cg_p, c->cg_q, ch, nc, c->partial, seg, n_seg, c->cg_ctl, c->st);
     c->launches += launch_cg_update(c->cg_p, c->cg_q, d_d, c->cg_r, ch, nc, seg, n_seg, tol, c->partial, c->cg_ctl, c->st);
     c->launches += launch_cg_direction(c->cg_r, c->cg_p, ch, nc, seg, c->st);
+    return check_launch(c, "cg step");
+  };
+  // Fixed-length solve of a small problem: the step's launches are issued once, into a graph, and replayed.
+  double step_flop = 0.0;
+  for (int m = 1; m <= c->L; ++m) step_flop += (m == 1 ? 4.0 : 8.0) * (double)c->w[m - 1] * c->w[m] * (double)c->nS;
+  const bool use_graph = !watch && !d_iterates && !c->profiling && c->graph_enabled && c->graph_ok && max_iter >= 4 &&
+                         step_flop < 120e9;
+  gn_ctx::CgGraph& cgg = c->cg_graph[mode];
+  while (it < max_iter && active > 0.5) {
+    // Section 4.4: all partitions stop once cg_min steps are done and the stated share of them have finished
+    if (rule44 && it >= c->cg_min && (double)n_seg - active >= c->cg_share * (double)n_seg) break;
+    if (use_graph && it >= 1) {
+      // (the first step ran as plain launches: every workspace it needs exists and the stored factors are built)
+      const bool fits = cgg.exec && cgg.alloc_gen == c->alloc_gen && cgg.nS == c->nS && cgg.coef == coef && cgg.d == d_d &&
+                        cgg.stored == (c->factors_valid ? 1 : 0) && cgg.method == c->bd_method && cgg.n_seg == n_seg;
+      if (!fits) {
+        if (cgg.exec) { cudaGraphExecDestroy(cgg.exec); cgg.exec = nullptr; }
+        const int64_t before = c->launches;
+        const uint64_t gen = c->alloc_gen;
+        cudaGraph_t graph = nullptr;
+        gn_status st = GN_OK;
+        if (cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+          st = one_step();
+          const cudaError_t e = cudaStreamEndCapture(c->st, &graph);
+          if (st == GN_OK && e == cudaSuccess && graph && gen == c->alloc_gen &&
+              cudaGraphInstantiate(&cgg.exec, graph, 0) == cudaSuccess) {
+            cgg.alloc_gen = gen; cgg.nS = c->nS; cgg.coef = coef; cgg.d = d_d; cgg.stored = c->factors_valid ? 1 : 0;
+            cgg.method = c->bd_method; cgg.n_seg = n_seg; cgg.launches = c->launches - before;
+          } else {
+            cgg.exec = nullptr;
+          }
+          if (graph) cudaGraphDestroy(graph);
+          c->launches = before;              // nothing has run yet: the captured step runs when the graph is launched
+        }
+        cudaGetLastError();
+        if (!cgg.exec) {                     // capture is not available here: plain launches from now on
+          c->graph_ok = false;
+          c->sticky = GN_OK;
+          GN_TRY(one_step());
+          ++it;
+          continue;
+        }
+      }
+      if (c->graph_ok && cgg.exec) {
+        GN_CUDA(c, cudaGraphLaunch(cgg.exec, c->st));
+        c->launches += cgg.launches;
+        ++c->graph_replays;
+        ++it;
+        continue;
+      }
+    }
+    GN_TRY(one_step());
     if (d_iterates)
       GN_CUDA(c, cudaMemcpyAsync(d_iterates + (int64_t)it * c->n, d_d, c->n * sizeof(float), cudaMemcpyDeviceToDevice, c->st));
-    GN_TRY(check_launch(c, "cg step"));
     if (watch) {
       GN_CUDA(c, cudaMemcpyAsync(c->h_ctl, c->cg_ctl, sizeof(CgControl), cudaMemcpyDeviceToHost, c->st));
       GN_TRY(sync(c, "cg step"));
@@ -1532,6 +1605,7 @@ gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   if (!c) return GN_EINVAL;
   if (option == 2) { if (value < 0) return fail(c, GN_EINVAL, "count must be >= 0"); c->fail_alloc_in = value; return GN_OK; }
   if (option == 3) { quiesce(c); c->side_enabled = value != 0; return GN_OK; }
+  if (option == 6) { c->graph_enabled = value != 0; return GN_OK; }
   if (option == 5) { c->parts_enabled = value != 0; return GN_OK; }
   if (option == 4) { c->chain_level = value < 0 ? 0 : (value > 2 ? 2 : value); return GN_OK; }
   if (option == 0) c->group_enabled = value != 0;

@@ -89,3 +89,40 @@ def test_parts_written_by_the_epilogue_are_the_parts_a_separate_pass_would_write
     assert relb(res[1], orc.grad(th, w, C, p["X"], p["Y"]), w) <= TOL["fp32"]
     ref_b = orc.Gv_blockdiag(th, w, C, XS, p["v"])
     assert relb(res[3], ref_b, w) <= TOL["fp32"] and relb(res[4], ref_b, w) <= TOL["fp32"]
+
+
+@pytest.mark.parametrize("mode", ["fp32", "tf32"])
+@pytest.mark.parametrize("name", ["tiny", "ragged", "mid"])
+def test_replayed_cg_step_gives_the_bits_of_plain_launches(name, mode):
+    """Fixed-length CG solves of small problems capture their second step as a CUDA graph and replay it; the graph is
+    kept across solves.  Same iterates and residual norms, bit for bit, as plain launches: over two subsamples, two
+    damping values and both kinds of system, with an early-stopping solve (which never uses the graph) in between."""
+    import torch
+    p = wl.make(name)
+    g = dev(orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]).astype(np.float32))
+    idx2 = np.ascontiguousarray(p["idx"][::-1])
+    runs = []
+    for graph in (0, 1):
+        ctx = make_ctx(p, mode)
+        ctx.debug_option(6, graph)
+        got = []
+        for idx, lam in ((p["idx"], 1.0), (idx2, 1.0), (idx2, 0.5)):
+            ctx.set_subsample(dev(idx))
+            for blockdiag in (False, True):
+                d, its, res = ctx.cg_solve(g, lam, blockdiag=blockdiag, max_iter=9, tol=0.0)
+                assert its == 9
+                got.append((d.clone(), res.copy()))
+            d, its, res = ctx.cg_solve(g, lam, blockdiag=True, max_iter=50, tol=1e-2)
+            got.append((d.clone(), res.copy()))
+        runs.append(got)
+        # 6 fixed-length solves of 9 steps: the first step of each is plain, the other 8 are replays
+        assert ctx.graph_replays == (6 * 8 if graph else 0)
+        ctx.close()
+    for (d0, r0), (d1, r1) in zip(*runs):
+        assert torch.equal(d0, d1)
+        assert np.array_equal(r0, r1)
+    # and against the checker (first solve, full system)
+    XS = p["X"][p["idx"]]
+    d_ref, _, _ = orc.cg_solve(p["theta"], p["widths"], p["C"], XS, g.cpu().numpy(), 1.0, False, 9, 0.0)
+    tol = 1e-4 if mode == "fp32" else 2e-2
+    assert np.linalg.norm(runs[1][0][0].cpu().numpy() - d_ref) <= tol * np.linalg.norm(d_ref)
