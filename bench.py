@@ -357,6 +357,29 @@ def run_ours(args):
     breakdown["set_subsample"] = {"ms": 1e3 * t_sub,
                                   "Gv_per_s_amortised": {str(k): k / (t_sub + k * t_gv) for k in (10, 50, 250)}}
 
+    # ---- the same products in FP32-accurate mode (error-compensated tensor-core contractions), for the record of
+    # that mode in the default run
+    if args.mode == "tf32" and not args.no_fp32_leg:
+        ctx32 = gn.GnContext(p["widths"], p["C"], X, Y, gn.GN_FP32_ACCURATE)
+        ctx32.set_theta(theta)
+        ctx32.set_subsample(idx_dev[0])
+        leg = {}
+        for name, fn, mac in (("Gv", ctx32.Gv, macs["full"]), ("Gv_blockdiag", ctx32.Gv_blockdiag, macs["block_paper"])):
+            for _ in range(2):
+                fn(v, out=out)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(max(3, args.product_reps // 2)):
+                fn(v, out=out)
+            b.record()
+            torch.cuda.synchronize()
+            t = a.elapsed_time(b) * 1e-3 / max(3, args.product_reps // 2)
+            leg[name] = {"per_s": 1.0 / t, "ms": 1e3 * t, "algorithmic_tflops": 2.0 * mac * p["nS"] / t / 1e12}
+        breakdown["fp32_accurate_mode"] = leg
+        ctx32.close()
+        del ctx32
+
     # ---- a library TF32 product of 8192^3 in the same run: what a plain GEMM sustains on this GPU (context only)
     lib_tf32 = None
     if args.mode == "tf32":
@@ -483,6 +506,8 @@ def main():
     ap.add_argument("--product-reps", type=int, default=10)
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-fp32-leg", dest="no_fp32_leg", action="store_true",
+                    help="skip the FP32-accurate products of the breakdown (they need a second context's workspaces)")
     ap.add_argument("--dry-run", action="store_true",
                     help="rehearse the launch of the ranks and the aggregation over them on CPU (gloo); no kernels, no value")
     args = ap.parse_args()
