@@ -838,6 +838,7 @@ gn_status product_split(gn_ctx* c, const float* v, float* out, float coef) {
     c->capSplit = need;
   }
   const float inv = (float)(1.0 / (double)nS);
+  std::vector<GemmArgs> batch;
   for (int m = 1; m <= L; ++m) {
     const int sa = c->split[m - 1], sb = c->split[m], np = c->w[m - 1], nm = c->w[m];
     const int64_t stride = nS * nm;
@@ -849,8 +850,11 @@ gn_status product_split(gn_ctx* c, const float* v, float* out, float coef) {
       if (a == 0) g.bias = bm(c, v, m);
       if (m == L) g.alpha = 2.f;                          // B = 2I
       g.D = c->SU + a * stride; g.ldd = nm;
-      run_gemm(c, g);
+      batch.push_back(g);
     }
+    // the groups' contractions are independent of one another: up to sixteen at a time to the group launcher
+    for (size_t b0 = 0; b0 < batch.size(); b0 += 16) run_gemm_group(c, batch.data() + b0, (int)std::min<size_t>(16, batch.size() - b0));
+    batch.clear();
     const float* Q = c->SU;
     if (m < L) {
       c->launches += launch_factor_apply(c->DF[m], c->SU, nS, nL, nm, sb, sa, stride, c->SQ, c->st);
@@ -867,8 +871,10 @@ gn_status product_split(gn_ctx* c, const float* v, float* out, float coef) {
       g.alpha = inv;
       g.cin = v + c->w_off[m] + t0; g.ld_cin = np; g.beta = coef;
       g.D = out + c->w_off[m] + t0; g.ldd = np;
-      run_gemm(c, g);
+      batch.push_back(g);
     }
+    for (size_t b0 = 0; b0 < batch.size(); b0 += 16) run_gemm_group(c, batch.data() + b0, (int)std::min<size_t>(16, batch.size() - b0));
+    batch.clear();
     GN_TRY(ensure_colsum(c, nS, nm));
     c->launches += launch_colsum(Q, nS, nm, nm, inv, v + c->b_off[m], coef, out + c->b_off[m], c->colsum_scratch, c->st);
   }
