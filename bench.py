@@ -33,8 +33,14 @@ METRIC = "gauss_newton_matvecs_per_s"
 UNIT = "matvec/s"
 FP32_LANES_PER_SM, SMS = 128, 148
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant GEMM kernel from an ncu capture of the
-# kernel as it stands (profiles/); None where no capture of the current kernel exists
-TRAFFIC = {}
+# kernel as it stands.  Multi-pass counters are only taken on the small case (|S| = 3000), so the figure belongs to
+# that workload; for every other workload `traffic` is None and the small-case figure is quoted beside it.
+TRAFFIC = {("tf32", "mnist2000_5"): {"bytes_per_launch": 150.4e6, "kernel": "gemm_tf32_2cta_kernel",
+                                     "launch": "forward R pass of a hidden layer, 3000 x 2000 x (2000 + 2000); 128 MB algorithmic",
+                                     "source": "profiles/gemm_tf32_2cta_mnist2000_5_ncu.md"},
+           ("fp32", "mnist2000_5"): {"bytes_per_launch": 143.2e6, "kernel": "gemm_tf32x3_kernel",
+                                     "launch": "3000 x 2000 x 2000-class contraction on hi / lo parts",
+                                     "source": "profiles/gemm_tf32x3_mnist2000_5_ncu.md"}}
 
 
 def peaks():
@@ -460,7 +466,9 @@ def run_ours(args):
                             "ffma": "gemm_ffma_kernel"}[main],
                  "achieved": achieved, "frac": achieved / peak if achieved else None,
                  "traffic": (TRAFFIC.get((args.mode, args.workload)) or {}).get("bytes_per_launch"),
-                 "traffic_note": TRAFFIC.get((args.mode, args.workload)),
+                 "traffic_note": TRAFFIC.get((args.mode, args.workload)) or
+                                 {"small_case": TRAFFIC.get((args.mode, "mnist2000_5")),
+                                  "why_null": "counters of the current kernel were taken on the small case only"},
                  "launches": kern["launches"], "avg_launch_us": 1e3 * kern["ms"] / max(1, kern["launches"]),
                  "share_of_step": kern["ms"] / ms_profiled if ms_profiled > 0 else None,
                  "timing": "CUDA events around every launch of the kernel, on its stream, in a second pass over the same "
