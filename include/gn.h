@@ -231,11 +231,17 @@ gn_status gn_Gv_blockdiag_host(gn_ctx* ctx, const float* h_v, float* h_out);
  *   tol            sigma of Eq. (CG-stopping-cond): stop once ||(A + lambda I) d + g|| <= tol ||g||
  *                  (per block with blockdiag); tol <= 0 runs exactly max_iter steps.
  *   d_d            device [n], receives d.
- *   iters_host     optional, receives the number of steps taken.
+ *   iters_host     optional, receives the number of steps taken (steps at whose start some system was still
+ *                  active: a right-hand side of zero, or a residual that reaches exactly zero, ends the count).
  *   d_iterates     optional device [max_iter][n]: row k receives d after step k+1.
  *   resnorm_host   optional host [max_iter+1]: entry k is the residual norm after k steps
  *                  (over all coordinates).
- * Synchronises the stream once per step (the stop test is taken on the host).
+ * The step lengths, the stop tests, the step count and the residual history are computed and kept on the device.
+ * With tol <= 0 (and no termination rule set by gn_set_cg_termination) all max_iter steps are enqueued without
+ * waiting and the stream is synchronised once, at the end; such a solve of a small problem (less than 120 GFLOP
+ * per step) captures its second step as a CUDA graph and replays it, and keeps the graph for later solves of the same
+ * shape.  With tol > 0 or a termination rule the host reads two numbers after every step (one synchronisation per
+ * step), because it has to stop issuing steps.
  */
 gn_status gn_cg_solve(gn_ctx* ctx, const float* d_g, double lambda, int blockdiag, int max_iter,
                       double tol, float* d_d, int* iters_host, float* d_iterates,

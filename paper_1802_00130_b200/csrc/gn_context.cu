@@ -38,8 +38,12 @@ struct gn_ctx {
   int64_t nS = 0, capS = 0;
   int32_t* idx = nullptr;
   std::vector<float*> Z;    // Z[0] = X_S, Z[m] = [nS][n_m]
-  std::vector<float*> RZ;   // RZ[m] = [m * nS][n_m]: forward directional derivatives (stacked streams)
-  std::vector<float*> DS;   // DS[m] = [m * nS][n_m]: backward quantities d(.)/d s^m
+  // RZ[m], DS[m]: forward directional derivatives and backward quantities d(.)/d s^m, [|S|][n_m]; once the
+  // propagate form of the block-diagonal product has been asked for they are m |S| rows deep (its L streams
+  // stacked along rows), see ensure_stacked
+  std::vector<float*> RZ;
+  std::vector<float*> DS;
+  bool stacked = false;     // RZ / DS hold m * capS rows (else capS rows)
   // stored Jacobian factors d z^L / d s^m on the subsample (block-diagonal product, Section 3.3.1)
   std::vector<float*> DF;   // DF[m] = [nS * n_L][n_m], m = 1..L-1
   int64_t capF = 0;         // rows of S the factor buffers hold
@@ -697,7 +701,31 @@ gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
 // Eq. (approx-jaco), one block per layer.  The perturbation of layer k is pushed to the output and
 // pulled back to layer k only; the L streams are stacked along rows, stream j occupying rows
 // [(j-1)|S|, j|S|) of every buffer at or above layer j, so each layer runs one stacked GEMM.
+// The propagate form stacks its L streams along rows: the first time it is asked for, RZ_m and DS_m are regrown
+// to m |S| rows (contexts that only ever use the full product and the stored factors never pay for that).
+gn_status ensure_stacked(gn_ctx* c) {
+  if (c->stacked) return GN_OK;
+  quiesce(c);
+  drop_parts(c);
+  for (int m = 1; m <= c->L; ++m) { dev_free(c, c->RZ[m]); dev_free(c, c->DS[m]); }
+  c->stacked = true;
+  for (int m = 1; m <= c->L; ++m) {
+    gn_status st = dev_alloc(c, &c->RZ[m], (int64_t)m * c->capS * c->w[m]);
+    if (st == GN_OK && m < c->L) st = dev_alloc(c, &c->DS[m], (int64_t)m * c->capS * c->w[m]);
+    if (st != GN_OK) {
+      // leave a consistent, empty state: the next set_subsample allocates afresh
+      for (int k = 1; k <= c->L; ++k) { dev_free(c, c->RZ[k]); dev_free(c, c->DS[k]); }
+      for (int k = 0; k <= c->L; ++k) dev_free(c, c->Z[k]);
+      dev_free(c, c->idx);
+      c->capS = 0; c->have_sub = false; c->factors_valid = false;
+      return st;
+    }
+  }
+  return GN_OK;
+}
+
 gn_status product_blockdiag(gn_ctx* c, const float* v, float* out, float coef) {
+  GN_TRY(ensure_stacked(c));
   SideJoin side_guard(c);
   ++c->parts_epoch;
   const int L = c->L;
@@ -1264,8 +1292,9 @@ static gn_status set_subsample_impl(gn_ctx* c, const int32_t* idx, int64_t nS, c
     GN_TRY(dev_alloc(c, &c->idx, nS));
     for (int m = 0; m <= c->L; ++m) GN_TRY(dev_alloc(c, &c->Z[m], nS * c->w[m]));
     for (int m = 1; m <= c->L; ++m) {
-      GN_TRY(dev_alloc(c, &c->RZ[m], m * nS * c->w[m]));
-      if (m < c->L) GN_TRY(dev_alloc(c, &c->DS[m], m * nS * c->w[m]));
+      const int64_t depth = c->stacked ? m : 1;
+      GN_TRY(dev_alloc(c, &c->RZ[m], depth * nS * c->w[m]));
+      if (m < c->L) GN_TRY(dev_alloc(c, &c->DS[m], depth * nS * c->w[m]));
     }
     c->capS = nS;
   }
