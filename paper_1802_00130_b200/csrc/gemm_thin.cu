@@ -136,7 +136,7 @@ template <int MMAX>
 __global__ void __launch_bounds__(256) gemm_thin_m_partial_kernel(const ThinMParams p) {
   // 256 threads = 2 row-halves x 128 column threads: half h takes rows h, h + 2, ... of the chunk, so
   // that twice as many 16-byte loads of B are in flight; the halves are added at the end.
-  __shared__ float As[TM_ROWS][MMAX];
+  __shared__ __align__(16) float As[TM_ROWS][MMAX];    // (MMAX is a multiple of 4: a row is read back as 16-byte groups)
   __shared__ float4 Hs[MMAX][128];
   const int ct = threadIdx.x & 127, half = threadIdx.x >> 7;
   const int n = (blockIdx.x * 128 + ct) * 4;
@@ -158,10 +158,15 @@ __global__ void __launch_bounds__(256) gemm_thin_m_partial_kernel(const ThinMPar
       for (int r = half; r < cnt; r += 2) {
         const float4 b = __ldg(reinterpret_cast<const float4*>(p.B + (rb + r) * p.ldb + n));
 #pragma unroll
-        for (int m = 0; m < MMAX; ++m) {
-          const float a = As[r][m];
-          acc[m].x = fmaf(a, b.x, acc[m].x); acc[m].y = fmaf(a, b.y, acc[m].y);
-          acc[m].z = fmaf(a, b.z, acc[m].z); acc[m].w = fmaf(a, b.w, acc[m].w);
+        for (int m4 = 0; m4 < MMAX / 4; ++m4) {
+          const float4 a4 = *reinterpret_cast<const float4*>(&As[r][4 * m4]);   // one shared-memory read per four rows of A
+          const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int m = 4 * m4 + j;
+            acc[m].x = fmaf(av[j], b.x, acc[m].x); acc[m].y = fmaf(av[j], b.y, acc[m].y);
+            acc[m].z = fmaf(av[j], b.z, acc[m].z); acc[m].w = fmaf(av[j], b.w, acc[m].w);
+          }
         }
       }
     }
@@ -222,7 +227,7 @@ __global__ void __launch_bounds__(128, 4) gemm_thin_k_kernel(const ThinKParams p
   // that 8 independent 16-byte loads per thread are in flight (a store between two loads would
   // otherwise pin their order, since D may alias the inputs as far as the compiler knows).
   constexpr int RB = 64, RG = 8;
-  __shared__ float As[RB][KMAX];
+  __shared__ __align__(16) float As[RB][KMAX];         // (KMAX is a multiple of 4: a row is read back as 16-byte groups)
   const int n = (blockIdx.x * 128 + threadIdx.x) * 4;
   const bool n_ok = n < p.N;
   float4 b[KMAX];
@@ -257,10 +262,15 @@ __global__ void __launch_bounds__(128, 4) gemm_thin_k_kernel(const ThinKParams p
         const int m = mb + r0 + i;
         float4 acc = bz;
 #pragma unroll
-        for (int k = 0; k < KMAX; ++k) {
-          const float a = As[r0 + i][k];
-          acc.x = fmaf(a, b[k].x, acc.x); acc.y = fmaf(a, b[k].y, acc.y);
-          acc.z = fmaf(a, b[k].z, acc.z); acc.w = fmaf(a, b[k].w, acc.w);
+        for (int k4 = 0; k4 < KMAX / 4; ++k4) {
+          const float4 a4 = *reinterpret_cast<const float4*>(&As[r0 + i][4 * k4]);
+          const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int k = 4 * k4 + j;
+            acc.x = fmaf(av[j], b[k].x, acc.x); acc.y = fmaf(av[j], b[k].y, acc.y);
+            acc.z = fmaf(av[j], b[k].z, acc.z); acc.w = fmaf(av[j], b[k].w, acc.w);
+          }
         }
         float t[4] = {acc.x, acc.y, acc.z, acc.w};
         if (p.e.sigmoid) {
