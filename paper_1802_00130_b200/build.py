@@ -32,7 +32,9 @@ def build(force=False, verbose=False):
     if not force and not is_stale():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
-    cmd = [nvcc] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + SOURCES
+    # GN_NVTX=1: named ranges around the phases of the path for timeline tools (header-only NVTX, off by default)
+    extra = ["-DGN_NVTX"] if os.environ.get("GN_NVTX") == "1" else []
+    cmd = [nvcc] + FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + SOURCES
     res = subprocess.run(cmd, cwd=CSRC, capture_output=True, text=True)
     if verbose:
         sys.stderr.write(res.stderr)

@@ -11,6 +11,21 @@
 #include "../../include/gn.h"
 #include "gn_kernels.h"
 
+// Named ranges around the phases of the path (stored forward pass, f / gradient, products, CG solve) for timeline
+// tools; compiled in only with -DGN_NVTX (paper_1802_00130_b200/build.py: GN_NVTX=1 in the environment).
+#ifdef GN_NVTX
+#include <nvtx3/nvToolsExt.h>
+namespace {
+struct PhaseRange {
+  explicit PhaseRange(const char* name) { nvtxRangePushA(name); }
+  ~PhaseRange() { nvtxRangePop(); }
+};
+}  // namespace
+#define GN_PHASE(name) PhaseRange gn_phase_range_(name)
+#else
+#define GN_PHASE(name) do { } while (0)
+#endif
+
 using namespace gn;
 
 struct gn_ctx {
@@ -664,6 +679,7 @@ gn_status layer_backward(gn_ctx* c, int m, const float* ds_w, int64_t w_rows, co
 
 // out = coef v + (1/|S|) J^T (2 J v) over the stored subsample (Eq. sampled-Gauss).
 gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
+  GN_PHASE("G v");
   SideJoin side_guard(c);
   ++c->parts_epoch;
   const int L = c->L;
@@ -773,6 +789,7 @@ bool stored_factors_applicable(const gn_ctx* c) {
 // (Eqs. communi-jaco, ztox-jaco, Jelement-store).  Done once per (theta, S).
 gn_status ensure_factors(gn_ctx* c) {
   if (c->factors_valid) return GN_OK;
+  GN_PHASE("Jacobian factors");
   ++c->parts_epoch;
   const int L = c->L, nL = c->w[L];
   const int64_t nS = c->nS;
@@ -916,6 +933,7 @@ gn_status product_split(gn_ctx* c, const float* v, float* out, float coef) {
 constexpr int kFactorBreakEven = 8;
 
 gn_status product_blockdiag_any(gn_ctx* c, const float* v, float* out, float coef) {
+  GN_PHASE("block-diagonal G v");
   if (c->has_split) return product_split(c, v, out, coef);
   bool stored = c->bd_method == 2;
   if (c->bd_method == 0 && stored_factors_applicable(c))
@@ -942,6 +960,7 @@ gn_status ensure_batch(gn_ctx* c) {
 
 // f and (optionally) the gradient over all rows in row batches (Section 6.1 in its one-GPU form).
 gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
+  GN_PHASE("f / gradient");
   GN_TRY(ensure_batch(c));
   const int L = c->L;
   const int64_t Rb = c->capB;
@@ -1262,6 +1281,7 @@ gn_status gn_set_theta_host(gn_ctx* c, const float* h_theta) {
 }
 
 static gn_status set_subsample_impl(gn_ctx* c, const int32_t* idx, int64_t nS, cudaMemcpyKind kind) {
+  GN_PHASE("set_subsample");
   if (!c) return GN_EINVAL;
   if (!idx) return fail(c, GN_EINVAL, "idx is NULL");
   if (nS < 1) return fail(c, GN_EINVAL, "the subsample must have at least one row");
@@ -1375,6 +1395,7 @@ gn_status gn_Gv_blockdiag_host(gn_ctx* c, const float* h_v, float* h_out) { retu
 
 gn_status gn_cg_solve(gn_ctx* c, const float* d_g, double lambda, int blockdiag, int max_iter, double tol,
                       float* d_d, int* iters_host, float* d_iterates, double* resnorm_host) {
+  GN_PHASE("CG solve");
   if (!c) return GN_EINVAL;
   if (!d_g || !d_d) return fail(c, GN_EINVAL, "g / d is NULL");
   if (max_iter < 1) return fail(c, GN_EINVAL, "max_iter must be >= 1");
