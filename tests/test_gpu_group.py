@@ -126,3 +126,29 @@ def test_replayed_cg_step_gives_the_bits_of_plain_launches(name, mode):
     d_ref, _, _ = orc.cg_solve(p["theta"], p["widths"], p["C"], XS, g.cpu().numpy(), 1.0, False, 9, 0.0)
     tol = 1e-4 if mode == "fp32" else 2e-2
     assert np.linalg.norm(runs[1][0][0].cpu().numpy() - d_ref) <= tol * np.linalg.norm(d_ref)
+
+
+def test_a_context_on_the_callers_own_stream_gives_the_same_bits():
+    """Everything is enqueued on the stream given to gn_create (here a non-default stream of the caller's; the other
+    tests leave it to the context to make one): products, gradient and a graph-replayed CG solve, bit for bit."""
+    import torch
+    import paper_1802_00130_b200 as gn
+    p = wl.make("mid")
+    X, Y, th, idx, v = dev(p["X"]), dev(p["Y"]), dev(p["theta"]), dev(p["idx"]), dev(p["v"])
+    g = dev(orc.grad(p["theta"], p["widths"], p["C"], p["X"], p["Y"]).astype(np.float32))
+    torch.cuda.synchronize()
+    outs = []
+    for own in (False, True):
+        stream = torch.cuda.Stream() if own else None
+        ctx = gn.GnContext(p["widths"], p["C"], X, Y, gn.GN_TF32, stream=stream)
+        ctx.set_theta(th)
+        ctx.set_subsample(idx)
+        res = [ctx.Gv(v), ctx.Gv_blockdiag(v), ctx.grad()]
+        d, its, resn = ctx.cg_solve(g, 1.0, blockdiag=False, max_iter=8, tol=0.0)
+        assert its == 8 and ctx.graph_replays == 7
+        res.append(d)
+        torch.cuda.synchronize()
+        outs.append([r.clone() for r in res] + [torch.from_numpy(resn)])
+        ctx.close()
+    for a, b in zip(*outs):
+        assert torch.equal(a.cpu(), b.cpu())
