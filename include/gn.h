@@ -302,6 +302,16 @@ gn_status gn_newton_iter(gn_ctx* ctx, float* d_theta, const int32_t* d_idx, int6
 gn_status gn_debug_timeout_probe(gn_ctx* ctx, double limit_ms);
 
 /*
+ * gn_debug_check_canaries - every device allocation of the context ends in 256 bytes of slack, the last 128 of
+ * which are set to a guard pattern when the allocation is made and are never part of any operand.  This call
+ * synchronises, reads the guard bytes of every live allocation back and returns GN_ECUDA (with the size of the
+ * damaged workspace in gn_last_error) if any of them has changed, i.e. if some kernel wrote past the end of a
+ * workspace; *n_checked (optional) receives the number of allocations looked at.  A stand-in, for writes past
+ * the end, for a memory checker where none can be run.
+ */
+gn_status gn_debug_check_canaries(gn_ctx* ctx, int64_t* n_checked);
+
+/*
  * gn_debug_activations - copy the stored Z_m (m in 1..L, [|S|][n_m]) of the current subsample to a
  * device buffer; a test hook for the stored forward pass (Eq. xtoz).
  */

@@ -44,6 +44,7 @@ _SIGNATURES = {
     "gn_newton_iter": (_i32, [_vp, _vp, _vp, _i64, _vp, _vp, _vp]),
     "gn_debug_timeout_probe": (_i32, [_vp, _dbl]),
     "gn_debug_option": (_i32, [_vp, _i32, _i32]),
+    "gn_debug_check_canaries": (_i32, [_vp, C.POINTER(_i64)]),
     "gn_profile": (_i32, [_vp, _i32]),
     "gn_profile_read": (_i32, [_vp, C.POINTER(_dbl), C.POINTER(_dbl), C.POINTER(_i64)]),
     "gn_thin_m_gemm_noalloc": (_i32, [_i32, _i32, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp, C.c_char_p, _i64]),
@@ -343,6 +344,12 @@ class GnContext:
     def debug_option(self, option, value):
         """Test hook: switch a launch strategy (0 = grouped launches, 1 = K slices of left-over tiles)."""
         self._check(self._lib.gn_debug_option(self._h, int(option), int(value)))
+
+    def debug_check_canaries(self):
+        """Test hook: raises GnError if a kernel wrote past the end of a workspace; returns the allocations checked."""
+        n = _i64()
+        self._check(self._lib.gn_debug_check_canaries(self._h, C.byref(n)))
+        return int(n.value)
 
     def debug_activations(self, m):
         import torch

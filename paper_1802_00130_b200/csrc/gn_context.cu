@@ -175,6 +175,8 @@ gn_status cuda_fail(gn_ctx* c, cudaError_t e, const char* where) {
     if (s__ != GN_OK) return s__;         \
   } while (0)
 
+constexpr int kCanaryByte = 0xA5;
+
 template <class T>
 gn_status dev_alloc(gn_ctx* c, T** p, int64_t count) {
   *p = nullptr;
@@ -188,6 +190,12 @@ gn_status dev_alloc(gn_ctx* c, T** p, int64_t count) {
   if (e != cudaSuccess) {
     cudaGetLastError();
     return fail(c, GN_ENOMEM, std::string("cudaMalloc of ") + std::to_string(count * (int64_t)sizeof(T)) + " bytes: " + cudaGetErrorString(e));
+  }
+  // the last 128 bytes of the slack are a canary: nothing of the library may write there (gn_debug_check_canaries)
+  if (cudaMemset(static_cast<char*>(q) + (size_t)count * sizeof(T) + 128, kCanaryByte, 128) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(q);
+    return fail(c, GN_ECUDA, "cudaMemset of a fresh allocation failed");
   }
   c->bytes += count * (int64_t)sizeof(T);
   ++c->alloc_gen;
@@ -1667,6 +1675,25 @@ gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   if (option == 0) c->group_enabled = value != 0;
   else if (option == 1) c->sk_enabled = value != 0 && c->sk_enabled;
   else return fail(c, GN_EINVAL, "unknown option");
+  return GN_OK;
+}
+
+gn_status gn_debug_check_canaries(gn_ctx* c, int64_t* n_checked) {
+  if (!c) return GN_EINVAL;
+  GN_TRY(sync(c, "canary check"));
+  if (c->st2) cudaStreamSynchronize(c->st2);
+  unsigned char host[128];
+  int64_t checked = 0;
+  for (const auto& o : c->owned) {
+    if (!o.p) continue;
+    GN_CUDA(c, cudaMemcpy(host, static_cast<const char*>(o.p) + o.bytes + 128, 128, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < 128; ++i)
+      if (host[i] != kCanaryByte)
+        return fail(c, GN_ECUDA, "the guard bytes after a workspace of " + std::to_string(o.bytes) + " bytes were overwritten (offset " +
+                                     std::to_string(i) + " past its slack)");
+    ++checked;
+  }
+  if (n_checked) *n_checked = checked;
   return GN_OK;
 }
 

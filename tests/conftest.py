@@ -24,3 +24,22 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def guard_bytes_checked_when_a_context_closes(request, monkeypatch):
+    """Every GPU test that closes a context first has the library read back the guard bytes behind each of its
+    workspaces (gn_debug_check_canaries): a kernel that wrote past the end of one fails the test that ran it."""
+    if "gpu" not in request.keywords:
+        yield
+        return
+    import paper_1802_00130_b200 as gn
+    plain_close = gn.GnContext.close
+
+    def close(self):
+        if getattr(self, "_h", None):
+            assert self.debug_check_canaries() > 0
+        plain_close(self)
+
+    monkeypatch.setattr(gn.GnContext, "close", close)
+    yield
