@@ -302,6 +302,17 @@ gn_status gn_newton_iter(gn_ctx* ctx, float* d_theta, const int32_t* d_idx, int6
 gn_status gn_debug_timeout_probe(gn_ctx* ctx, double limit_ms);
 
 /*
+ * gn_debug_plan_group - the work list a grouped (or chained, keep_order != 0) launch of the CTA-pair kernel would use
+ * for n <= 5 contractions of shapes M[i] x N[i] x K[i] on `pairs` (1..80) CTA pairs; host arithmetic only, no device
+ * and no context needed.  Outputs, per problem k in LAUNCH order: order[k] = its index in the caller's list, tiles[k] =
+ * its 256-row tiles, waves[k] = how many whole waves of them every pair runs (tiles q, q + pairs, ...), and
+ * counts[k * pairs + q] = tiles of it that pair q runs in all (host arrays of n, n, n and n * pairs entries).
+ * Returns the number of pairs the launch would use, or -1 for bad arguments.
+ */
+int32_t gn_debug_plan_group(int32_t n, const int32_t* M, const int32_t* N, const int32_t* K, int32_t pairs,
+                            int32_t keep_order, int32_t* counts, int32_t* waves, int32_t* order, int32_t* tiles);
+
+/*
  * gn_debug_check_canaries - every device allocation of the context ends in 256 bytes of slack, the last 128 of
  * which are set to a guard pattern when the allocation is made and are never part of any operand.  This call
  * synchronises, reads the guard bytes of every live allocation back and returns GN_ECUDA (with the size of the

@@ -45,6 +45,8 @@ _SIGNATURES = {
     "gn_debug_timeout_probe": (_i32, [_vp, _dbl]),
     "gn_debug_option": (_i32, [_vp, _i32, _i32]),
     "gn_debug_check_canaries": (_i32, [_vp, C.POINTER(_i64)]),
+    "gn_debug_plan_group": (_i32, [_i32, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32), _i32, _i32, C.POINTER(_i32),
+                                   C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
     "gn_profile": (_i32, [_vp, _i32]),
     "gn_profile_read": (_i32, [_vp, C.POINTER(_dbl), C.POINTER(_dbl), C.POINTER(_i64)]),
     "gn_thin_m_gemm_noalloc": (_i32, [_i32, _i32, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp, C.c_char_p, _i64]),
@@ -117,6 +119,20 @@ def _host_ptr(a, dtype, count=None):
     if count is not None and a.size != count:
         raise ValueError(f"expected {count} elements, got {a.size}")
     return _vp(a.ctypes.data)
+
+
+def plan_group(shapes, pairs=74, keep_order=False):
+    """Work list of a grouped launch for [(M, N, K), ...] (host arithmetic of the library, no device needed):
+    returns (pairs_used, order, tiles, waves, counts) with counts[k][q] = tiles of the k-th problem in launch order
+    that pair q runs."""
+    n = len(shapes)
+    arr = lambda xs: (C.c_int32 * len(xs))(*[int(x) for x in xs])
+    M, N, K = arr([s[0] for s in shapes]), arr([s[1] for s in shapes]), arr([s[2] for s in shapes])
+    counts, waves, order, tiles = (C.c_int32 * (n * pairs))(), (C.c_int32 * n)(), (C.c_int32 * n)(), (C.c_int32 * n)()
+    used = lib().gn_debug_plan_group(n, M, N, K, int(pairs), int(bool(keep_order)), counts, waves, order, tiles)
+    if used < 0:
+        raise ValueError("bad shapes / pair count")
+    return used, list(order), list(tiles), list(waves), [list(counts[k * pairs:(k + 1) * pairs]) for k in range(n)]
 
 
 def thin_m_gemm_noalloc(A, B, out, stream=None):

@@ -1531,6 +1531,49 @@ int launch_gemm_tf32_group(const GemmArgs* gs, int n, const int* dep_prob, const
   return 1;
 }
 
+// Host-only view of the work list a grouped launch would use (no device needed): for problems of the given shapes
+// on `pairs` CTA pairs, counts[k * pairs + q] = tiles of the k-th problem IN LAUNCH ORDER that pair q runs,
+// waves[k] = how many of them are whole waves (tiles q, q + pairs, ...), order[k] = index of that problem in the
+// caller's list, tiles[k] = its tile count.  keep_order != 0 keeps the caller's order (a chain).  Returns the number
+// of pairs the launch would use, or -1 for bad arguments.
+int gemm_tf32_plan_group(int n, const int* M, const int* N, const int* K, int pairs, int keep_order, int* counts,
+                         int* waves, int* order_out, int* tiles_out) {
+  if (n < 1 || n > MAX_GROUP || pairs < 1 || pairs > MAX_PAIRS_LAUNCH) return -1;
+  GroupParams gp = {};
+  struct Item { int src; double cost; };
+  Item order[MAX_GROUP];
+  Tf32Params tmp[MAX_GROUP];
+  long long total_tiles = 0;
+  for (int i = 0; i < n; ++i) {
+    if (M[i] < 1 || N[i] < 1 || K[i] < 1) return -1;
+    const int bn = choose_bn2(M[i], N[i], true);
+    tmp[i] = Tf32Params{};
+    tmp[i].bn = bn;
+    tmp[i].kblocks[0] = (K[i] + BK - 1) / BK;
+    tmp[i].tiles_n = (N[i] + bn - 1) / bn;
+    tmp[i].tiles = ((M[i] + 2 * BM - 1) / (2 * BM)) * tmp[i].tiles_n;
+    order[i].src = i;
+    order[i].cost = tile_cost(tmp[i]);
+    total_tiles += tmp[i].tiles;
+  }
+  if (!keep_order)
+    for (int i = 1; i < n; ++i)
+      for (int j = i; j > 0 && order[j].cost > order[j - 1].cost; --j) { Item t = order[j]; order[j] = order[j - 1]; order[j - 1] = t; }
+  const int P = total_tiles < pairs ? (int)total_tiles : pairs;
+  double load[MAX_PAIRS_LAUNCH];
+  for (int q = 0; q < P; ++q) load[q] = 0.0;
+  for (int k = 0; k < n; ++k) {
+    gp.pr[k] = tmp[order[k].src];
+    deal_tiles(gp, k, order[k].cost, P, load);
+    waves[k] = gp.pr[k].waves;
+    order_out[k] = order[k].src;
+    tiles_out[k] = gp.pr[k].tiles;
+    for (int q = 0; q < pairs; ++q)
+      counts[k * pairs + q] = q < P ? gp.pr[k].waves + (gp.rstart[k][q + 1] - gp.rstart[k][q]) : 0;
+  }
+  return P;
+}
+
 // ---- error-compensated form ---------------------------------------------------------------------
 // 4 k-blocks = 128 terms (384 products) per accumulation in tensor memory: the truncation bias of one chunk stays
 // below 1e-6 relative (measured), and the running sums outside are round-to-nearest.

@@ -1678,6 +1678,12 @@ gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   return GN_OK;
 }
 
+int32_t gn_debug_plan_group(int32_t n, const int32_t* M, const int32_t* N, const int32_t* K, int32_t pairs, int32_t keep_order,
+                            int32_t* counts, int32_t* waves, int32_t* order, int32_t* tiles) {
+  if (!M || !N || !K || !counts || !waves || !order || !tiles) return -1;
+  return gemm_tf32_plan_group(n, M, N, K, pairs, keep_order, counts, waves, order, tiles);
+}
+
 gn_status gn_debug_check_canaries(gn_ctx* c, int64_t* n_checked) {
   if (!c) return GN_EINVAL;
   GN_TRY(sync(c, "canary check"));

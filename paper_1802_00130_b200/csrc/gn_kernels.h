@@ -79,6 +79,10 @@ bool gemm_tf32_group_eligible(const GemmArgs* gs, int n);
 int launch_gemm_tf32_group(const GemmArgs* gs, int n, const int* dep_prob, const int* dep_all, int* done,
                            int done_stride, int* err_flag, cudaStream_t st);
 
+// The work list of such a launch, computed without a device (see gemm_tf32.cu); for tests of the host logic.
+int gemm_tf32_plan_group(int n, const int* M, const int* N, const int* K, int pairs, int keep_order, int* counts,
+                         int* waves, int* order_out, int* tiles_out);
+
 // Streaming FP32 kernels for contractions with one dimension <= 16 (the n_L-wide output layer).
 // gemm_thin_kind says which of them (if any) takes a problem; THIN_M needs a scratch buffer of
 // gemm_thin_scratch_floats(g) floats.  launch_gemm_thin returns the launches made (0 = not taken).
