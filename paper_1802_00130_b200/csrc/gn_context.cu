@@ -451,8 +451,10 @@ void run_gemm(gn_ctx* c, const GemmArgs& g, cudaStream_t st = nullptr) {
   ++c->gemm_seq;
   const ThinKind thin = gemm_thin_kind(g);
   // In TF32 mode the n_L-wide forward products go to the tensor-core kernel as one 32- or 64-column
-  // tile: TMA streams A about 2.5x faster than the SIMT streaming kernel does (measured).
-  const bool thin_n_on_tensor = thin == THIN_N && c->prec == GN_TF32 && gemm_tf32_eligible(g);
+  // tile: TMA streams A about 2.5x faster than the SIMT streaming kernel does (measured) - once there are enough
+  // 128-row tiles to occupy the SMs; below 48 tiles (a CTA walks its whole K range alone, 53 us at K = 4000 whatever
+  // the row count) the streaming kernel, one warp per four rows, is the faster one (3000 rows: 3-4 % of a product).
+  const bool thin_n_on_tensor = thin == THIN_N && c->prec == GN_TF32 && gemm_tf32_eligible(g) && g.M >= 48 * 128;
   if (thin != THIN_NONE && !thin_n_on_tensor) {
     const int64_t need = gemm_thin_scratch_floats(g);
     if (need > c->thin_cap) {
