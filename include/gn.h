@@ -303,7 +303,7 @@ gn_status gn_debug_timeout_probe(gn_ctx* ctx, double limit_ms);
 
 /*
  * gn_debug_plan_group - the work list a grouped (or chained, keep_order != 0) launch of the CTA-pair kernel would use
- * for n <= 5 contractions of shapes M[i] x N[i] x K[i] on `pairs` (1..80) CTA pairs; host arithmetic only, no device
+ * for n <= 6 contractions of shapes M[i] x N[i] x K[i] on `pairs` (1..80) CTA pairs; host arithmetic only, no device
  * and no context needed.  Outputs, per problem k in LAUNCH order: order[k] = its index in the caller's list, tiles[k] =
  * its 256-row tiles, waves[k] = how many whole waves of them every pair runs (tiles q, q + pairs, ...), and
  * counts[k * pairs + q] = tiles of it that pair q runs in all (host arrays of n, n, n and n * pairs entries).
@@ -367,7 +367,9 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
  * layers of a pass as one launch whose tiles wait for the tiles they read (value 0 = one launch per layer, 1 = the
  * stored forward pass, the default, 2 = also the forward R pass of a product).  Option 5 (GN_FP32_ACCURATE contexts): the error-compensated kernel also writes the hi / lo parts
  * of a result that a later contraction takes as an operand (value 0 = a separate pass splits it).  Option 6: fixed-length
- * CG solves of small problems replay one captured step as a CUDA graph (value 0 = plain launches).  Results do not
+ * CG solves of small problems replay one captured step as a CUDA graph (value 0 = plain launches).  Option 7: the
+ * weight blocks of the stored-factor block product as two chained halves of the subsample's rows (value 0 = one
+ * contraction per block; the two forms differ in the order of two partial sums, i.e. by rounding).  Results do not
  * depend on options 0, 3, 4, 5 and 6 (tiles, sums and parts are computed identically); GN_EINVAL for an unknown option.
  */
 gn_status gn_debug_option(gn_ctx* ctx, int option, int value);

@@ -65,7 +65,7 @@ struct Tf32Params {
 // its tiles of the problem's whole waves (q, q + P, ...) and then tiles rstart[g][q] .. rstart[g][q + 1] - 1 of the
 // tiles left over after those waves; the host deals the left-over tiles so that the pairs' total loads come out even
 // (longest tiles first), which lets the short tiles of one problem fill the partial last wave of another.
-constexpr int MAX_GROUP = 5;
+constexpr int MAX_GROUP = 6;
 constexpr int MAX_PAIRS_LAUNCH = 80;        // >= SMs / 2
 struct GroupParams {
   int n_prob;
@@ -779,7 +779,8 @@ gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constan
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                   zc[h][4 * e + j] = zrow ? __ldg(reinterpret_cast<const float2*>(zrow + 8 * j)) : make_float2(0.f, 0.f);
-                  ci[h][4 * e + j] = crow ? __ldg(reinterpret_cast<const float2*>(crow + 8 * j)) : make_float2(0.f, 0.f);
+                  // (L2-coherent read: in a chained launch this operand may have been written by another pair of this very launch)
+                  ci[h][4 * e + j] = crow ? __ldcg(reinterpret_cast<const float2*>(crow + 8 * j)) : make_float2(0.f, 0.f);
                 }
               }
           }
@@ -847,7 +848,7 @@ gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constan
                       if (sigm) x = 1.f / (1.f + __expf(-x));
                       if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
                       x *= alpha;
-                      if (crow) x = fmaf(beta, __ldg(crow + n), x);
+                      if (crow) x = fmaf(beta, __ldcg(crow + n), x);
                       drow[n] = x;
                     }
                   }

@@ -86,6 +86,7 @@ struct gn_ctx {
   // pass (where it measured 8 % faster), 2 also the forward R pass of a product (where cutting left-over tiles along K,
   // which a chained launch does not do, measured as fast or faster)
   int chain_level = 1;
+  bool split_k_enabled = true; // weight blocks of the stored-factor product as two chained halves of the rows
   int* chain_ctr = nullptr; int64_t chain_ctr_cap = 0;   // finished-tile counters of such a launch
   // FP32-accurate mode on the tensor cores (3 x TF32): hi / lo parts of the operands
   int acc_method = 0;        // 0 choose (tensor cores where the shape allows), 1 FP32 FMA only, 2 as 0
@@ -852,13 +853,37 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
   // 2. q_i = D_i^T 2 D_i u_i per sample (Eqs. direct-JV-cost, JTv)
   for (int m = 1; m < L; ++m)
     c->launches += launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], 1, 1, 0, c->DS[m], c->st);
-  // 3. the weight and bias blocks
-  for (int m0 = 1; m0 <= L; m0 += kGroup) {
-    GemmArgs gs[kGroup];
+  // 3. the weight and bias blocks.  The weight blocks are few long tiles (64 of 375 k-blocks per 2000 x 2000 layer at
+  // |S| = 12000: 160 tiles on 74 pairs for three layers leave a third of the last round idle), so with a long enough
+  // K each block is cut into its two halves of the rows: the first half writes alpha Z^T Q + beta v, the second adds
+  // its alpha Z^T Q to that (a chained launch: a second-half tile waits for the first-half tiles of its row panel).
+  // Twice as many tiles of half the length fill the rounds better; the order of the two partial sums is fixed.
+  const bool halves = c->prec == GN_TF32 && c->chain_level >= 1 && c->split_k_enabled && nS >= 4096 && L - 1 >= 1 && L - 1 <= kGroup;
+  if (halves) {
+    GemmArgs gs[2 * kGroup];
+    int dep[2 * kGroup], dep_all[2 * kGroup];
     int n = 0;
-    for (int m = m0; m <= L && m < m0 + kGroup; ++m)
-      gs[n++] = weight_block_args(c, m, m < L ? c->DS[m] : c->RZ[m], c->Z[m - 1], nS, inv, v, coef, out);
-    run_gemm_group(c, gs, n);
+    const int64_t h0 = (nS / 2 + 31) / 32 * 32;              // first half: a whole number of k-blocks
+    const int nl = L - 1;                                     // the hidden layers' blocks (the n_L-row block is a streaming kernel)
+    for (int part = 0; part < 2; ++part)
+      for (int m = 1; m <= nl; ++m) {
+        const int64_t r0 = part == 0 ? 0 : h0, rows = part == 0 ? h0 : nS - h0;
+        GemmArgs g = weight_block_args(c, m, c->DS[m] + r0 * c->w[m], c->Z[m - 1] + r0 * c->w[m - 1], rows, inv,
+                                       part == 0 ? v : out, part == 0 ? coef : 1.f, out);
+        dep[n] = part == 0 ? -1 : m - 1;                      // the first-half problem of the same layer
+        dep_all[n] = 0;
+        gs[n++] = g;
+      }
+    run_gemm_chain(c, gs, dep, dep_all, n);
+    run_gemm(c, weight_block_args(c, L, c->RZ[L], c->Z[L - 1], nS, inv, v, coef, out));
+  } else {
+    for (int m0 = 1; m0 <= L; m0 += kGroup) {
+      GemmArgs gs[kGroup];
+      int n = 0;
+      for (int m = m0; m <= L && m < m0 + kGroup; ++m)
+        gs[n++] = weight_block_args(c, m, m < L ? c->DS[m] : c->RZ[m], c->Z[m - 1], nS, inv, v, coef, out);
+      run_gemm_group(c, gs, n);
+    }
   }
   for (int m = 1; m <= L; ++m)
     GN_TRY(bias_block(c, m, m < L ? c->DS[m] : c->RZ[m], nS, inv, v, coef, out));
@@ -1671,6 +1696,7 @@ gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   if (!c) return GN_EINVAL;
   if (option == 2) { if (value < 0) return fail(c, GN_EINVAL, "count must be >= 0"); c->fail_alloc_in = value; return GN_OK; }
   if (option == 3) { quiesce(c); c->side_enabled = value != 0; return GN_OK; }
+  if (option == 7) { c->split_k_enabled = value != 0; return GN_OK; }
   if (option == 6) { c->graph_enabled = value != 0; return GN_OK; }
   if (option == 5) { c->parts_enabled = value != 0; return GN_OK; }
   if (option == 4) { c->chain_level = value < 0 ? 0 : (value > 2 ? 2 : value); return GN_OK; }

@@ -64,7 +64,7 @@ int launch_gemm_tf32x3(const GemmArgs& g, int* err_flag, cudaStream_t st);
 int64_t gemm_tf32_workspace_floats();
 int gemm_tf32_workspace_flags();
 int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_flags, cudaStream_t st);
-// Up to five problems, each suited to the CTA-pair kernel (M > 128, N >= 128), as ONE launch whose pairs walk a
+// Up to six problems, each suited to the CTA-pair kernel (M > 128, N >= 128), as ONE launch whose pairs walk a
 // common, host-balanced work list.  Whole tiles only.
 //   dep_prob == nullptr: independent problems, longest tiles first; the tiles of one fill the partial last wave
 //   of another.
@@ -74,7 +74,7 @@ int launch_gemm_tf32(const GemmArgs& g, int* err_flag, float* sk_ws, int* sk_fla
 //   of each draining the GPU.  `done`: device scratch of n * done_stride ints (done_stride > M / 256 + 1),
 //   cleared by the call.
 // Returns launches made, or -1 if the group cannot run this way (run the problems one by one, in order).
-constexpr int kGemmGroupMax = 5;
+constexpr int kGemmGroupMax = 6;
 bool gemm_tf32_group_eligible(const GemmArgs* gs, int n);
 int launch_gemm_tf32_group(const GemmArgs* gs, int n, const int* dep_prob, const int* dep_all, int* done,
                            int done_stride, int* err_flag, cudaStream_t st);

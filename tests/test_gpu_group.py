@@ -152,3 +152,29 @@ def test_a_context_on_the_callers_own_stream_gives_the_same_bits():
         ctx.close()
     for a, b in zip(*outs):
         assert torch.equal(a.cpu(), b.cpu())
+
+
+def test_weight_blocks_of_the_stored_factor_product_in_two_chained_halves():
+    """From 4096 subsample rows on, TF32 mode cuts every hidden-layer weight block of the stored-factor product into
+    the two halves of the rows; the second half adds onto the first inside one chained launch.  Same result as the
+    uncut blocks up to the order of two partial sums, deterministic, and within the mode's bound of the checker."""
+    import torch
+    p = wl.make_custom([300, 520, 392, 264, 10], l=5200, nS=5000, C=52.0, seed=47, x="sparse80")
+    XS = p["X"][p["idx"]]
+    ref = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], XS, p["v"])
+    outs = {}
+    for cut in (1, 0):
+        ctx = make_ctx(p, "tf32")
+        ctx.debug_option(7, cut)
+        ctx.set_blockdiag_method(2)
+        ctx.set_subsample(dev(p["idx"]))
+        a = ctx.Gv_blockdiag(dev(p["v"])).clone()
+        b = ctx.Gv_blockdiag(dev(p["v"])).clone()
+        assert torch.equal(a, b)                              # deterministic
+        outs[cut] = (a.cpu().numpy(), ctx.kernel_launches)
+        assert relb(outs[cut][0], ref, p["widths"]) <= TOL["tf32"]
+        ctx.close()
+    assert not np.array_equal(outs[1][0], outs[0][0])          # the cut form did run (another order of sums)
+    # ... and differs by rounding only: the tensor core adds into its FP32 accumulator with truncation (a relative bias
+    # of about 1e-9 per term), so one accumulation over 5000 rows and two over 2500 differ by about 1e-5
+    assert relb(outs[1][0], outs[0][0], p["widths"]) <= 1e-4

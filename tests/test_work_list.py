@@ -57,6 +57,6 @@ def test_bad_arguments_are_refused():
     with pytest.raises(ValueError):
         gn.plan_group([(0, 10, 10)])
     with pytest.raises(ValueError):
-        gn.plan_group([(256, 256, 256)] * 6)                 # more problems than a launch takes
+        gn.plan_group([(256, 256, 256)] * 7)                 # more problems than a launch takes
     with pytest.raises(ValueError):
         gn.plan_group([(256, 256, 256)], pairs=81)
