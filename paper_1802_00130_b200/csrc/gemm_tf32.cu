@@ -541,6 +541,104 @@ __device__ __forceinline__ bool next_work(const GroupParams& gp, int pair, int i
   return false;
 }
 
+// Epilogue of one whole, 16-byte-aligned 32 x 32 chunk of a warp's quadrant in the fragment layout of
+// tmem_ld_16x256b_x4: value v[4j + 2e + i] of half h is element (row 16h + 8e + lane / 4, column 8j + 2 (lane % 4) + i).
+// The epilogue warps are few (two per scheduler) and run beside the main loop, so what bounds them is their own
+// instruction stream, not the memory system: the same chunk took 10.7 us with every option tested per element
+// and 3.6 us as a plain store.  MODE fixes the options at compile time: 0 = alpha * acc (+ bias), 1 = sigmoid,
+// 2 = times the sigmoid derivative of `dsig`, 3 = plus beta * cin; 4 = any combination, tested at run time (its operands
+// are read where they are used, so that it needs no more registers than the others: the kernel is at its limit
+// of 168 and a spill here would be paid by every mode).
+struct EpiArgs {
+  const float* dsig; const float* cin; const float* bias; float* D;
+  long long ldd, ld_dsig, ld_cin;
+  int dsig_rows, dsig_div;   // row m of the tile reads row (m / dsig_div) % dsig_rows of dsig ...
+  int dsig_direct;           // ... which is m itself when dsig_div == 1 and dsig_rows >= M (no division per row)
+  float alpha, beta;
+  int M, sigm;
+};
+
+__device__ __forceinline__ long long dsig_row(const EpiArgs& a, int m) {
+  return a.dsig_direct ? m : (m / a.dsig_div) % a.dsig_rows;
+}
+
+template <int MODE>
+__device__ __forceinline__ void epilogue_full_chunk(const EpiArgs& a, uint32_t taddr, int mq, int nb, int lane,
+                                                    const float* ws, int slices) {
+  const bool use_sigm = MODE == 4 ? a.sigm != 0 : MODE == 1;
+  const bool use_dsig = MODE == 4 ? a.dsig != nullptr : MODE == 2;
+  const bool use_cin = MODE == 4 ? a.cin != nullptr : MODE == 3;
+  float2 op[2][8];                             // [h][4e + j]: the chunk of dsig (mode 2) or of cin (mode 3)
+  if (MODE == 2 || MODE == 3) {                // all global reads of the chunk in flight before anything waits
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int m = mq + 16 * h + 8 * e;
+        const float* row = nullptr;
+        if (m < a.M) row = MODE == 3 ? a.cin + (long long)m * a.ld_cin + nb
+                                     : a.dsig + dsig_row(a, m) * a.ld_dsig + nb;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float2 x = make_float2(0.f, 0.f);
+          // (cin: L2-coherent read, in a chained launch it may have been written by another pair of this very launch)
+          if (row) x = MODE == 3 ? __ldcg(reinterpret_cast<const float2*>(row + 8 * j)) : __ldg(reinterpret_cast<const float2*>(row + 8 * j));
+          op[h][4 * e + j] = x;
+        }
+      }
+  }
+  float2 bz[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) bz[j] = a.bias ? __ldg(reinterpret_cast<const float2*>(a.bias + nb + 8 * j)) : make_float2(0.f, 0.f);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {                // one 16-row half of the chunk at a time (16 accumulator registers live)
+    float v[16];
+    if (slices == 0) {
+      tmem_ld_16x256b_x4(taddr + ((uint32_t)(16 * h) << 16), v);
+      tmem_ld_wait();
+    } else {                                   // a tile cut along K: sum of the slices' partials, slice 0 first
+#pragma unroll
+      for (int i = 0; i < 16; ++i) v[i] = 0.f;
+      for (int s2 = 0; s2 < slices; ++s2) {
+        const float* wsr = ws + (long long)s2 * (2 * BM * BN_MAX) + (16 * h) * BN_MAX;
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float2 x = __ldcg(reinterpret_cast<const float2*>(wsr + (8 * e) * BN_MAX + 8 * j));
+            v[4 * j + 2 * e] += x.x; v[4 * j + 2 * e + 1] += x.y;
+          }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int m = mq + 16 * h + 8 * e;
+      if (m >= a.M) continue;
+      float* drow = a.D + (long long)m * a.ldd + nb;
+      const float* crow = (MODE == 4 && use_cin) ? a.cin + (long long)m * a.ld_cin + nb : nullptr;
+      const float* zrow = (MODE == 4 && use_dsig) ? a.dsig + dsig_row(a, m) * a.ld_dsig + nb : nullptr;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float x0 = v[4 * j + 2 * e] + bz[j].x, x1 = v[4 * j + 2 * e + 1] + bz[j].y;
+        if (use_sigm) { x0 = 1.f / (1.f + __expf(-x0)); x1 = 1.f / (1.f + __expf(-x1)); }
+        if (use_dsig) {
+          const float2 z = MODE == 4 ? __ldg(reinterpret_cast<const float2*>(zrow + 8 * j)) : op[h][4 * e + j];
+          x0 *= z.x * (1.f - z.x); x1 *= z.y * (1.f - z.y);
+        }
+        x0 *= a.alpha; x1 *= a.alpha;
+        if (MODE == 3) {
+          const float2 cc = op[h][4 * e + j];
+          x0 = fmaf(a.beta, cc.x, x0); x1 = fmaf(a.beta, cc.y, x1);
+        } else if (MODE == 4 && use_cin) {
+          const float2 cc = __ldcg(reinterpret_cast<const float2*>(crow + 8 * j));
+          x0 = fmaf(a.beta, cc.x, x0); x1 = fmaf(a.beta, cc.y, x1);
+        }
+        *reinterpret_cast<float2*>(drow + 8 * j) = make_float2(x0, x1);
+      }
+    }
+  }
+}
+
 constexpr int B2_STAGE_MAX = (BN_MAX / 2) * BK * 4;          // 16 KB: this CTA's half of the B tile
 constexpr int STAGE2_BYTES = A_STAGE_BYTES + B2_STAGE_MAX;   // 32 KB
 
@@ -751,108 +849,77 @@ gemm_tf32_2cta_kernel(const __grid_constant__ GroupMaps gm, const __grid_constan
       }
       {
         const int mq = m0 + quad * 32 + rsub;                    // this thread's rows are mq + 16h + 8e
-        const float* const dsig = p.dsig;
-        const float* const cin = p.cin;
-        const float* const bias = p.bias;
-        float* const D = p.D;
-        const long long ldd = p.ldd, ld_dsig = p.ld_dsig, ld_cin = p.ld_cin;
-        const int dsig_rows = p.dsig_rows, dsig_div = p.dsig_div;
-        const float alpha = p.alpha, beta = p.beta;
-        const int M = p.M, N = p.N, sigm = p.sigmoid, vec_epi = p.vec_epi;
+        EpiArgs ea;
+        ea.dsig = p.dsig; ea.cin = p.cin; ea.bias = p.bias; ea.D = p.D;
+        ea.ldd = p.ldd; ea.ld_dsig = p.ld_dsig; ea.ld_cin = p.ld_cin;
+        ea.dsig_rows = p.dsig_rows; ea.dsig_div = p.dsig_div;
+        ea.dsig_direct = p.dsig_div == 1 && p.dsig_rows >= p.M;
+        ea.alpha = p.alpha; ea.beta = p.beta; ea.M = p.M; ea.sigm = p.sigmoid;
+        const int N = p.N, vec_epi = p.vec_epi;
+        const int n_opt = (p.sigmoid ? 1 : 0) + (p.dsig ? 1 : 0) + (p.cin ? 1 : 0);
+        const int mode = n_opt == 0 ? 0 : n_opt > 1 ? 4 : p.sigmoid ? 1 : p.dsig ? 2 : 3;
         // whole tile: this warp's chunks are half, half + 2, ...; sliced tile: the pair's share of the
         // chunks is sl, sl + slices, ..., dealt alternately to the two warps of a quadrant
         const int c_first = w.sliced ? sl + half * p.slices : half;
         const int c_step = w.sliced ? 2 * p.slices : 2;
+        const int n_slices = w.sliced ? p.slices : 0;
+        const float* const ws0 = w.sliced ? p.sk_ws + (((long long)grp * 2 + rank) * BM + quad * 32 + rsub) * BN_MAX + csub : nullptr;
         for (int c = c_first; c < n_chunks; c += c_step) {
           const int nb = n0 + c * 32 + csub;                     // this thread's columns are nb + 8j, nb + 8j + 1
-          const bool fullc = vec_epi && n0 + c * 32 + 32 <= N;   // warp-uniform: whole chunk in range, 16-byte aligned rows
-          float2 zc[2][8], ci[2][8];                             // [h][4e + j]
-          if (fullc) {                        // all global reads of the chunk in flight before anything waits
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-              for (int e = 0; e < 2; ++e) {
-                const int m = mq + 16 * h + 8 * e;
-                const bool m_ok = m < M;
-                const float* zrow = (dsig && m_ok) ? dsig + (long long)((m / dsig_div) % dsig_rows) * ld_dsig + nb : nullptr;
-                const float* crow = (cin && m_ok) ? cin + (long long)m * ld_cin + nb : nullptr;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  zc[h][4 * e + j] = zrow ? __ldg(reinterpret_cast<const float2*>(zrow + 8 * j)) : make_float2(0.f, 0.f);
-                  // (L2-coherent read: in a chained launch this operand may have been written by another pair of this very launch)
-                  ci[h][4 * e + j] = crow ? __ldcg(reinterpret_cast<const float2*>(crow + 8 * j)) : make_float2(0.f, 0.f);
-                }
-              }
+          const uint32_t taddr = tq + (uint32_t)(c * 32);
+          if (vec_epi && n0 + c * 32 + 32 <= N) {                // warp-uniform: whole chunk in range, 16-byte aligned rows
+            const float* ws = ws0 + c * 32;
+            switch (mode) {
+              case 0: epilogue_full_chunk<0>(ea, taddr, mq, nb, lane, ws, n_slices); break;
+              case 1: epilogue_full_chunk<1>(ea, taddr, mq, nb, lane, ws, n_slices); break;
+              case 2: epilogue_full_chunk<2>(ea, taddr, mq, nb, lane, ws, n_slices); break;
+              case 3: epilogue_full_chunk<3>(ea, taddr, mq, nb, lane, ws, n_slices); break;
+              default: epilogue_full_chunk<4>(ea, taddr, mq, nb, lane, ws, n_slices); break;
+            }
+            continue;
           }
-          float2 bz[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            bz[j] = (bias && fullc) ? __ldg(reinterpret_cast<const float2*>(bias + nb + 8 * j)) : make_float2(0.f, 0.f);
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {         // one 16-row half of the chunk at a time (16 accumulator registers live)
+          // ragged or unaligned chunk: element by element
+#pragma unroll 1
+          for (int h = 0; h < 2; ++h) {
             float v[16];
             if (!w.sliced) {
-              tmem_ld_16x256b_x4(tq + ((uint32_t)(16 * h) << 16) + (uint32_t)(c * 32), v);
+              tmem_ld_16x256b_x4(taddr + ((uint32_t)(16 * h) << 16), v);
               tmem_ld_wait();
             } else {
-              // sum of the slices' partials, slice 0 first
 #pragma unroll
               for (int i = 0; i < 16; ++i) v[i] = 0.f;
-              for (int s2 = 0; s2 < p.slices; ++s2) {
-                const float* wsr = p.sk_ws + (((long long)(grp + s2) * 2 + rank) * BM + quad * 32 + rsub + 16 * h) * BN_MAX + csub + c * 32;
+              for (int s2 = 0; s2 < n_slices; ++s2) {
+                const float* wsr = ws0 + c * 32 + (long long)s2 * (2 * BM * BN_MAX) + (16 * h) * BN_MAX;
 #pragma unroll
                 for (int e = 0; e < 2; ++e)
 #pragma unroll
                   for (int j = 0; j < 4; ++j) {
-                    const float2 x = __ldcg(reinterpret_cast<const float2*>(wsr + (long long)(8 * e) * BN_MAX + 8 * j));
+                    const float2 x = __ldcg(reinterpret_cast<const float2*>(wsr + (8 * e) * BN_MAX + 8 * j));
                     v[4 * j + 2 * e] += x.x; v[4 * j + 2 * e + 1] += x.y;
                   }
               }
             }
-            if (fullc) {
 #pragma unroll
-              for (int e = 0; e < 2; ++e) {
-                const int m = mq + 16 * h + 8 * e;
-                if (m >= M) continue;
-                float* drow = D + (long long)m * ldd + nb;
+            for (int e = 0; e < 2; ++e) {
+              const int m = mq + 16 * h + 8 * e;
+              if (m >= ea.M) continue;
+              const float* zrow = ea.dsig ? ea.dsig + dsig_row(ea, m) * ea.ld_dsig : nullptr;
+              const float* crow = ea.cin ? ea.cin + (long long)m * ea.ld_cin : nullptr;
+              float* drow = ea.D + (long long)m * ea.ldd;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  float x[2] = {v[4 * j + 2 * e] + bz[j].x, v[4 * j + 2 * e + 1] + bz[j].y};
-                  const float z[2] = {zc[h][4 * e + j].x, zc[h][4 * e + j].y};
-                  const float cc[2] = {ci[h][4 * e + j].x, ci[h][4 * e + j].y};
+              for (int j = 0; j < 4; ++j)
 #pragma unroll
-                  for (int i = 0; i < 2; ++i) {
-                    if (sigm) x[i] = 1.f / (1.f + __expf(-x[i]));
-                    if (dsig) x[i] *= z[i] * (1.f - z[i]);
-                    x[i] *= alpha;
-                    if (cin) x[i] = fmaf(beta, cc[i], x[i]);
+                for (int i = 0; i < 2; ++i) {
+                  const int n = nb + 8 * j + i;
+                  if (n < N) {
+                    float x = v[4 * j + 2 * e + i] + (ea.bias ? __ldg(ea.bias + n) : 0.f);
+                    if (ea.sigm) x = 1.f / (1.f + __expf(-x));
+                    if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
+                    x *= ea.alpha;
+                    if (crow) x = fmaf(ea.beta, __ldcg(crow + n), x);
+                    drow[n] = x;
                   }
-                  *reinterpret_cast<float2*>(drow + 8 * j) = make_float2(x[0], x[1]);
                 }
-              }
-            } else {                             // ragged or unaligned chunk: element by element
-#pragma unroll
-              for (int e = 0; e < 2; ++e) {
-                const int m = mq + 16 * h + 8 * e;
-                if (m >= M) continue;
-                const float* zrow = dsig ? dsig + (long long)((m / dsig_div) % dsig_rows) * ld_dsig : nullptr;
-                const float* crow = cin ? cin + (long long)m * ld_cin : nullptr;
-                float* drow = D + (long long)m * ldd;
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-#pragma unroll
-                  for (int i = 0; i < 2; ++i) {
-                    const int n = nb + 8 * j + i;
-                    if (n < N) {
-                      float x = v[4 * j + 2 * e + i] + (bias ? __ldg(bias + n) : 0.f);
-                      if (sigm) x = 1.f / (1.f + __expf(-x));
-                      if (zrow) { const float z = __ldg(zrow + n); x *= z * (1.f - z); }
-                      x *= alpha;
-                      if (crow) x = fmaf(beta, __ldcg(crow + n), x);
-                      drow[n] = x;
-                    }
-                  }
-              }
             }
           }
         }
