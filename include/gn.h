@@ -368,9 +368,11 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
  * stored forward pass, the default, 2 = also the forward R pass of a product).  Option 5 (GN_FP32_ACCURATE contexts): the error-compensated kernel also writes the hi / lo parts
  * of a result that a later contraction takes as an operand (value 0 = a separate pass splits it).  Option 6: fixed-length
  * CG solves of small problems replay one captured step as a CUDA graph (value 0 = plain launches).  Option 7: the
- * weight blocks of the stored-factor block product as two chained halves of the subsample's rows (value 0 = one
- * contraction per block; the two forms differ in the order of two partial sums, i.e. by rounding).  Results do not
- * depend on options 0, 3, 4, 5 and 6 (tiles, sums and parts are computed identically); GN_EINVAL for an unknown option.
+ * weight blocks of the stored-factor block product as two chained parts of the subsample's rows (value 0 = one
+ * contraction per block; the two forms differ in the order of two partial sums, i.e. by rounding).  Option 8: the
+ * hidden layers of a backward pass (full product, gradient) as one chained launch (value 0 = one grouped launch
+ * per layer).  Results do not depend on options 0, 3, 4, 5, 6 and, with whole tiles (option 1 off), 8 (tiles, sums
+ * and parts are computed identically); GN_EINVAL for an unknown option.
  */
 gn_status gn_debug_option(gn_ctx* ctx, int option, int value);
 

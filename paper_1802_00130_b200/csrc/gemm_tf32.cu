@@ -1604,8 +1604,9 @@ int launch_gemm_tf32_group(const GemmArgs* gs, int n, const int* dep_prob, const
 // waves[k] = how many of them are whole waves (tiles q, q + pairs, ...), order[k] = index of that problem in the
 // caller's list, tiles[k] = its tile count.  keep_order != 0 keeps the caller's order (a chain).  Returns the number
 // of pairs the launch would use, or -1 for bad arguments.
-int gemm_tf32_plan_group(int n, const int* M, const int* N, const int* K, int pairs, int keep_order, int* counts,
-                         int* waves, int* order_out, int* tiles_out) {
+namespace {
+int plan_group_impl(int n, const int* M, const int* N, const int* K, int pairs, int keep_order, int* counts,
+                    int* waves, int* order_out, int* tiles_out, double* makespan) {
   if (n < 1 || n > MAX_GROUP || pairs < 1 || pairs > MAX_PAIRS_LAUNCH) return -1;
   GroupParams gp = {};
   struct Item { int src; double cost; };
@@ -1633,13 +1634,32 @@ int gemm_tf32_plan_group(int n, const int* M, const int* N, const int* K, int pa
   for (int k = 0; k < n; ++k) {
     gp.pr[k] = tmp[order[k].src];
     deal_tiles(gp, k, order[k].cost, P, load);
-    waves[k] = gp.pr[k].waves;
-    order_out[k] = order[k].src;
-    tiles_out[k] = gp.pr[k].tiles;
-    for (int q = 0; q < pairs; ++q)
-      counts[k * pairs + q] = q < P ? gp.pr[k].waves + (gp.rstart[k][q + 1] - gp.rstart[k][q]) : 0;
+    if (waves) waves[k] = gp.pr[k].waves;
+    if (order_out) order_out[k] = order[k].src;
+    if (tiles_out) tiles_out[k] = gp.pr[k].tiles;
+    if (counts)
+      for (int q = 0; q < pairs; ++q)
+        counts[k * pairs + q] = q < P ? gp.pr[k].waves + (gp.rstart[k][q + 1] - gp.rstart[k][q]) : 0;
+  }
+  if (makespan) {
+    *makespan = 0.0;
+    for (int q = 0; q < P; ++q) if (load[q] > *makespan) *makespan = load[q];
   }
   return P;
+}
+}  // namespace
+
+int gemm_tf32_plan_group(int n, const int* M, const int* N, const int* K, int pairs, int keep_order, int* counts,
+                         int* waves, int* order_out, int* tiles_out) {
+  return plan_group_impl(n, M, N, K, pairs, keep_order, counts, waves, order_out, tiles_out, nullptr);
+}
+
+// Load of the fullest CTA pair, in k-blocks of a 256-wide tile, if the problems went out as one grouped
+// (keep_order == 0) or chained launch on this device; negative for bad arguments.  Host arithmetic only.
+double gemm_tf32_group_makespan(int n, const int* M, const int* N, const int* K, int keep_order) {
+  double ms = 0.0;
+  if (plan_group_impl(n, M, N, K, num_sms() / 2, keep_order, nullptr, nullptr, nullptr, nullptr, &ms) < 0) return -1.0;
+  return ms;
 }
 
 // ---- error-compensated form ---------------------------------------------------------------------

@@ -86,7 +86,9 @@ struct gn_ctx {
   // pass (where it measured 8 % faster), 2 also the forward R pass of a product (where cutting left-over tiles along K,
   // which a chained launch does not do, measured as fast or faster)
   int chain_level = 1;
-  bool split_k_enabled = true; // weight blocks of the stored-factor product as two chained halves of the rows
+  bool split_k_enabled = true; // weight blocks of the stored-factor product as two chained parts of the rows
+  int64_t cut_for_nS = -1, cut_rows = 0;   // rows of the first part, chosen once per subsample size
+  bool back_chain_enabled = false;         // hidden layers of a backward pass as one chained launch (measured slower: off)
   int* chain_ctr = nullptr; int64_t chain_ctr_cap = 0;   // finished-tile counters of such a launch
   // FP32-accurate mode on the tensor cores (3 x TF32): hi / lo parts of the operands
   int acc_method = 0;        // 0 choose (tensor cores where the shape allows), 1 FP32 FMA only, 2 as 0
@@ -688,6 +690,52 @@ gn_status layer_backward(gn_ctx* c, int m, const float* ds_w, int64_t w_rows, co
   return GN_OK;
 }
 
+// Layers m_top .. 1 of a backward pass over `rows` rows, delta s^{m_top} = ds_top being complete: every layer's
+// activation gradient (Eqs. communi-g, ztox-g) into DSbuf[m - 1] and its weight and bias blocks (Eqs. xtow-g,
+// xtow-g-bias) into `out`.  In TF32 mode the contractions go out as ONE chain, [activation gradient, weight block] per
+// layer: an activation-gradient tile waits for the tiles of its row panel one layer up, a weight block for all of
+// them, and the pairs' loads are levelled over the whole pass instead of per layer (one ramp, one exposed
+// epilogue and one ragged last round instead of one per layer).  The bias sums of the layers below m_top can
+// then only start when the chain has ended.  zprev[m - 1] = z^{m-1}; layer 1 takes w1_rows rows (the caller adds
+// the rest) of an operand that is padded or not (w1_padded).
+gn_status backward_hidden_layers(gn_ctx* c, int m_top, const float* ds_top, const std::vector<const float*>& zprev,
+                                 std::vector<float*>& DSbuf, int64_t rows, float alpha, const float* cin, float beta,
+                                 float* out, int64_t w1_rows, bool w1_padded) {
+  if (m_top < 1) return GN_OK;
+  if (!(c->prec == GN_TF32 && c->back_chain_enabled && m_top >= 2)) {
+    const float* ds = ds_top;
+    for (int m = m_top; m >= 1; --m) {
+      const int64_t wr = m == 1 ? w1_rows : rows;
+      if (m == 1) GN_TRY(weight_block(c, 1, ds, zprev[0], wr, alpha, cin, beta, out, w1_padded));
+      else GN_TRY(layer_backward(c, m, ds, wr, ds, rows, zprev[(size_t)m - 1], rows, alpha, cin, beta, out, DSbuf[(size_t)m - 1]));
+      if (m > 1) ds = DSbuf[(size_t)m - 1];
+    }
+    return GN_OK;
+  }
+  std::vector<GemmArgs> gs;
+  std::vector<int> dep, dep_all;
+  GN_TRY(bias_block(c, m_top, ds_top, m_top == 1 ? w1_rows : rows, alpha, cin, beta, out));   // (its operand is ready now)
+  int producer = -1;                        // index of the problem that writes delta s^m
+  const float* ds = ds_top;
+  for (int m = m_top; m >= 1; --m) {
+    int next_producer = -1;
+    if (m > 1) {
+      gs.push_back(backward_data_args(c, m, ds, rows, zprev[(size_t)m - 1], rows, DSbuf[(size_t)m - 1], true));
+      dep.push_back(producer); dep_all.push_back(0);
+      next_producer = (int)gs.size() - 1;
+    }
+    gs.push_back(weight_block_args(c, m, ds, zprev[(size_t)m - 1], m == 1 ? w1_rows : rows, alpha, cin, beta, out,
+                                   m == 1 ? w1_padded : true));
+    dep.push_back(producer); dep_all.push_back(1);
+    producer = next_producer;
+    if (m > 1) ds = DSbuf[(size_t)m - 1];
+  }
+  run_gemm_chain(c, gs.data(), dep.data(), dep_all.data(), (int)gs.size());
+  for (int m = m_top - 1; m >= 1; --m)
+    GN_TRY(bias_block(c, m, DSbuf[(size_t)m], m == 1 ? w1_rows : rows, alpha, cin, beta, out));
+  return GN_OK;
+}
+
 // out = coef v + (1/|S|) J^T (2 J v) over the stored subsample (Eq. sampled-Gauss).
 gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
   GN_PHASE("G v");
@@ -716,12 +764,12 @@ gn_status product_full(gn_ctx* c, const float* v, float* out, float coef) {
     }
     run_gemm_chain(c, gs.data(), dep.data(), dep_all.data(), L, 2);
   }
-  const float* ds = c->RZ[L];
   const float inv = (float)(1.0 / (double)nS);
-  for (int m = L; m >= 1; --m) {
-    GN_TRY(layer_backward(c, m, ds, nS, ds, nS, c->Z[m - 1], nS, inv, v, coef, out, m > 1 ? c->DS[m - 1] : nullptr));
-    if (m > 1) ds = c->DS[m - 1];
-  }
+  std::vector<const float*> zprev((size_t)L);
+  for (int m = 1; m <= L; ++m) zprev[(size_t)m - 1] = c->Z[m - 1];
+  // the output layer (streaming kernels at n_L <= 16) on its own, the hidden layers as one pass
+  GN_TRY(layer_backward(c, L, c->RZ[L], nS, c->RZ[L], nS, c->Z[L - 1], nS, inv, v, coef, out, L > 1 ? c->DS[L - 1] : nullptr));
+  if (L > 1) GN_TRY(backward_hidden_layers(c, L - 1, c->DS[L - 1], zprev, c->DS, nS, inv, v, coef, out, nS, true));
   return check_launch(c, "G v");
 }
 
@@ -855,16 +903,34 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
     c->launches += launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], 1, 1, 0, c->DS[m], c->st);
   // 3. the weight and bias blocks.  The weight blocks are few long tiles (64 of 375 k-blocks per 2000 x 2000 layer at
   // |S| = 12000: 160 tiles on 74 pairs for three layers leave a third of the last round idle), so with a long enough
-  // K each block is cut into its two halves of the rows: the first half writes alpha Z^T Q + beta v, the second adds
-  // its alpha Z^T Q to that (a chained launch: a second-half tile waits for the first-half tiles of its row panel).
-  // Twice as many tiles of half the length fill the rounds better; the order of the two partial sums is fixed.
+  // K each block is cut into two parts of the rows: the first writes alpha Z^T Q + beta v, the second adds
+  // its alpha Z^T Q to that (a chained launch: a second-part tile waits for the first-part tiles of its row panel).
+  // More and shorter tiles fill the rounds better, and a short second part fills them best (the long tiles go
+  // first, the short ones level the loads): the cut is the one of 1/2, 5/8, 3/4 of the rows for which the host's
+  // work list comes out shortest.  The order of the two partial sums is fixed.
   const bool halves = c->prec == GN_TF32 && c->chain_level >= 1 && c->split_k_enabled && nS >= 4096 && L - 1 >= 1 && L - 1 <= kGroup;
   if (halves) {
     GemmArgs gs[2 * kGroup];
     int dep[2 * kGroup], dep_all[2 * kGroup];
     int n = 0;
-    const int64_t h0 = (nS / 2 + 31) / 32 * 32;              // first half: a whole number of k-blocks
     const int nl = L - 1;                                     // the hidden layers' blocks (the n_L-row block is a streaming kernel)
+    if (c->cut_for_nS != nS) {
+      double best = -1.0;
+      for (int eighths = 4; eighths <= 6; ++eighths) {
+        const int64_t r = (nS * eighths / 8 + 31) / 32 * 32;  // first part: a whole number of k-blocks
+        int Ms[2 * kGroup], Ns[2 * kGroup], Ks[2 * kGroup];
+        for (int part = 0; part < 2; ++part)
+          for (int m = 1; m <= nl; ++m) {
+            const int k = part * nl + m - 1;
+            Ms[k] = c->w[m]; Ns[k] = c->w[m - 1]; Ks[k] = (int)(part == 0 ? r : nS - r);
+          }
+        const double t = gemm_tf32_group_makespan(2 * nl, Ms, Ns, Ks, 1);
+        if (t >= 0.0 && (best < 0.0 || t < best)) { best = t; c->cut_rows = r; }
+      }
+      if (best < 0.0) c->cut_rows = (nS / 2 + 31) / 32 * 32;
+      c->cut_for_nS = nS;
+    }
+    const int64_t h0 = c->cut_rows;
     for (int part = 0; part < 2; ++part)
       for (int m = 1; m <= nl; ++m) {
         const int64_t r0 = part == 0 ? 0 : h0, rows = part == 0 ? h0 : nS - h0;
@@ -1020,23 +1086,23 @@ gn_status fun_grad(gn_ctx* c, float* d_grad, double* f_host) {
     }
     if (d_grad) {
       SideJoin side_guard(c);     // the next batch overwrites what the side stream reads
-      for (int m = L; m >= 1; --m) {
-        const float* Zprev = m == 1 ? X0 : c->Zb[m - 1];
-        const float* cin0 = b == 0 ? c->theta : d_grad;
-        const float beta0 = b == 0 ? inv_C : 1.f;
-        if (m == 1 && r0 + rows == c->l && rows > 64) {
-          // layer 1 reads the caller's X, which has no slack after its last row: all but the final 32
-          // rows use the padded fast path, the rest is added by a second, unpadded contraction
-          const int64_t head = rows - 32;
-          GN_TRY(weight_block(c, 1, c->Db[1], X0, head, inv_l, cin0, beta0, d_grad, true));
-          GN_TRY(weight_block(c, 1, c->Db[1] + head * c->w[1], X0 + head * c->w[0], 32, inv_l, d_grad, 1.f, d_grad, false));
-        } else if (m == 1) {
-          GN_TRY(weight_block(c, 1, c->Db[1], Zprev, rows, inv_l, cin0, beta0, d_grad, r0 + rows != c->l));
-        } else {
-          GN_TRY(layer_backward(c, m, c->Db[m], rows, c->Db[m], rows, c->Zb[m - 1], rows, inv_l, cin0, beta0, d_grad,
-                                c->Db[m - 1]));
-        }
+      const float* cin0 = b == 0 ? c->theta : d_grad;
+      const float beta0 = b == 0 ? inv_C : 1.f;
+      std::vector<const float*> zprev((size_t)L);
+      for (int m = 1; m <= L; ++m) zprev[(size_t)m - 1] = m == 1 ? X0 : c->Zb[m - 1];
+      // layer 1 reads the caller's X, which has no slack after its last row: in the last batch all but the final
+      // 32 rows use the padded fast path, the rest is added by a second, unpadded contraction
+      const bool last = r0 + rows == c->l;
+      const bool tail = last && rows > 64;
+      const int64_t head = tail ? rows - 32 : rows;
+      if (L > 1) {
+        GN_TRY(layer_backward(c, L, c->Db[L], rows, c->Db[L], rows, c->Zb[L - 1], rows, inv_l, cin0, beta0, d_grad, c->Db[L - 1]));
+        GN_TRY(backward_hidden_layers(c, L - 1, c->Db[L - 1], zprev, c->Db, rows, inv_l, cin0, beta0, d_grad, head, tail || !last));
+      } else {
+        GN_TRY(weight_block(c, 1, c->Db[1], X0, head, inv_l, cin0, beta0, d_grad, tail || !last));
       }
+      if (tail)
+        GN_TRY(weight_block(c, 1, c->Db[1] + head * c->w[1], X0 + head * c->w[0], 32, inv_l, d_grad, 1.f, d_grad, false));
     }
   }
   if (f_host) {
@@ -1697,6 +1763,7 @@ gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   if (option == 2) { if (value < 0) return fail(c, GN_EINVAL, "count must be >= 0"); c->fail_alloc_in = value; return GN_OK; }
   if (option == 3) { quiesce(c); c->side_enabled = value != 0; return GN_OK; }
   if (option == 7) { c->split_k_enabled = value != 0; return GN_OK; }
+  if (option == 8) { c->back_chain_enabled = value != 0; return GN_OK; }
   if (option == 6) { c->graph_enabled = value != 0; return GN_OK; }
   if (option == 5) { c->parts_enabled = value != 0; return GN_OK; }
   if (option == 4) { c->chain_level = value < 0 ? 0 : (value > 2 ? 2 : value); return GN_OK; }

@@ -82,6 +82,7 @@ int launch_gemm_tf32_group(const GemmArgs* gs, int n, const int* dep_prob, const
 // The work list of such a launch, computed without a device (see gemm_tf32.cu); for tests of the host logic.
 int gemm_tf32_plan_group(int n, const int* M, const int* N, const int* K, int pairs, int keep_order, int* counts,
                          int* waves, int* order_out, int* tiles_out);
+double gemm_tf32_group_makespan(int n, const int* M, const int* N, const int* K, int keep_order);
 
 // Streaming FP32 kernels for contractions with one dimension <= 16 (the n_L-wide output layer).
 // gemm_thin_kind says which of them (if any) takes a problem; THIN_M needs a scratch buffer of

@@ -25,12 +25,13 @@ def test_grouped_launches_give_the_bits_of_single_launches(name):
     import torch
     p = CASES[name]()
     outs = []
-    for grouped, side, chain in ((0, 0, 0), (1, 1, 2), (1, 0, 0), (0, 1, 1), (0, 0, 2)):
+    for grouped, side, chain, back in ((0, 0, 0, 0), (1, 1, 2, 1), (1, 0, 0, 0), (0, 1, 1, 1), (0, 0, 2, 0), (0, 0, 1, 1)):
         ctx = make_ctx(p, "tf32")
         ctx.debug_option(1, 0)                  # whole tiles only in every run: K slices change the order of sums
         ctx.debug_option(0, grouped)
         ctx.debug_option(3, side)
         ctx.debug_option(4, chain)
+        ctx.debug_option(8, back)               # hidden layers of a backward pass as one chained launch
         ctx.set_subsample(dev(p["idx"]))
         v = dev(p["v"])
         res = [ctx.Gv(v).clone()]
