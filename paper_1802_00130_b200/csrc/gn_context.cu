@@ -655,8 +655,10 @@ gn_status bias_block(gn_ctx* c, int m, const float* ds, int64_t rows, float alph
 
 gn_status weight_block(gn_ctx* c, int m, const float* ds, const float* Zprev, int64_t rows, float alpha,
                        const float* cin, float beta, float* out, bool padded = true) {
+  // (the bias sums first: forked to the side stream before the contraction is enqueued, they run beside it)
+  GN_TRY(bias_block(c, m, ds, rows, alpha, cin, beta, out));
   run_gemm(c, weight_block_args(c, m, ds, Zprev, rows, alpha, cin, beta, out, padded));
-  return bias_block(c, m, ds, rows, alpha, cin, beta, out);
+  return GN_OK;
 }
 
 // Activation-space half (Eq. communi-g / communi-jaco followed by Eq. ztox-g):
@@ -806,23 +808,25 @@ gn_status product_blockdiag(gn_ctx* c, const float* v, float* out, float coef) {
   const int L = c->L;
   const int64_t nS = c->nS;
   for (int k = 1; k <= L; ++k) {
+    // the streams that entered below layer k move up one layer; stream k enters (disjoint rows of R z^k: independent)
+    GemmArgs gs[2];
+    int n = 0;
     if (k > 1) {
-      GemmArgs g;
+      GemmArgs& g = gs[n++];
       g.M = (int)((k - 1) * nS); g.N = c->w[k];
       g.A1 = c->RZ[k - 1]; g.lda1 = c->w[k - 1]; g.B1 = Wm(c, c->theta, k); g.ldb1 = c->w[k - 1]; g.K1 = c->w[k - 1];
       if (k < L) { g.dsig = c->Z[k]; g.ld_dsig = c->w[k]; g.dsig_rows = (int)nS; }
       else g.alpha = 2.f;
       g.D = c->RZ[k]; g.ldd = c->w[k];
-      run_gemm(c, g);
     }
-    GemmArgs g;
+    GemmArgs& g = gs[n++];
     g.M = (int)nS; g.N = c->w[k];
     g.A1 = c->Z[k - 1]; g.lda1 = c->w[k - 1]; g.B1 = Wm(c, v, k); g.ldb1 = c->w[k - 1]; g.K1 = c->w[k - 1];
     g.bias = bm(c, v, k);
     if (k < L) { g.dsig = c->Z[k]; g.ld_dsig = c->w[k]; g.dsig_rows = (int)nS; }
     else g.alpha = 2.f;
     g.D = c->RZ[k] + (k - 1) * nS * c->w[k]; g.ldd = c->w[k];
-    run_gemm(c, g);
+    run_gemm_group(c, gs, n);
   }
   const float* cur = c->RZ[L];
   const float inv = (float)(1.0 / (double)nS);
@@ -901,7 +905,11 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
   // 2. q_i = D_i^T 2 D_i u_i per sample (Eqs. direct-JV-cost, JTv)
   for (int m = 1; m < L; ++m)
     c->launches += launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], 1, 1, 0, c->DS[m], c->st);
-  // 3. the weight and bias blocks.  The weight blocks are few long tiles (64 of 375 k-blocks per 2000 x 2000 layer at
+  // 3. the weight and bias blocks.  The bias sums and the n_L-row weight block go first: they run on the side
+  // stream beside the large weight blocks, which is only possible if they are forked before those are enqueued.
+  for (int m = 1; m <= L; ++m)
+    GN_TRY(bias_block(c, m, m < L ? c->DS[m] : c->RZ[m], nS, inv, v, coef, out));
+  // The weight blocks are few long tiles (64 of 375 k-blocks per 2000 x 2000 layer at
   // |S| = 12000: 160 tiles on 74 pairs for three layers leave a third of the last round idle), so with a long enough
   // K each block is cut into two parts of the rows: the first writes alpha Z^T Q + beta v, the second adds
   // its alpha Z^T Q to that (a chained launch: a second-part tile waits for the first-part tiles of its row panel).
@@ -940,8 +948,8 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
         dep_all[n] = 0;
         gs[n++] = g;
       }
-    run_gemm_chain(c, gs, dep, dep_all, n);
     run_gemm(c, weight_block_args(c, L, c->RZ[L], c->Z[L - 1], nS, inv, v, coef, out));
+    run_gemm_chain(c, gs, dep, dep_all, n);
   } else {
     for (int m0 = 1; m0 <= L; m0 += kGroup) {
       GemmArgs gs[kGroup];
@@ -951,8 +959,6 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
       run_gemm_group(c, gs, n);
     }
   }
-  for (int m = 1; m <= L; ++m)
-    GN_TRY(bias_block(c, m, m < L ? c->DS[m] : c->RZ[m], nS, inv, v, coef, out));
   return check_launch(c, "block-diagonal G v (stored factors)");
 }
 
