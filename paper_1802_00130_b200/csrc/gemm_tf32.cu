@@ -978,6 +978,54 @@ struct X3Params {
   int chunk_kb;
 };
 
+// One whole, 16-byte-aligned chunk of 32 finished sums of a row (lane = row) through the epilogue options and out,
+// with the options fixed at compile time as in epilogue_full_chunk: 0 = alpha * sum (+ bias), 1 = sigmoid,
+// 2 = times the sigmoid derivative of zrow, 3 = plus beta * crow, 4 = any combination, tested per element.  In modes
+// 2 and 3 the 128 bytes of the operand are requested before the first of them is used (the running sums of the
+// other chunks leave room for that one buffer); in mode 4 the loads stay beside their use, two steps at a time.
+template <int MODE>
+__device__ __forceinline__ void x3_store_chunk(const Tf32Params& p, const float* run, const float* zrow, const float* crow,
+                                               float* drow, int nb, float* hrow, float* lrow) {
+  const bool use_sigm = MODE == 4 ? p.sigmoid != 0 : MODE == 1;
+  const bool use_dsig = MODE == 4 ? zrow != nullptr : MODE == 2;
+  const bool use_cin = MODE == 4 ? crow != nullptr : MODE == 3;
+  float4 op[8];
+  if (MODE == 2 || MODE == 3) {
+    const float4* src = reinterpret_cast<const float4*>(MODE == 2 ? zrow : crow);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) op[q] = __ldg(src + q);
+  }
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    float4 bz = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.bias) bz = __ldg(reinterpret_cast<const float4*>(p.bias + nb) + q);
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f), o2 = o;
+    if (MODE == 2 || MODE == 3) o = op[q];
+    if (MODE == 4 && use_dsig) o = __ldg(reinterpret_cast<const float4*>(zrow) + q);
+    if (MODE == 4 && use_cin) o2 = __ldg(reinterpret_cast<const float4*>(crow) + q);
+    float x[4] = {run[4 * q] + bz.x, run[4 * q + 1] + bz.y, run[4 * q + 2] + bz.z, run[4 * q + 3] + bz.w};
+    const float z[4] = {o.x, o.y, o.z, o.w};
+    const float cv[4] = {MODE == 4 ? o2.x : o.x, MODE == 4 ? o2.y : o.y, MODE == 4 ? o2.z : o.z, MODE == 4 ? o2.w : o.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (use_sigm) x[e] = 1.f / (1.f + expf(-x[e]));
+      if (use_dsig) x[e] *= z[e] * (1.f - z[e]);
+      x[e] *= p.alpha;
+      if (use_cin) x[e] = fmaf(p.beta, cv[e], x[e]);
+    }
+    reinterpret_cast<float4*>(drow)[q] = make_float4(x[0], x[1], x[2], x[3]);
+    if (hrow) {
+      float h[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { h[e] = round_tf32(x[e]); x[e] = round_tf32(x[e] - h[e]); }
+      reinterpret_cast<float4*>(hrow)[q] = make_float4(h[0], h[1], h[2], h[3]);
+      reinterpret_cast<float4*>(lrow)[q] = make_float4(x[0], x[1], x[2], x[3]);
+    }
+    // the running sums leave few registers: keep the loads of at most two steps in flight
+    if (MODE == 4 && (q & 1)) asm volatile("" ::: "memory");
+  }
+}
+
 template <int STAGES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(X3_THREADS, 1)
 gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, const X3Params xp) {
@@ -1144,38 +1192,22 @@ gemm_tf32x3_kernel(const __grid_constant__ MapSet maps, const Tf32Params p, cons
       const float* zrow = p.dsig ? p.dsig + (long long)((m / p.dsig_div) % p.dsig_rows) * p.ld_dsig : nullptr;
       const float* crow = p.cin ? p.cin + (long long)m * p.ld_cin : nullptr;
       float* drow = p.D + (long long)m * p.ldd;
+      const int n_opt = (p.sigmoid ? 1 : 0) + (p.dsig ? 1 : 0) + (p.cin ? 1 : 0);
+      const int xmode = n_opt == 0 ? 0 : n_opt > 1 ? 4 : p.sigmoid ? 1 : p.dsig ? 2 : 3;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int c = half + 2 * j;
         if (c >= n_cc) continue;
         const int nb = n0 + c * 32;
         if (p.vec_epi && nb + 32 <= p.N) {
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            float4 bz = make_float4(0.f, 0.f, 0.f, 0.f), zc = bz, cc = bz;
-            if (p.bias) bz = __ldg(reinterpret_cast<const float4*>(p.bias + nb) + q);
-            if (zrow) zc = __ldg(reinterpret_cast<const float4*>(zrow + nb) + q);
-            if (crow) cc = __ldg(reinterpret_cast<const float4*>(crow + nb) + q);
-            float x[4] = {run[j][4 * q] + bz.x, run[j][4 * q + 1] + bz.y, run[j][4 * q + 2] + bz.z, run[j][4 * q + 3] + bz.w};
-            const float z[4] = {zc.x, zc.y, zc.z, zc.w};
-            const float cv[4] = {cc.x, cc.y, cc.z, cc.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              if (p.sigmoid) x[e] = 1.f / (1.f + expf(-x[e]));
-              if (zrow) x[e] *= z[e] * (1.f - z[e]);
-              x[e] *= p.alpha;
-              if (crow) x[e] = fmaf(p.beta, cv[e], x[e]);
-            }
-            reinterpret_cast<float4*>(drow + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
-            if (p.Dhi) {
-              float h[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) { h[e] = round_tf32(x[e]); x[e] = round_tf32(x[e] - h[e]); }
-              reinterpret_cast<float4*>(p.Dhi + (long long)m * p.ld_parts + nb)[q] = make_float4(h[0], h[1], h[2], h[3]);
-              reinterpret_cast<float4*>(p.Dlo + (long long)m * p.ld_parts + nb)[q] = make_float4(x[0], x[1], x[2], x[3]);
-            }
-            // the running sums leave few registers: keep the loads of at most two steps in flight
-            if (q & 1) asm volatile("" ::: "memory");
+          float* const hrow = p.Dhi ? p.Dhi + (long long)m * p.ld_parts + nb : nullptr;
+          float* const lrow = p.Dhi ? p.Dlo + (long long)m * p.ld_parts + nb : nullptr;
+          switch (xmode) {
+            case 0: x3_store_chunk<0>(p, run[j], zrow ? zrow + nb : nullptr, crow ? crow + nb : nullptr, drow + nb, nb, hrow, lrow); break;
+            case 1: x3_store_chunk<1>(p, run[j], zrow ? zrow + nb : nullptr, crow ? crow + nb : nullptr, drow + nb, nb, hrow, lrow); break;
+            case 2: x3_store_chunk<2>(p, run[j], zrow ? zrow + nb : nullptr, crow ? crow + nb : nullptr, drow + nb, nb, hrow, lrow); break;
+            case 3: x3_store_chunk<3>(p, run[j], zrow ? zrow + nb : nullptr, crow ? crow + nb : nullptr, drow + nb, nb, hrow, lrow); break;
+            default: x3_store_chunk<4>(p, run[j], zrow ? zrow + nb : nullptr, crow ? crow + nb : nullptr, drow + nb, nb, hrow, lrow); break;
           }
         } else {
 #pragma unroll
