@@ -35,10 +35,10 @@ FP32_LANES_PER_SM, SMS = 128, 148
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant GEMM kernel from an ncu capture of the
 # kernel as it stands.  Multi-pass counters are only taken on the small case (|S| = 3000), so the figure belongs to
 # that workload; for every other workload `traffic` is None and the small-case figure is quoted beside it.
-TRAFFIC = {("tf32", "mnist2000_5"): {"bytes_per_launch": 150.4e6, "kernel": "gemm_tf32_2cta_kernel",
+TRAFFIC = {("tf32", "mnist2000_5"): {"bytes_per_launch": 145.1e6, "kernel": "gemm_tf32_2cta_kernel",
                                      "launch": "forward R pass of a hidden layer, 3000 x 2000 x (2000 + 2000); 128 MB algorithmic",
                                      "source": "profiles/gemm_tf32_2cta_mnist2000_5_ncu.md"},
-           ("fp32", "mnist2000_5"): {"bytes_per_launch": 143.2e6, "kernel": "gemm_tf32x3_kernel",
+           ("fp32", "mnist2000_5"): {"bytes_per_launch": 144.4e6, "kernel": "gemm_tf32x3_kernel",
                                      "launch": "3000 x 2000 x 2000-class contraction on hi / lo parts",
                                      "source": "profiles/gemm_tf32x3_mnist2000_5_ncu.md"}}
 
