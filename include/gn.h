@@ -371,7 +371,7 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
  * weight blocks of the stored-factor block product as two chained parts of the subsample's rows (value 0 = one
  * contraction per block; the two forms differ in the order of two partial sums, i.e. by rounding).  Option 8: the
  * hidden layers of a backward pass (full product, gradient) as one chained launch (value 0 = one grouped launch
- * per layer).  Results do not depend on options 0, 3, 4, 5, 6 and, with whole tiles (option 1 off), 8 (tiles, sums
+ * per layer, 1 = always, 2 = for passes of few rows, where it is the faster form: the default).  Results do not depend on options 0, 3, 4, 5, 6 and, with whole tiles (option 1 off), 8 (tiles, sums
  * and parts are computed identically); GN_EINVAL for an unknown option.
  */
 gn_status gn_debug_option(gn_ctx* ctx, int option, int value);

@@ -88,7 +88,7 @@ struct gn_ctx {
   int chain_level = 1;
   bool split_k_enabled = true; // weight blocks of the stored-factor product as two chained parts of the rows
   int64_t cut_for_nS = -1, cut_rows = 0;   // rows of the first part, chosen once per subsample size
-  bool back_chain_enabled = false;         // hidden layers of a backward pass as one chained launch (measured slower: off)
+  int back_chain = 2;                      // hidden layers of a backward pass as one chained launch: 0 never, 1 always, 2 where it pays
   int* chain_ctr = nullptr; int64_t chain_ctr_cap = 0;   // finished-tile counters of such a launch
   // FP32-accurate mode on the tensor cores (3 x TF32): hi / lo parts of the operands
   int acc_method = 0;        // 0 choose (tensor cores where the shape allows), 1 FP32 FMA only, 2 as 0
@@ -704,7 +704,15 @@ gn_status backward_hidden_layers(gn_ctx* c, int m_top, const float* ds_top, cons
                                  std::vector<float*>& DSbuf, int64_t rows, float alpha, const float* cin, float beta,
                                  float* out, int64_t w1_rows, bool w1_padded) {
   if (m_top < 1) return GN_OK;
-  if (!(c->prec == GN_TF32 && c->back_chain_enabled && m_top >= 2)) {
+  // One launch instead of one per layer saves the ramp, the exposed last epilogue and the ragged last round of
+  // every layer, but it has to end with layer 1's weight block, whose tiles are as long as the pass has rows, and
+  // the lower layers' bias sums wait for all of it: measured at 784-2000-2000-2000-10, it wins below about 4000
+  // rows (full product 0.40 -> 0.37 ms at 1500 rows, 0.56 -> 0.52 at 3000; 784-300-300-10 0.161 -> 0.143) and loses
+  // above (0.94 -> 1.00 at 6000, 1.13 -> 1.30 at 8000).
+  int widest = 0;
+  for (int m = 1; m <= m_top; ++m) widest = std::max(widest, c->w[m]);
+  const bool chain = c->back_chain == 1 || (c->back_chain == 2 && (double)rows * widest <= 7.0e6);
+  if (!(c->prec == GN_TF32 && chain && m_top >= 2)) {
     const float* ds = ds_top;
     for (int m = m_top; m >= 1; --m) {
       const int64_t wr = m == 1 ? w1_rows : rows;
@@ -1769,7 +1777,7 @@ gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   if (option == 2) { if (value < 0) return fail(c, GN_EINVAL, "count must be >= 0"); c->fail_alloc_in = value; return GN_OK; }
   if (option == 3) { quiesce(c); c->side_enabled = value != 0; return GN_OK; }
   if (option == 7) { c->split_k_enabled = value != 0; return GN_OK; }
-  if (option == 8) { c->back_chain_enabled = value != 0; return GN_OK; }
+  if (option == 8) { c->back_chain = value < 0 ? 0 : (value > 2 ? 2 : value); return GN_OK; }
   if (option == 6) { c->graph_enabled = value != 0; return GN_OK; }
   if (option == 5) { c->parts_enabled = value != 0; return GN_OK; }
   if (option == 4) { c->chain_level = value < 0 ? 0 : (value > 2 ? 2 : value); return GN_OK; }
