@@ -357,6 +357,20 @@ gn_status gn_debug_gemm(gn_ctx* ctx, int kind, int M, int N, int K, const float*
                         int a_kmajor, const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd);
 
 /*
+ * gn_debug_gemm_epilogue - gn_debug_gemm with the epilogue options every contraction kernel of the path takes:
+ *   D = alpha * dsig'( f(A B + 1 bias^T) ) + beta * cin,
+ * f = logistic sigmoid if `sigmoid` != 0 (Eq. xtoz), else the identity; dsig'(x)_{mn} = x_{mn} z_{mn} (1 - z_{mn}) with
+ * z = d_dsig (the sigmoid derivative of Eq. ztox-g from stored activations) if d_dsig != NULL, else x; d_bias is
+ * [N], d_dsig and d_cin are [M][ld_*] row-major device arrays, each may be NULL (cin == NULL: no accumulate term).
+ * The path itself uses one option at a time (plus the bias); this hook lets a test put every combination through
+ * every kernel.  Errors as gn_debug_gemm; GN_EINVAL also for a leading dimension below N.
+ */
+gn_status gn_debug_gemm_epilogue(gn_ctx* ctx, int kind, int M, int N, int K, const float* dA, int64_t lda, int a_kmajor,
+                                 const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd, const float* d_bias,
+                                 int sigmoid, const float* d_dsig, int64_t ld_dsig, float alpha, const float* d_cin,
+                                 int64_t ld_cin, float beta);
+
+/*
  * gn_debug_option - test and measurement hook: switch a launch strategy of the context for A/B runs.
  * option 0: independent contractions of a layer issued as one launch of the CTA-pair kernel (value 0 =
  * one launch per contraction); option 1: cutting left-over tiles along K between CTA pairs (value 0 = whole

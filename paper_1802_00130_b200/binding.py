@@ -51,6 +51,8 @@ _SIGNATURES = {
     "gn_profile_read": (_i32, [_vp, C.POINTER(_dbl), C.POINTER(_dbl), C.POINTER(_i64)]),
     "gn_thin_m_gemm_noalloc": (_i32, [_i32, _i32, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp, C.c_char_p, _i64]),
     "gn_debug_gemm": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64]),
+    "gn_debug_gemm_epilogue": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _i64,
+                                      _vp, _i32, _vp, _i64, C.c_float, _vp, _i64, C.c_float]),
 }
 
 
@@ -342,6 +344,21 @@ class GnContext:
         self._check(self._lib.gn_debug_gemm(self._h, int(kind), M, N, K, _dev_ptr(A, torch.float32), A.stride(0),
                                             int(a_kmajor), _dev_ptr(B, torch.float32), B.stride(0), int(b_kmajor),
                                             _dev_ptr(D, torch.float32), D.stride(0)))
+        return D
+
+    def debug_gemm_epilogue(self, kind, A, B, a_kmajor=True, b_kmajor=True, bias=None, sigmoid=False, dsig=None,
+                            alpha=1.0, cin=None, beta=0.0):
+        """Test hook: debug_gemm with the epilogue options of the path's contraction kernels (see gn.h)."""
+        import torch
+        M, K = (A.shape if a_kmajor else A.shape[::-1])
+        N = B.shape[0] if b_kmajor else B.shape[1]
+        D = torch.empty((M, N), dtype=torch.float32, device=A.device)
+        ptr = lambda t: None if t is None else _dev_ptr(t, torch.float32)
+        self._check(self._lib.gn_debug_gemm_epilogue(
+            self._h, int(kind), M, N, K, _dev_ptr(A, torch.float32), A.stride(0), int(a_kmajor),
+            _dev_ptr(B, torch.float32), B.stride(0), int(b_kmajor), _dev_ptr(D, torch.float32), D.stride(0),
+            ptr(bias), int(bool(sigmoid)), ptr(dsig), 0 if dsig is None else dsig.stride(0), float(alpha),
+            ptr(cin), 0 if cin is None else cin.stride(0), float(beta)))
         return D
 
     def newton_iter(self, theta, idx, direction, params):

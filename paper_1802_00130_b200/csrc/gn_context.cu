@@ -1670,15 +1670,34 @@ gn_status gn_profile_read(gn_ctx* c, double* gemm_ms, double* gemm_flop, int64_t
   return GN_OK;
 }
 
+static gn_status debug_gemm_impl(gn_ctx* c, int kind, GemmArgs g);
+
 gn_status gn_debug_gemm(gn_ctx* c, int kind, int M, int N, int K, const float* dA, int64_t lda, int a_kmajor,
                         const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd) {
+  return gn_debug_gemm_epilogue(c, kind, M, N, K, dA, lda, a_kmajor, dB, ldb, b_kmajor, dD, ldd, nullptr, 0, nullptr, 0,
+                                1.f, nullptr, 0, 0.f);
+}
+
+gn_status gn_debug_gemm_epilogue(gn_ctx* c, int kind, int M, int N, int K, const float* dA, int64_t lda, int a_kmajor,
+                                 const float* dB, int64_t ldb, int b_kmajor, float* dD, int64_t ldd, const float* d_bias,
+                                 int sigmoid, const float* d_dsig, int64_t ld_dsig, float alpha, const float* d_cin,
+                                 int64_t ld_cin, float beta) {
   if (!c) return GN_EINVAL;
   if (!dA || !dB || !dD || M < 1 || N < 1 || K < 1 || kind < 0 || kind > 7) return fail(c, GN_EINVAL, "bad GEMM arguments");
+  if ((d_dsig && ld_dsig < N) || (d_cin && ld_cin < N)) return fail(c, GN_EINVAL, "leading dimension of an epilogue operand below N");
   GemmArgs g;
   g.M = M; g.N = N; g.K1 = K;
   g.A1 = dA; g.lda1 = lda; g.a_kmajor = a_kmajor != 0;
   g.B1 = dB; g.ldb1 = ldb; g.b_kmajor = b_kmajor != 0;
   g.D = dD; g.ldd = ldd;
+  g.bias = d_bias; g.sigmoid = sigmoid != 0;
+  if (d_dsig) { g.dsig = d_dsig; g.ld_dsig = ld_dsig; g.dsig_rows = M; }
+  g.alpha = alpha;
+  if (d_cin) { g.cin = d_cin; g.ld_cin = ld_cin; g.beta = beta; }
+  return debug_gemm_impl(c, kind, g);
+}
+
+static gn_status debug_gemm_impl(gn_ctx* c, int kind, GemmArgs g) {
   // kinds 3..6 are the tensor-core kernel with options: 3 = MN-major operands declared padded,
   // 4 = one CTA per tile forced, 5 = CTA pair per tile forced, 6 = as 5 without splitting tiles
   // between pairs (all with padded operands)
