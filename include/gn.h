@@ -385,7 +385,9 @@ gn_status gn_debug_gemm_epilogue(gn_ctx* ctx, int kind, int M, int N, int K, con
  * weight blocks of the stored-factor block product as two chained parts of the subsample's rows (value 0 = one
  * contraction per block; the two forms differ in the order of two partial sums, i.e. by rounding).  Option 8: the
  * hidden layers of a backward pass (full product, gradient) as one chained launch (value 0 = one grouped launch
- * per layer, 1 = always, 2 = for passes of few rows, where it is the faster form: the default).  Results do not depend on options 0, 3, 4, 5, 6 and, with whole tiles (option 1 off), 8 (tiles, sums
+ * per layer, 1 = always, 2 = for passes of few rows, where it is the faster form: the default).  Option 9: in the
+ * stored-factor block product the factor of the last hidden layer, W^L * sigma'(z^{L-1}), is formed on the fly from
+ * W^L and the stored activations instead of being read back (value 0 = read back; same bits either way).  Results do not depend on options 0, 3, 4, 5, 6, 9 and, with whole tiles (option 1 off), 8 (tiles, sums
  * and parts are computed identically); GN_EINVAL for an unknown option.
  */
 gn_status gn_debug_option(gn_ctx* ctx, int option, int value);

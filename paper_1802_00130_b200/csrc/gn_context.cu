@@ -88,6 +88,7 @@ struct gn_ctx {
   int chain_level = 1;
   bool split_k_enabled = true; // weight blocks of the stored-factor product as two chained parts of the rows
   int64_t cut_for_nS = -1, cut_rows = 0;   // rows of the first part, chosen once per subsample size
+  bool fly_enabled = true;                 // last hidden layer's factor formed on the fly in the stored-factor product
   int back_chain = 2;                      // hidden layers of a backward pass as one chained launch: 0 never, 1 always, 2 where it pays
   int* chain_ctr = nullptr; int64_t chain_ctr_cap = 0;   // finished-tile counters of such a launch
   // FP32-accurate mode on the tensor cores (3 x TF32): hi / lo parts of the operands
@@ -911,8 +912,15 @@ gn_status product_blockdiag_stored(gn_ctx* c, const float* v, float* out, float 
     run_gemm_group(c, gs, n);
   }
   // 2. q_i = D_i^T 2 D_i u_i per sample (Eqs. direct-JV-cost, JTv)
-  for (int m = 1; m < L; ++m)
-    c->launches += launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], 1, 1, 0, c->DS[m], c->st);
+  // (the factor of the last hidden layer is W^L * sigma'(z^{L-1}): formed on the fly where the kernel allows it,
+  // the stored copy being needed only as the operand of the recurrence that builds the factors below it)
+  for (int m = 1; m < L; ++m) {
+    int done = 0;
+    if (m == L - 1 && c->fly_enabled)
+      done = launch_factor_apply_last(Wm(c, c->theta, L), c->Z[L - 1], c->RZ[m], nS, nL, c->w[m], c->DS[m], c->st);
+    if (!done) done = launch_factor_apply(c->DF[m], c->RZ[m], nS, nL, c->w[m], 1, 1, 0, c->DS[m], c->st);
+    c->launches += done;
+  }
   // 3. the weight and bias blocks.  The bias sums and the n_L-row weight block go first: they run on the side
   // stream beside the large weight blocks, which is only possible if they are forked before those are enqueued.
   for (int m = 1; m <= L; ++m)
@@ -1797,6 +1805,7 @@ gn_status gn_debug_option(gn_ctx* c, int option, int value) {
   if (option == 3) { quiesce(c); c->side_enabled = value != 0; return GN_OK; }
   if (option == 7) { c->split_k_enabled = value != 0; return GN_OK; }
   if (option == 8) { c->back_chain = value < 0 ? 0 : (value > 2 ? 2 : value); return GN_OK; }
+  if (option == 9) { c->fly_enabled = value != 0; return GN_OK; }
   if (option == 6) { c->graph_enabled = value != 0; return GN_OK; }
   if (option == 5) { c->parts_enabled = value != 0; return GN_OK; }
   if (option == 4) { c->chain_level = value < 0 ? 0 : (value > 2 ? 2 : value); return GN_OK; }

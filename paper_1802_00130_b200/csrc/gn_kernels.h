@@ -133,6 +133,8 @@ int launch_factor_last(const float* WL, const float* Zprev, int64_t rows, int nL
 // (Eqs. direct-JV-cost, JTv; B = 2I).  n_L <= 32.
 int launch_factor_apply(const float* D, const float* U, int64_t rows, int nL, int n, int groups, int streams,
                         int64_t stream_stride, float* Q, cudaStream_t st);
+int launch_factor_apply_last(const float* WL, const float* Zprev, const float* U, int64_t rows, int nL, int n, float* Q,
+                             cudaStream_t st);
 
 // ---- conjugate gradient ------------------------------------------------------------------------
 // The n coordinates are cut into chunks, each inside one segment (one segment for the full system,

@@ -540,11 +540,15 @@ int launch_sum_partials(const double* partial, int count, double* out, bool accu
 
 // Register-resident form for groups of at most 1024 * STRIPS columns (n and every group boundary multiples
 // of 4): every thread keeps its n_L x 4 x STRIPS slice of D_i in registers across the passes and the streams,
-// so D is read exactly once.
-template <int NLMAX, int STRIPS>
+// so D is read exactly once.  FLY: the factor of the last hidden layer has the closed form D_i[u][t] = W^L[u][t] *
+// z (1 - z) (what factor_last_kernel stores); it is formed here, with the same two multiplications, from W^L (80 KB,
+// cache-resident) and the sample's row of Z instead of being streamed from memory: 8 KB instead of 80 KB per sample
+// at n_L = 10, the same bits.
+template <int NLMAX, int STRIPS, bool FLY>
 __global__ void __launch_bounds__(256) factor_apply_reg_kernel(const float* __restrict__ D, const float* __restrict__ U,
                                                                int nL, int n, int groups, int streams,
-                                                               long long stream_stride, float* __restrict__ Q) {
+                                                               long long stream_stride, float* __restrict__ Q,
+                                                               const float* __restrict__ WL, const float* __restrict__ Zprev) {
   __shared__ float red[8][NLMAX];
   __shared__ float pu[NLMAX];
   const long long i = blockIdx.x;
@@ -556,9 +560,23 @@ __global__ void __launch_bounds__(256) factor_apply_reg_kernel(const float* __re
   for (int s = 0; s < STRIPS; ++s) {
     const int j = col0 + (s * 256 + threadIdx.x) * 4;
     const bool ok = j < col1;
+    if (FLY) {
+      float4 ds = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (ok) {
+        const float4 z = __ldg(reinterpret_cast<const float4*>(Zprev + i * n + j));
+        ds = make_float4(z.x * (1.f - z.x), z.y * (1.f - z.y), z.z * (1.f - z.z), z.w * (1.f - z.w));
+      }
 #pragma unroll
-    for (int u = 0; u < NLMAX; ++u)
-      dv[s][u] = (ok && u < nL) ? __ldg(reinterpret_cast<const float4*>(d + (long long)u * n + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int u = 0; u < NLMAX; ++u) {
+        float4 wv = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ok && u < nL) wv = __ldg(reinterpret_cast<const float4*>(WL + (long long)u * n + j));
+        dv[s][u] = make_float4(wv.x * ds.x, wv.y * ds.y, wv.z * ds.z, wv.w * ds.w);
+      }
+    } else {
+#pragma unroll
+      for (int u = 0; u < NLMAX; ++u)
+        dv[s][u] = (ok && u < nL) ? __ldg(reinterpret_cast<const float4*>(d + (long long)u * n + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
   }
   for (int a = 0; a < streams; ++a) {
     const float* u_row = U + a * stream_stride + i * n;
@@ -621,7 +639,7 @@ int launch_factor_apply(const float* D, const float* U, int64_t rows, int nL, in
   }
   const dim3 grid((unsigned)rows, (unsigned)groups);
   const long long ss = stream_stride;
-#define GN_FA_REG(NL, STR) { factor_apply_reg_kernel<NL, STR><<<grid, 256, 0, st>>>(D, U, nL, n, groups, streams, ss, Q); return 1; }
+#define GN_FA_REG(NL, STR) { factor_apply_reg_kernel<NL, STR, false><<<grid, 256, 0, st>>>(D, U, nL, n, groups, streams, ss, Q, nullptr, nullptr); return 1; }
   if (vec && widest <= 1024 && nL <= 4)  GN_FA_REG(4, 1)
   if (vec && widest <= 1024 && nL <= 10) GN_FA_REG(10, 1)
   if (vec && widest <= 2048 && nL <= 4)  GN_FA_REG(4, 2)
@@ -633,6 +651,24 @@ int launch_factor_apply(const float* D, const float* U, int64_t rows, int nL, in
   else if (nL <= 16) factor_apply_kernel<16><<<grid, 256, 0, st>>>(D, U, nL, n, groups, streams, ss, Q);
   else factor_apply_kernel<32><<<grid, 256, 0, st>>>(D, U, nL, n, groups, streams, ss, Q);
   return 1;
+}
+
+// The same product for the last hidden layer without its stored factor (see factor_apply_reg_kernel): one group, one
+// stream.  Returns 0, having launched nothing, if the register-resident form does not take the shape.
+int launch_factor_apply_last(const float* WL, const float* Zprev, const float* U, int64_t rows, int nL, int n, float* Q,
+                             cudaStream_t st) {
+  const bool vec = (n % 4 == 0) && ((reinterpret_cast<uintptr_t>(WL) & 15) == 0) && ((reinterpret_cast<uintptr_t>(Zprev) & 15) == 0) &&
+                   ((reinterpret_cast<uintptr_t>(U) & 15) == 0) && ((reinterpret_cast<uintptr_t>(Q) & 15) == 0);
+  if (!vec) return 0;
+  const dim3 grid((unsigned)rows, 1);
+#define GN_FA_FLY(NL, STR) { factor_apply_reg_kernel<NL, STR, true><<<grid, 256, 0, st>>>(nullptr, U, nL, n, 1, 1, 0, Q, WL, Zprev); return 1; }
+  if (n <= 1024 && nL <= 4)  GN_FA_FLY(4, 1)
+  if (n <= 1024 && nL <= 10) GN_FA_FLY(10, 1)
+  if (n <= 2048 && nL <= 4)  GN_FA_FLY(4, 2)
+  if (n <= 2048 && nL <= 10) GN_FA_FLY(10, 2)
+  if (n <= 1024 && nL <= 16) GN_FA_FLY(16, 1)
+#undef GN_FA_FLY
+  return 0;
 }
 
 int launch_axpby(int64_t n, float a, const float* x, float b, const float* y, float* out, cudaStream_t st) {

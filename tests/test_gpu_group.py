@@ -179,3 +179,23 @@ def test_weight_blocks_of_the_stored_factor_product_in_two_chained_halves():
     # ... and differs by rounding only: the tensor core adds into its FP32 accumulator with truncation (a relative bias
     # of about 1e-9 per term), so one accumulation over 5000 rows and two over 2500 differ by about 1e-5
     assert relb(outs[1][0], outs[0][0], p["widths"]) <= 1e-4
+
+
+@pytest.mark.parametrize("mode", ["tf32", "fp32"])
+@pytest.mark.parametrize("name", ["mid", "mnist2000_5", "svhn1000"])
+def test_last_factor_formed_on_the_fly_gives_the_bits_of_the_stored_one(name, mode):
+    """Stored-factor block product (Section 3.3.1 / 4.2): the factor of the last hidden layer has the closed form
+    W^L * sigma'(z^{L-1}); forming it inside the per-sample kernel gives the bits of reading the stored copy back."""
+    import torch
+    p = CASES[name]()
+    outs = []
+    for fly in (0, 1):
+        ctx = make_ctx(p, mode)
+        ctx.debug_option(9, fly)
+        ctx.set_blockdiag_method(2)
+        ctx.set_subsample(dev(p["idx"]))
+        outs.append(ctx.Gv_blockdiag(dev(p["v"])).clone())
+        ctx.close()
+    assert torch.equal(outs[0], outs[1])
+    ref = orc.Gv_blockdiag(p["theta"], p["widths"], p["C"], p["X"][p["idx"]], p["v"])
+    assert relb(outs[1].cpu().numpy(), ref, p["widths"]) <= TOL[mode]
