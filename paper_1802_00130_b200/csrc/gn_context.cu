@@ -594,8 +594,10 @@ gn_status ensure_partials(gn_ctx* c, int64_t count) {
   return GN_OK;
 }
 
+// Scratch of the column sums: two slots of equal size (slot 1 starts at colsum_cap / 2), so that the sums of two
+// layers can run at the same time on two streams.
 gn_status ensure_colsum(gn_ctx* c, int64_t rows, int cols) {
-  const int64_t need = colsum_scratch_floats(rows, cols);
+  const int64_t need = 2 * ((colsum_scratch_floats(rows, cols) + 3) / 4 * 4);
   if (need <= c->colsum_cap) return GN_OK;
   quiesce(c);
   dev_free(c, c->colsum_scratch, c->colsum_cap);
@@ -646,11 +648,12 @@ GemmArgs weight_block_args(const gn_ctx* c, int m, const float* ds, const float*
   return g;
 }
 
+// on_main: on the context's stream, in the second scratch slot, instead of the side stream and the first.
 gn_status bias_block(gn_ctx* c, int m, const float* ds, int64_t rows, float alpha, const float* cin, float beta,
-                     float* out) {
+                     float* out, bool on_main = false) {
   GN_TRY(ensure_colsum(c, rows, c->w[m]));
   c->launches += launch_colsum(ds, rows, c->w[m], c->w[m], alpha, cin + c->b_off[m], beta, out + c->b_off[m],
-                               c->colsum_scratch, side_fork(c));
+                               c->colsum_scratch + (on_main ? c->colsum_cap / 2 : 0), on_main ? c->st : side_fork(c));
   return GN_OK;
 }
 
@@ -742,8 +745,10 @@ gn_status backward_hidden_layers(gn_ctx* c, int m_top, const float* ds_top, cons
     if (m > 1) ds = DSbuf[(size_t)m - 1];
   }
   run_gemm_chain(c, gs.data(), dep.data(), dep_all.data(), (int)gs.size());
+  // (nothing is left to hide these sums behind: they alternate between the side stream and this one, each with its
+  // own scratch, so that two of them run at a time)
   for (int m = m_top - 1; m >= 1; --m)
-    GN_TRY(bias_block(c, m, DSbuf[(size_t)m], m == 1 ? w1_rows : rows, alpha, cin, beta, out));
+    GN_TRY(bias_block(c, m, DSbuf[(size_t)m], m == 1 ? w1_rows : rows, alpha, cin, beta, out, ((m_top - 1 - m) & 1) != 0));
   return GN_OK;
 }
 
